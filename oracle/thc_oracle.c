@@ -1,0 +1,329 @@
+/*
+ * THC oracle: a plain, slow CPU statement of one Tensor Homomorphic Compression round.
+ *
+ * TEST INFRASTRUCTURE ONLY.  Nothing in the product path may include, link or call this
+ * file; it shares no code with the CUDA library.  It exists so that tests can compare
+ * the CUDA path with something a reader can check against the paper by eye.
+ *
+ * What it follows (THC paper, arxiv 2302.08545):
+ *   - Randomized Hadamard Transform, Section 5.1:  RHT(x) = (1/sqrt(d)) H D x and
+ *     RHT^-1(x) = (1/sqrt(d)) D H x, with D a shared Rademacher diagonal ("D^r",
+ *     Algorithm 3 line "R_i = RHT(x_i)").
+ *   - Norm-based preliminary stage, Section 5.3 and Algorithm 3:
+ *     ell = max_i ||x_i||,  M = (t_p / sqrt(d)) * ell,  m = -M.
+ *   - Truncation (clamp to [m, M]), Section 5.1 / Algorithm 3 "Truncation".
+ *   - Stochastic quantization, Section 4.1: a in [q0, q1] goes to q0 with probability
+ *     (q1 - a)/(q1 - q0) and to q1 otherwise.
+ *   - Non-uniform THC, Algorithm 2: quantize onto the sub-grid {m + T[z] (M-m)/g},
+ *     send the table index z; the PS sums T[z_i]; the worker computes
+ *     m + (Y/n) (M-m)/g.
+ *   - Packing of indices and of the sum, Section 3 (THC overview).
+ *
+ * The paper leaves many things open (blocking, Hadamard ordering, the random source,
+ * the floating-point operation sequence, the bit layout).  The readings taken here:
+ *   R1  "d" of the paper is one RHT block of B = 2^k coordinates; the vector is
+ *       zero-padded to a multiple of B; every block has its own ell and M (max over
+ *       workers).  ell is the Euclidean norm (Algorithm 3), not its square.
+ *   R2  H is the Sylvester (natural order) Hadamard matrix, H[i][j] = (-1)^popcount(i&j).
+ *       H v is evaluated by radix-2 butterflies, stride 1 first, then 2, 4, ... B/2,
+ *       in fp32; the factor c_B = (float)(1/sqrt(B)) is applied once, afterwards.
+ *   R3  D is shared by all workers and re-drawn per round: sign bit of padded
+ *       coordinate j is bit (j mod 128) of Philox4x32-10(key = seed,
+ *       counter = (j/128 lo, j/128 hi, 0xFFFFFFFF, round)).
+ *   R4  The uniform variate of coordinate j at worker i is the 16-bit field (j mod 8)
+ *       of Philox4x32-10(key = seed, counter = (j/8 lo, j/8 hi, i, round)).
+ *   R5  Position on the grid in fp32: y = clamp(fma(r, kappa, g/2), 0, g) with
+ *       kappa = (float)(g / (2 M)).  Clamping y to [0, g] is the truncation of r to
+ *       [-M, M] carried through the (monotone) affine map of Algorithm 2.
+ *   R6  Rounding decision: z0 = the largest index <= 2^b - 2 with T[z0] <= floor(y)
+ *       (capped so that y = g falls in the last interval);
+ *       up iff u16 < RN(2^16 * (y - T[z0]) / (T[z0+1] - T[z0])), the product taken as
+ *       one fused multiply-add of (y - T[z0]) with R16[z0] = 65536 / (T[z0+1]-T[z0]).
+ *       So P(up) is the paper's (a - q0)/(q1 - q0) rounded to a multiple of 2^-16.
+ *   R7  Packing: index j occupies bits [(j mod 8/b) * b, +b) of byte j*b/8; sums are
+ *       little-endian unsigned w-bit integers in coordinate order.
+ *   R8  Degenerate block (M == 0 or M not finite): all indices are 0 and the block
+ *       decompresses to exact zeros.
+ *
+ * All fp32 operations are single IEEE round-to-nearest operations; compile with
+ * -ffp-contract=off so that only the fmaf() calls written below are fused.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------------------------
+ * Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as
+ * 1, 2, 3", SC'11).  Ten rounds; the key is bumped by the Weyl constants between
+ * rounds.  The THC paper only asks for independent random choices (Appendix A.2);
+ * the generator is reading R3/R4.
+ * ---------------------------------------------------------------------------------- */
+void thc_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* Sign of padded coordinate j in round `round` (reading R3): +1 or -1. */
+int thc_oracle_sign(uint64_t seed, uint32_t round, uint64_t j)
+{
+    uint64_t call = j >> 7;
+    uint32_t ctr[4] = { (uint32_t)call, (uint32_t)(call >> 32), 0xFFFFFFFFu, round };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    thc_oracle_philox4x32_10(ctr, key, out);
+    uint32_t bit = (uint32_t)(j & 127u);
+    return ((out[bit >> 5] >> (bit & 31u)) & 1u) ? -1 : +1;
+}
+
+/* 16-bit uniform field of coordinate j at worker `worker` (reading R4). */
+uint32_t thc_oracle_u16(uint64_t seed, uint32_t round, uint32_t worker, uint64_t j)
+{
+    uint64_t call = j >> 3;
+    uint32_t ctr[4] = { (uint32_t)call, (uint32_t)(call >> 32), worker, round };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    thc_oracle_philox4x32_10(ctr, key, out);
+    uint32_t e = (uint32_t)(j & 7u);
+    uint32_t word = out[e >> 1];
+    return (e & 1u) ? (word >> 16) : (word & 0xFFFFu);
+}
+
+/* ------------------------------------------------------------------------------------
+ * Unnormalised Hadamard transform H_B v, in place, fp32, radix-2, ascending stride
+ * (reading R2).  Section 5.1: "the special recursive structure of H".
+ * ---------------------------------------------------------------------------------- */
+void thc_oracle_fwht(float *v, uint64_t B)
+{
+    for (uint64_t h = 1; h < B; h <<= 1) {
+        for (uint64_t base = 0; base < B; base += 2 * h) {
+            for (uint64_t j = base; j < base + h; ++j) {
+                float a = v[j];
+                float b = v[j + h];
+                v[j] = a + b;
+                v[j + h] = a - b;
+            }
+        }
+    }
+}
+
+static float c_of_block(uint32_t k)
+{
+    return (float)(1.0 / sqrt((double)((uint64_t)1 << k)));
+}
+
+/* ------------------------------------------------------------------------------------
+ * Preliminary stage (Section 5.3, Algorithm 3): per block, ell = max_i ||x_i|| and
+ * M = t_p * ell / sqrt(B).  x is [n][d] row-major; blocks are zero-padded (R1).
+ * scales[kblk] receives M as fp32.  A non-finite norm gives M = 0 (R8).
+ * ---------------------------------------------------------------------------------- */
+void thc_oracle_scales(const float *x, uint32_t n, uint64_t d, uint32_t k, double t_p,
+                       float *scales)
+{
+    uint64_t B = (uint64_t)1 << k;
+    uint64_t nb = (d + B - 1) / B;
+#pragma omp parallel for schedule(dynamic)
+    for (int64_t blk = 0; blk < (int64_t)nb; ++blk) {
+        double ell = 0.0;
+        uint64_t lo = (uint64_t)blk * B;
+        uint64_t hi = lo + B < d ? lo + B : d;
+        for (uint32_t i = 0; i < n; ++i) {
+            double s = 0.0;
+            for (uint64_t j = lo; j < hi; ++j) {
+                double a = (double)x[(uint64_t)i * d + j];
+                s += a * a;
+            }
+            double norm = sqrt(s);
+            if (!(norm <= ell)) ell = norm;   /* also lets NaN through */
+        }
+        float M = (float)(t_p * ell / sqrt((double)B));
+        if (!isfinite(M)) M = 0.0f;
+        scales[blk] = M;
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * Forward RHT of one worker's vector (Section 5.1): r = c_B * H_B (D x) per block.
+ * x has d entries, r has d_pad = nb * B entries.
+ * ---------------------------------------------------------------------------------- */
+void thc_oracle_rht_forward(const float *x, uint64_t d, uint32_t k, uint64_t seed,
+                            uint32_t round, float *r)
+{
+    uint64_t B = (uint64_t)1 << k;
+    uint64_t nb = (d + B - 1) / B;
+    float c = c_of_block(k);
+#pragma omp parallel for schedule(dynamic)
+    for (int64_t blk = 0; blk < (int64_t)nb; ++blk) {
+        float *v = r + (uint64_t)blk * B;
+        for (uint64_t t = 0; t < B; ++t) {
+            uint64_t j = (uint64_t)blk * B + t;
+            float a = j < d ? x[j] : 0.0f;
+            v[t] = thc_oracle_sign(seed, round, j) < 0 ? -a : a;
+        }
+        thc_oracle_fwht(v, B);
+        for (uint64_t t = 0; t < B; ++t) v[t] = v[t] * c;
+    }
+}
+
+/* Inverse RHT (Section 5.1): out = D (c_B * H_B v) per block; v has d_pad entries and is
+ * overwritten; out receives the first d coordinates. */
+void thc_oracle_rht_inverse(float *v, uint64_t d, uint32_t k, uint64_t seed, uint32_t round,
+                            float *out)
+{
+    uint64_t B = (uint64_t)1 << k;
+    uint64_t nb = (d + B - 1) / B;
+    float c = c_of_block(k);
+#pragma omp parallel for schedule(dynamic)
+    for (int64_t blk = 0; blk < (int64_t)nb; ++blk) {
+        float *w = v + (uint64_t)blk * B;
+        thc_oracle_fwht(w, B);
+        for (uint64_t t = 0; t < B; ++t) {
+            uint64_t j = (uint64_t)blk * B + t;
+            if (j >= d) break;
+            float a = w[t] * c;
+            out[j] = thc_oracle_sign(seed, round, j) < 0 ? -a : a;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * Stochastic quantization of already-rotated coordinates to table indices
+ * (Algorithm 2 worker lines; Section 4.1; readings R5, R6, R8).
+ *   r       d_pad rotated coordinates of worker `worker`
+ *   scales  M per block
+ *   table   T[0..2^b-1], 0 = T[0] < ... < T[2^b-1] = g
+ *   z       receives one index per coordinate (unpacked, one byte each)
+ * ---------------------------------------------------------------------------------- */
+void thc_oracle_quantize(const float *r, uint64_t d_pad, uint32_t k, const float *scales,
+                         uint32_t b, uint32_t g, const uint16_t *table, uint64_t seed,
+                         uint32_t round, uint32_t worker, uint8_t *z)
+{
+    uint64_t B = (uint64_t)1 << k;
+    uint32_t levels = 1u << b;
+#pragma omp parallel for schedule(static)
+    for (int64_t jj = 0; jj < (int64_t)d_pad; ++jj) {
+        uint64_t j = (uint64_t)jj;
+        float M = scales[j / B];
+        if (!(M > 0.0f) || !isfinite(M)) { z[j] = 0; continue; }          /* R8 */
+        float kappa = (float)((double)g / (2.0 * (double)M));
+        float half_g = 0.5f * (float)g;
+        float y = fmaf(r[j], kappa, half_g);                              /* R5 */
+        if (!(y >= 0.0f)) y = 0.0f;                                       /* NaN -> 0 */
+        if (y > (float)g) y = (float)g;
+        int f = (int)floorf(y);
+        if (f > (int)g - 1) f = (int)g - 1;
+        uint32_t z0 = 0;                                                  /* R6 */
+        while (z0 + 1 <= levels - 2 && (int)table[z0 + 1] <= f) ++z0;
+        float gap = (float)((int)table[z0 + 1] - (int)table[z0]);
+        float r16 = 65536.0f / gap;
+        float delta = y - (float)table[z0];
+        float tau = fmaf(delta, r16, 8388608.0f);                         /* RN to integer */
+        uint32_t threshold = (uint32_t)(tau - 8388608.0f);
+        uint32_t u = thc_oracle_u16(seed, round, worker, j);
+        z[j] = (uint8_t)(z0 + (u < threshold ? 1u : 0u));
+    }
+}
+
+/* Bit-packing (Section 3; reading R7). packed has d_pad*b/8 bytes. */
+void thc_oracle_pack(const uint8_t *z, uint64_t d_pad, uint32_t b, uint8_t *packed)
+{
+    uint64_t nbytes = d_pad * b / 8;
+    memset(packed, 0, nbytes);
+    uint32_t per_byte = 8 / b;
+    for (uint64_t j = 0; j < d_pad; ++j) {
+        packed[j / per_byte] |= (uint8_t)(z[j] << ((j % per_byte) * b));
+    }
+}
+
+void thc_oracle_unpack(const uint8_t *packed, uint64_t d_pad, uint32_t b, uint8_t *z)
+{
+    uint32_t per_byte = 8 / b;
+    uint32_t mask = (1u << b) - 1u;
+    for (uint64_t j = 0; j < d_pad; ++j) {
+        z[j] = (uint8_t)((packed[j / per_byte] >> ((j % per_byte) * b)) & mask);
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * PS aggregation (Algorithm 2, PS line: Y = sum_i T[Z_i]).  packed is [n][d_pad*b/8];
+ * sum receives d_pad little-endian unsigned integers of w bits (w in 8, 16, 32).
+ * Wraps modulo 2^w exactly like a w-bit register would; the caller guarantees n*g fits.
+ * ---------------------------------------------------------------------------------- */
+void thc_oracle_aggregate(const uint8_t *packed, uint32_t n, uint64_t d_pad, uint32_t b,
+                          const uint16_t *table, uint32_t w, void *sum)
+{
+    uint64_t stride = d_pad * b / 8;
+    uint32_t per_byte = 8 / b;
+    uint32_t mask = (1u << b) - 1u;
+    for (uint64_t j = 0; j < d_pad; ++j) {
+        uint32_t y = 0;
+        for (uint32_t i = 0; i < n; ++i) {
+            uint8_t byte = packed[(uint64_t)i * stride + j / per_byte];
+            uint32_t zi = (byte >> ((j % per_byte) * b)) & mask;
+            y += table[zi];
+        }
+        if (w == 8) ((uint8_t *)sum)[j] = (uint8_t)y;
+        else if (w == 16) ((uint16_t *)sum)[j] = (uint16_t)y;
+        else ((uint32_t *)sum)[j] = y;
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * Worker decompression (Algorithm 2 last two lines + inverse RHT, Algorithm 3):
+ *   v = m + (Y/n) (M-m)/g = -M + Y * (2M/(g n)),  out = RHT^-1(v).
+ * `divisor` is n (or the number of workers actually summed).  thc_oracle_estimate is the
+ * "Estimate" line alone (d_pad values, still in the rotated domain).
+ * ---------------------------------------------------------------------------------- */
+void thc_oracle_estimate(const void *sum, uint32_t w, uint32_t divisor, uint64_t d_pad,
+                         uint32_t k, const float *scales, uint32_t g, float *v)
+{
+    uint64_t B = (uint64_t)1 << k;
+    for (uint64_t j = 0; j < d_pad; ++j) {
+        float M = scales[j / B];
+        if (!(M > 0.0f) || !isfinite(M)) { v[j] = 0.0f; continue; }      /* R8 */
+        uint32_t y = w == 8 ? ((const uint8_t *)sum)[j]
+                   : w == 16 ? ((const uint16_t *)sum)[j]
+                             : ((const uint32_t *)sum)[j];
+        float step = (float)(2.0 * (double)M / ((double)g * (double)divisor));
+        v[j] = fmaf((float)y, step, -M);
+    }
+}
+
+void thc_oracle_decompress(const void *sum, uint32_t w, uint32_t divisor, uint64_t d,
+                           uint32_t k, const float *scales, uint32_t g, uint64_t seed,
+                           uint32_t round, float *out)
+{
+    uint64_t B = (uint64_t)1 << k;
+    uint64_t nb = (d + B - 1) / B;
+    uint64_t d_pad = nb * B;
+    float *v = (float *)malloc(sizeof(float) * d_pad);
+    thc_oracle_estimate(sum, w, divisor, d_pad, k, scales, g, v);
+    thc_oracle_rht_inverse(v, d, k, seed, round, out);
+    free(v);
+}
+
+/* Value a single worker's index stands for on the real line, before the inverse RHT
+ * (Algorithm 2: the quantization value m + T[z] (M-m)/g).  Used to state the
+ * homomorphic identity of Definition 3. */
+void thc_oracle_dequantize(const uint8_t *z, uint64_t d_pad, uint32_t k, const float *scales,
+                           uint32_t g, const uint16_t *table, double *value)
+{
+    uint64_t B = (uint64_t)1 << k;
+    for (uint64_t j = 0; j < d_pad; ++j) {
+        double M = (double)scales[j / B];
+        value[j] = -M + (double)table[z[j]] * (2.0 * M / (double)g);
+    }
+}
