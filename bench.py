@@ -1,0 +1,332 @@
+#!/usr/bin/env python
+"""Benchmark of the THC hot path on B200: one JSON line per run.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg2]
+
+A step is one pass of the whole path over one batch of synthetic gradients:
+thc_prepare + thc_compress (all n simulated workers) + thc_aggregate + one thc_decompress.
+`value` is fp32-gradient GB/s (n * d * 4 bytes per step) with inputs resident in HBM;
+`e2e` is the same metric with the gradients coming from pinned host memory and the result
+copied back, every step.  With N > 1 every rank runs an independent replica of the workload
+(the path has no exchange between GPUs) and the value is the sum over ranks.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2302_08545_b200 import workloads as W  # noqa: E402
+
+METRIC = "gradient GB/s per compress+aggregate+decompress round; % of HBM roofline"
+UNIT = "GB/s"
+KERNELS_PER_STEP = {"prepare": 2, "compress": 2, "aggregate": 1, "decompress": 2}
+
+
+def pick_workload(name: str) -> W.Workload:
+    return {"cfg1": W.config1, "cfg2": W.config2, "cfg3": lambda: W.config3(4),
+            "cfg3b2": lambda: W.config3(2), "cfg4": W.config4}[name]()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    return 6650.0, "fallback (earlier pool measurement)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self._stop = threading.Event()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                                      "--format=csv,noheader,nounits"], capture_output=True,
+                                     text=True, timeout=5).stdout.strip()
+                if out:
+                    self.samples.append([s.strip() for s in out.splitlines()[0].split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._thread.join(timeout=6)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        sm = sorted(float(s[0]) for s in self.samples)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(s[2 + i] == "Active" for s in self.samples)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(self.samples[0][1]),
+                "reasons": reasons, "samples": len(sm)}
+
+
+def visible_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ------------------------------------------------------------------------- oracle timing
+def oracle_sample_workload(w: W.Workload, blocks: int) -> W.Workload:
+    """The same recipe on `blocks` RHT blocks per worker (blocks are independent)."""
+    return W.scaled(w, d=min(w.d, blocks * w.block))
+
+
+def time_oracle_round(w: W.Workload, x, repeats: int = 1):
+    """Wall-clock of the oracle's whole round on the host cores; returns (seconds, cores)."""
+    from oracle import oracle as O
+    cfg = O.Config(bits=w.bits, granularity=w.granularity, table=tuple(w.table), t_p=w.t_p,
+                   log2_block=w.log2_block, seed=w.seed)
+    xf = O.bf16_to_f32(x) if w.in_dtype == "bf16" else x
+    cores = len(os.sched_getaffinity(0))
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        O.thc_round(xf, cfg, rnd=0)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return best, cores
+
+
+def cpu_baseline(w: W.Workload, blocks: int = 25):
+    """Oracle on (up to) `blocks` RHT blocks per worker: about 15 s on 8 cores for cfg2."""
+    ws = oracle_sample_workload(w, blocks)
+    x = W.generate(ws)
+    secs, cores = time_oracle_round(ws, x)
+    gbs = ws.n * ws.d * 4 / secs / 1e9
+    return {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{blocks} RHT blocks of 2^{ws.log2_block} per worker, n={ws.n} "
+                      f"(d={ws.d} of {w.d}); one whole round incl. prepare, {secs:.2f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    w = pick_workload(args.workload)
+    blocks = 1
+    ws = oracle_sample_workload(w, blocks)
+    x = W.generate(ws)
+    for _ in range(args.warmup):
+        time_oracle_round(ws, x)
+    t0 = time.perf_counter()
+    cores = 0
+    for _ in range(args.steps):
+        _, cores = time_oracle_round(ws, x)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = ws.n * ws.d * 4 / dt / 1e9
+    sample = (f"each step = the oracle's whole round on {blocks} RHT block(s) per worker "
+              f"(d={ws.d} of {w.d}), n={ws.n}")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(w),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(w: W.Workload):
+    return {"workload": w.name, "n_workers": w.n, "d": w.d, "d_pad": w.d_pad,
+            "rht_block_log2": w.log2_block, "index_bits": w.bits, "granularity": w.granularity,
+            "acc_bits": w.acc_bits, "in_dtype": w.in_dtype,
+            "step": "prepare+compress+aggregate+decompress",
+            "l2": "inputs (n*d*4 bytes) far exceed the 126 MB L2; no flush between steps"}
+
+
+# ------------------------------------------------------------------------------ GPU arm
+def reduce_max(value: float, dist_mod, device=None) -> float:
+    """Max over ranks of a host float (the step time every rank agrees on)."""
+    if dist_mod is None or not dist_mod.is_initialized() or dist_mod.get_world_size() == 1:
+        return value
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist_mod.all_reduce(t, op=dist_mod.ReduceOp.MAX)
+    return float(t.item())
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2302_08545_b200 import runner, thc
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = pick_workload(args.workload)
+    thc.lib()                                   # fail loudly if the extension is missing
+    x = W.generate(w)                           # every rank: an independent replica
+    ctx = runner.context_for(w)
+    r = runner.Round(ctx, w.n, w.d, w.in_dtype, device=str(dev))
+    r.upload(x)
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+
+    calls = [("prepare", r.prepare), ("compress", lambda: r.compress(0)),
+             ("aggregate", r.aggregate), ("decompress", lambda: r.decompress(0))]
+
+    def step(events=None):
+        for name, fn in calls:
+            if events is not None:
+                a = torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+            fn()
+            if events is not None:
+                b = torch.cuda.Event(enable_timing=True)
+                b.record(stream)
+                events.append((name, a, b))
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+
+    # ---- timed region: inputs resident in HBM
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    events = []
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(visible_gpu_index(local_rank)) as clocks:
+        start.record(stream)
+        for _ in range(args.steps):
+            step(events)
+        end.record(stream)
+        torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    ms_local = start.elapsed_time(end) / args.steps
+    ms = reduce_max(ms_local, dist if world > 1 else None, dev)
+    per_call = {}
+    for name, a, b in events:
+        per_call.setdefault(name, []).append(a.elapsed_time(b))
+    per_call_ms = {k: float(np.mean(v)) for k, v in per_call.items()}
+    status = ctx.status()
+
+    # ---- end to end: gradients from pinned host memory, result copied back, every step
+    e2e_steps = max(1, min(args.steps, 5))
+    x_host = torch.from_numpy(x).pin_memory() if w.in_dtype == "f32" else \
+        torch.from_numpy(x).view(torch.int16).pin_memory()
+    out_host = torch.empty(w.d, dtype=torch.float32).pin_memory()
+
+    def e2e_step():
+        for i in range(w.n):
+            dst = r.grads[i] if w.in_dtype == "f32" else r.grads[i].view(torch.int16)
+            dst.copy_(x_host[i], non_blocking=True)
+        step()
+        out_host.copy_(r.out, non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e2.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = reduce_max(s2.elapsed_time(e2) / e2e_steps, dist if world > 1 else None, dev)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    grad_bytes = w.n * w.d * 4
+    ab = w.algorithmic_bytes()
+    peak, peak_src = measured_peaks()
+    value = world * grad_bytes / (ms * 1e-3) / 1e9
+    round_ms = per_call_ms["compress"] + per_call_ms["aggregate"] + per_call_ms["decompress"]
+    comp_ms = per_call_ms["compress"]
+    achieved = ab["compress"] / (comp_ms * 1e-3) / 1e9
+    in_bytes = w.n * w.d * (4 if w.in_dtype == "f32" else 2)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(w),
+        "clocks": clocks.summary(),
+        "e2e": {"value": world * grad_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+                "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": w.d * 4,
+                "ms_per_step": e2e_ms, "steps": e2e_steps},
+        "gpu_launches": args.steps * sum(KERNELS_PER_STEP.values()),
+        "roofline": {"kernel": "thc_compress (RHT + quantise + pack kernels)", "bound": "hbm",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_source": peak_src, "algorithmic_bytes_per_launch": ab["compress"],
+                     "ms_per_launch": comp_ms, "traffic": None},
+        "per_call_ms": per_call_ms,
+        "round_excl_prepare": {
+            "ms": round_ms, "gradient_gbs": grad_bytes / (round_ms * 1e-3) / 1e9,
+            "algorithmic_gbs": ab["round"] / (round_ms * 1e-3) / 1e9,
+            "frac_of_measured_hbm": ab["round"] / (round_ms * 1e-3) / 1e9 / peak,
+            "frac_of_8000_nominal": ab["round"] / (round_ms * 1e-3) / 1e9 / 8000.0},
+        "status_flags": status,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(w)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="thc", choices=["thc", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

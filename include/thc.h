@@ -1,0 +1,166 @@
+/*
+ * libthc -- the data-parallel hot path of Tensor Homomorphic Compression (THC,
+ * arxiv 2302.08545) as hand-written CUDA for sm_100a, behind a C ABI.
+ *
+ * One round, as the paper states it (Algorithm 3, the coloured THC lines):
+ *     thc_prepare     preliminary stage: per RHT block, M = t_p * max_i ||x_i|| / sqrt(B)
+ *     thc_compress    RHT -> truncate -> stochastic quantisation to b-bit table indices -> pack
+ *     thc_aggregate   the parameter server's only job: Y = sum_i T[Z_i], in integers
+ *     thc_decompress  Y/n -> real values -> inverse RHT
+ *
+ * Conventions shared by every call
+ *   - "device" pointers are CUDA device addresses on the device that was current when the
+ *     context was created; "host" pointers are ordinary host memory.
+ *   - Arrays of per-worker pointers (grads, packed, rotated) are HOST arrays holding DEVICE
+ *     pointers; the library copies them into kernel arguments, so they may be freed or
+ *     reused as soon as the call returns.
+ *   - Every device buffer is owned by the caller.  Device buffers must be 16-byte aligned.
+ *     The library owns only the context (a few hundred bytes of device memory for the
+ *     status word and scheduling counters, allocated by thc_create).
+ *   - The four round calls and thc_quantize_rotated only enqueue work on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream) and return without
+ *     synchronising.  They allocate nothing.  Calls that share a context must be issued
+ *     on one stream (or be ordered by the caller): they share the context's counters.
+ *   - Return value: THC_OK or a negative THC_E* code; thc_strerror() gives text, and for
+ *     THC_ECUDA the text of the CUDA error last seen by this thread's library calls.
+ *   - Conditions met on the device never trap: they set bits that thc_status() reports.
+ *
+ * Layouts (coordinate j = 0 .. d_pad-1, d_pad = d rounded up to a multiple of B = 2^k)
+ *   gradient   d elements, fp32 or bf16, contiguous; coordinates d..d_pad-1 count as zero
+ *   scales     one fp32 M per block, nblocks = d_pad / B entries
+ *   packed     d_pad*b/8 bytes per worker; index j in bits [(j mod 8/b)*b, +b) of byte j*b/8
+ *   sum        d_pad little-endian unsigned integers of acc_bits bits
+ *   rotated    d_pad fp32 per worker: the RHT output before truncation (optional)
+ *   out        d fp32
+ */
+#ifndef THC_H_
+#define THC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define THC_OK             0
+#define THC_EINVAL        (-1)  /* bad configuration or argument (null, misaligned, n = 0, ...) */
+#define THC_EUNSUPPORTED  (-2)  /* valid but not implemented (e.g. granularity > 255)           */
+#define THC_ECUDA         (-3)  /* a CUDA call failed, or the context has no device             */
+#define THC_EWORKSPACE    (-4)  /* workspace smaller than thc_sizes() asks for                  */
+
+#define THC_F32   0u
+#define THC_BF16  1u
+
+#define THC_MAX_WORKERS 64u
+
+/* thc_status() bits */
+#define THC_STATUS_NONFINITE     1u  /* a block's norm was NaN/Inf: its scale was set to 0        */
+#define THC_STATUS_ZERO_BLOCK    2u  /* a block had scale 0 (all-zero input): indices 0, output 0 */
+#define THC_STATUS_WAIT_TIMEOUT  4u  /* an on-device wait gave up; the call's output is invalid   */
+
+typedef struct thc_ctx thc_ctx;   /* opaque */
+
+/*
+ * Parameters of the method (Algorithm 3, "Input" line) plus the layout choices.
+ *   bits         b in {1, 2, 4, 8}: bits per table index (Section 4.3)
+ *   granularity  g with 2^b - 1 <= g <= 255 (Section 4.3, "granularity")
+ *   table        T[0 .. 2^b - 1], 0 = T[0] < T[1] < ... < T[2^b - 1] = g (Section 4.3);
+ *                the identity table with g = 2^b - 1 is Uniform THC (Section 4.2)
+ *   t_p          truncation threshold Phi^-1(1 - p/2) (Section 5.2), > 0
+ *   log2_block   k in [3, 24]: the RHT acts on blocks of B = 2^k coordinates (Section 5.1
+ *                applied per partition)
+ *   seed         shared by all workers: the diagonal D of the RHT must be common
+ *   in_dtype     THC_F32 or THC_BF16 (bf16 gradients are widened exactly on load)
+ *   workers      the largest number of workers thc_aggregate will sum (1..THC_MAX_WORKERS)
+ *   acc_bits     width of the sums: 8, 16 or 32, or 0 = smallest with workers*g <= 2^w - 1
+ *                (Section 8.4: the largest aggregate is g*n)
+ */
+typedef struct thc_config {
+    uint32_t bits;
+    uint32_t granularity;
+    uint16_t table[256];
+    double   t_p;
+    uint32_t log2_block;
+    uint64_t seed;
+    uint32_t in_dtype;
+    uint32_t workers;
+    uint32_t acc_bits;
+} thc_config;
+
+typedef struct thc_sizes_t {
+    uint64_t d_pad;            /* d rounded up to a multiple of the block              */
+    uint64_t nblocks;          /* d_pad / B = number of scales                         */
+    uint64_t packed_bytes;     /* per worker                                           */
+    uint64_t sum_bytes;        /* d_pad * acc_bits / 8                                 */
+    uint64_t rotated_bytes;    /* per worker, 4 * d_pad                                */
+    uint64_t workspace_bytes;  /* scratch any call may need for this (d, n_local)      */
+    uint32_t acc_bits;         /* the resolved accumulator width                       */
+    uint32_t reserved;
+} thc_sizes_t;
+
+/* Validate `cfg` (host only) and build a context.  If a CUDA device is present, the
+ * context's device block is allocated on the current device; without a device the context
+ * still answers thc_sizes() and validation, and every launching call returns THC_ECUDA.
+ * Errors: THC_EINVAL (see thc_config), THC_EUNSUPPORTED, THC_ECUDA. */
+int thc_create(const thc_config *cfg, thc_ctx **ctx);
+int thc_destroy(thc_ctx *ctx);
+
+/* Buffer sizes for gradients of d elements and calls that handle up to n_local workers at
+ * once.  Host only. */
+int thc_sizes(const thc_ctx *ctx, uint64_t d, uint32_t n_local, thc_sizes_t *sizes);
+
+/* Preliminary stage (Section 5.3; Algorithm 3, "Send ||x_i|| / Receive ell" and
+ * "M = (t_p / sqrt d) * ell"): scales[blk] = (float)(t_p * max_i ||x_i restricted to
+ * block blk||_2 / sqrt(B)), norms accumulated in fp64.  A non-finite norm gives scale 0 and
+ * sets THC_STATUS_NONFINITE.
+ *   grads   host array of n device pointers, each d elements of cfg.in_dtype
+ *   scales  device, nblocks fp32, written                                              */
+int thc_prepare(thc_ctx *ctx, const void *const *grads, uint32_t n, uint64_t d,
+                float *scales, void *workspace, uint64_t workspace_bytes, void *stream);
+
+/* Worker-side compression of n_local workers' gradients (Algorithm 3: RHT, truncation,
+ * stochastic quantisation, table index; Section 3: packing).  Worker i of this call is
+ * worker (worker_base + i) of the job: its id keys its random stream, so that workers
+ * round independently (Appendix A.2) while sharing D.
+ *   scales   device, from thc_prepare (or any agreed positive bounds)
+ *   packed   host array of n_local device pointers, packed_bytes each, written
+ *   rotated  NULL, or host array of n_local device pointers (NULL entries allowed), each
+ *            rotated_bytes: receives RHT(x_i), e.g. for error feedback or for tests      */
+int thc_compress(thc_ctx *ctx, const void *const *grads, uint32_t n_local, uint32_t worker_base,
+                 uint64_t d, uint32_t round, const float *scales, void *const *packed,
+                 float *const *rotated, void *workspace, uint64_t workspace_bytes,
+                 void *stream);
+
+/* The quantisation half of thc_compress alone (Algorithm 2, worker lines 1-4, after the
+ * truncation of Algorithm 3), on coordinates that are already rotated:
+ *   rotated  host array of n_local device pointers, d_pad fp32 each, read                */
+int thc_quantize_rotated(thc_ctx *ctx, const float *const *rotated, uint32_t n_local,
+                         uint32_t worker_base, uint64_t d, uint32_t round, const float *scales,
+                         void *const *packed, void *stream);
+
+/* Parameter-server aggregation (Algorithm 2, PS line: Y = sum_i T[Z_i]; Section 3: lookups
+ * and integer sums only).  n may be smaller than cfg.workers (partial aggregation, Section 6).
+ *   packed  host array of n device pointers, read
+ *   sum     device, sum_bytes, written                                                   */
+int thc_aggregate(thc_ctx *ctx, const void *const *packed, uint32_t n, uint64_t d,
+                  void *sum, void *stream);
+
+/* Worker-side decompression (Algorithm 2: Y_avg = Y / n, estimate = m + Y_avg (M - m)/g;
+ * Algorithm 3: inverse RHT).  `divisor` is the number of workers that were summed.
+ *   out  device, d fp32, written                                                         */
+int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, uint32_t round,
+                   const float *scales, float *out, void *workspace, uint64_t workspace_bytes,
+                   void *stream);
+
+/* Read and clear the status bits (synchronises `stream`).  flags is a host pointer. */
+int thc_status(thc_ctx *ctx, uint32_t *flags, void *stream);
+
+const char *thc_strerror(int code);
+
+/* Library build identification, e.g. "thc-b200 sm_100a". */
+const char *thc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* THC_H_ */

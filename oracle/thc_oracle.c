@@ -147,7 +147,7 @@ void thc_oracle_scales(const float *x, uint32_t n, uint64_t d, uint32_t k, doubl
                 s += a * a;
             }
             double norm = sqrt(s);
-            if (!(norm <= ell)) ell = norm;   /* also lets NaN through */
+            if (norm > ell || norm != norm) ell = norm;   /* a NaN norm sticks (R8) */
         }
         float M = (float)(t_p * ell / sqrt((double)B));
         if (!isfinite(M)) M = 0.0f;

@@ -1,0 +1,982 @@
+// libthc: kernels and C ABI.  See include/thc.h for the contract of every entry point.
+//
+// Structure of the transform.  An RHT block of B = 2^k coordinates is handled as one or two
+// passes over 2^14-coordinate tiles held in shared memory:
+//   pass A  a tile is 2^14 consecutive coordinates: load (+ sign flip or de-quantisation),
+//           stages of stride 1 .. 2^13 (or 2^(k-1) if k < 14)
+//   pass B  (only if k > 14) a tile is 2^(k-14) rows, 2^14 coordinates apart, by 2^(28-k)
+//           consecutive columns: the remaining stages of stride 2^14 .. 2^(k-1)
+// The last pass of a block ends in the fused epilogue: scale by 1/sqrt(B), then either
+// truncate + quantise + pack (compress) or sign flip + store (decompress).
+#include "../../include/thc.h"
+#include "thc_device.cuh"
+
+#include <math.h>
+#include <new>
+#include <stdio.h>
+#include <string.h>
+
+namespace thc {
+
+struct PtrArray { const void *p[THC_MAX_WORKERS]; };
+struct MutPtrArray { void *p[THC_MAX_WORKERS]; };
+
+enum LoadKind { kLoadGradF32, kLoadGradBF16, kLoadSum8, kLoadSum16, kLoadSum32, kLoadRaw };
+enum StoreKind { kStoreRaw, kStoreQuant, kStoreOut };
+
+// Geometry of the tiles one launch walks.
+struct TileGeom {
+    uint64_t d;            // valid coordinates per worker
+    uint64_t d_pad;
+    uint64_t row_stride;   // coordinates between consecutive tile rows
+    uint32_t k;            // log2 of the RHT block
+    uint32_t row_log2;     // tile = 2^row_log2 rows ...
+    uint32_t col_log2;     // ... of 2^col_log2 consecutive coordinates (sum = 14)
+    uint32_t lo_cbit;      // chunk-index bits [lo_cbit, hi_cbit) are transformed
+    uint32_t hi_cbit;
+    uint32_t blocks_in_tile;   // RHT blocks a tile overlaps (1 if k >= 14)
+    uint32_t lut_rep;          // lane replication of the quantiser table in shared memory
+    uint32_t granularity;
+    uint32_t divisor;          // decompress: workers summed
+    uint32_t round;
+    uint32_t worker_base;
+    float    c_block;          // (float)(1/sqrt(B))
+};
+
+__device__ __forceinline__ uint64_t tile_base(const TileGeom &g, uint32_t tile)
+{
+    if (g.row_log2 == 0) return (uint64_t)tile << kTileLog2;
+    const uint32_t panels = 1u << g.row_log2;          // panels per RHT block
+    const uint64_t blk = tile >> g.row_log2;
+    const uint64_t panel = tile & (panels - 1);
+    return (blk << g.k) + (panel << g.col_log2);
+}
+
+__device__ __forceinline__ uint64_t chunk_coord(const TileGeom &g, uint64_t base, int c)
+{
+    const int ccl = (int)g.col_log2 - 2;
+    const uint64_t row = (uint64_t)(c >> ccl);
+    const uint64_t cc = (uint64_t)(c & ((1 << ccl) - 1));
+    return base + row * g.row_stride + cc * 4;
+}
+
+// Sign words of every row of the tile, 32 coordinates per word.
+__device__ __forceinline__ void fill_sign_words(uint32_t *sw, const TileGeom &g, uint64_t base,
+                                                const PhiloxKeys &keys, int tid)
+{
+    const int cols = 1 << g.col_log2;
+    const int words_per_row = max(1, cols >> 5);
+    const int calls_per_row = max(1, cols >> 7);
+    const int rows = 1 << g.row_log2;
+    const int words_per_call = min(4, words_per_row);
+    for (int q = tid; q < rows * calls_per_row; q += kThreads) {
+        const int row = q / calls_per_row;
+        const int cr = q - row * calls_per_row;
+        const uint64_t j0 = base + (uint64_t)row * g.row_stride + (uint64_t)cr * 128;
+        const uint4 ph = sign_call(j0, g.round, keys);
+        const int first = (int)((j0 >> 5) & 3);
+        for (int wi = 0; wi < words_per_call; ++wi) {
+            const int src = first + wi;
+            const uint32_t w = src == 0 ? ph.x : src == 1 ? ph.y : src == 2 ? ph.z : ph.w;
+            sw[row * words_per_row + cr * 4 + wi] = w;
+        }
+    }
+}
+
+__device__ __forceinline__ uint32_t sign_bits_of_chunk(const uint32_t *sw, const TileGeom &g,
+                                                       int c, uint64_t j)
+{
+    const int ccl = (int)g.col_log2 - 2;
+    const int row = c >> ccl;
+    const int cc = c & ((1 << ccl) - 1);
+    const int words_per_row = max(1, (1 << g.col_log2) >> 5);
+    return sw[row * words_per_row + (cc >> 3)] >> (uint32_t)(j & 31);
+}
+
+__device__ __forceinline__ float4 load_f32x4_masked(const float *x, uint64_t j, uint64_t d)
+{
+    if (j + 4 <= d) return __ldg(reinterpret_cast<const float4 *>(x + j));
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (j + 0 < d) v.x = __ldg(x + j + 0);
+    if (j + 1 < d) v.y = __ldg(x + j + 1);
+    if (j + 2 < d) v.z = __ldg(x + j + 2);
+    if (j + 3 < d) v.w = __ldg(x + j + 3);
+    return v;
+}
+
+__device__ __forceinline__ float sum_to_float(uint32_t y)   // exact for y < 2^23
+{
+    return __uint_as_float(0x4B000000u | y) - 8388608.0f;
+}
+
+// One tile: load, butterfly rounds, store.  blockIdx.x = tile, blockIdx.y = local worker.
+template <int LOAD, int STORE, int BITS, bool IDENTITY>
+__global__ void __launch_bounds__(kThreads, 2)
+rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
+                const float *__restrict__ scales, DeviceBlock *dev, PhiloxKeys keys)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float4 *tile = reinterpret_cast<float4 *>(smem_raw);
+    uint32_t *sw = reinterpret_cast<uint32_t *>(smem_raw + kTileElems * 4);
+    float2 *blk_const = reinterpret_cast<float2 *>(smem_raw + kTileElems * 4 + kSignWordsMax * 4);
+    uint2 *lut = reinterpret_cast<uint2 *>(smem_raw + kTileElems * 4 + kSignWordsMax * 4 +
+                                           (size_t)g.blocks_in_tile * 8);
+
+    const int tid = threadIdx.x;
+    const uint32_t wl = blockIdx.y;
+    const uint64_t base = tile_base(g, blockIdx.x);
+    const uint64_t first_blk = base >> g.k;
+    const uint64_t nblocks = g.d_pad >> g.k;
+
+    // ---- per-tile constants
+    if (LOAD == kLoadGradF32 || LOAD == kLoadGradBF16 || STORE == kStoreOut)
+        fill_sign_words(sw, g, base, keys, tid);
+    if (STORE == kStoreQuant) {
+        // (kappa, g/2) per block; (0, 0) for a degenerate block
+        for (uint32_t b = tid; b < g.blocks_in_tile; b += kThreads) {
+            float2 c = make_float2(0.f, 0.f);
+            if (first_blk + b < nblocks) {
+                const float M = scales[first_blk + b];
+                if (M > 0.0f && isfinite(M)) {
+                    c.x = (float)((double)g.granularity / (2.0 * (double)M));
+                    c.y = 0.5f * (float)g.granularity;
+                }
+            }
+            blk_const[b] = c;
+        }
+        if (!IDENTITY) {
+            const int rep = (int)g.lut_rep;
+            for (int idx = tid; idx < (int)(g.granularity + 1) * rep; idx += kThreads) {
+                const int f = idx / rep;
+                lut[idx] = make_uint2(dev->lut_tz[f], __float_as_uint(dev->lut_r16[f]));
+            }
+        }
+    }
+    if (LOAD == kLoadSum8 || LOAD == kLoadSum16 || LOAD == kLoadSum32) {
+        // (step, -M) per block; (0, 0) for a degenerate block
+        for (uint32_t b = tid; b < g.blocks_in_tile; b += kThreads) {
+            float2 c = make_float2(0.f, 0.f);
+            if (first_blk + b < nblocks) {
+                const float M = scales[first_blk + b];
+                if (M > 0.0f && isfinite(M)) {
+                    c.x = (float)(2.0 * (double)M / ((double)g.granularity * (double)g.divisor));
+                    c.y = -M;
+                }
+            }
+            blk_const[b] = c;
+        }
+    }
+    __syncthreads();
+
+    // ---- load phase
+    if (LOAD == kLoadGradF32) {
+        const float *x = static_cast<const float *>(in.p[wl]);
+#pragma unroll 4
+        for (int i = 0; i < kTileChunks / kThreads; ++i) {
+            const int c = tid + i * kThreads;
+            const uint64_t j = base + (uint64_t)c * 4;
+            float4 v = load_f32x4_masked(x, j, g.d);
+            v = flip4(v, sw[c >> 3] >> ((c & 7) * 4));
+            tile[swz(c)] = stages01(v);
+        }
+    } else if (LOAD == kLoadGradBF16) {
+        const uint16_t *x = static_cast<const uint16_t *>(in.p[wl]);
+#pragma unroll 2
+        for (int i = 0; i < kTileChunks / 2 / kThreads; ++i) {
+            const int u = tid + i * kThreads;                 // 8 coordinates
+            const uint64_t j = base + (uint64_t)u * 8;
+            uint32_t w[4] = {0, 0, 0, 0};
+            if (j + 8 <= g.d) {
+                const uint4 q = __ldg(reinterpret_cast<const uint4 *>(x + j));
+                w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
+            } else {
+                for (int e = 0; e < 8; ++e)
+                    if (j + e < g.d) w[e >> 1] |= (uint32_t)__ldg(x + j + e) << ((e & 1) * 16);
+            }
+            float4 v0 = make_float4(__uint_as_float(w[0] << 16), __uint_as_float(w[0] & 0xFFFF0000u),
+                                    __uint_as_float(w[1] << 16), __uint_as_float(w[1] & 0xFFFF0000u));
+            float4 v1 = make_float4(__uint_as_float(w[2] << 16), __uint_as_float(w[2] & 0xFFFF0000u),
+                                    __uint_as_float(w[3] << 16), __uint_as_float(w[3] & 0xFFFF0000u));
+            const int c = 2 * u;
+            const uint32_t bits = sw[c >> 3] >> ((c & 7) * 4);
+            tile[swz(c)] = stages01(flip4(v0, bits));
+            tile[swz(c + 1)] = stages01(flip4(v1, bits >> 4));
+        }
+    } else if (LOAD == kLoadSum8 || LOAD == kLoadSum16 || LOAD == kLoadSum32) {
+        constexpr int kPer = LOAD == kLoadSum8 ? 16 : LOAD == kLoadSum16 ? 8 : 4;   // sums per 16 B
+        const unsigned char *y = static_cast<const unsigned char *>(in.p[0]);
+        for (int i = 0; i < kTileElems / kPer / kThreads; ++i) {
+            const int u = tid + i * kThreads;
+            const uint64_t j = base + (uint64_t)u * kPer;
+            uint4 q = make_uint4(0, 0, 0, 0);
+            if (j + kPer <= g.d_pad) {
+                q = __ldg(reinterpret_cast<const uint4 *>(y + j * (16 / kPer)));
+            } else if (j < g.d_pad) {          // only 8-bit sums with 8-coordinate blocks
+                const uint2 h = __ldg(reinterpret_cast<const uint2 *>(y + j * (16 / kPer)));
+                q.x = h.x; q.y = h.y;
+            }
+            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int cc = 0; cc < kPer / 4; ++cc) {
+                uint64_t bi = ((j + cc * 4) >> g.k) - first_blk;
+                if (bi >= g.blocks_in_tile) bi = 0;
+                const float2 bc = blk_const[bi];
+                float s[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int idx = cc * 4 + e;
+                    uint32_t val;
+                    if (LOAD == kLoadSum8) val = (w[idx >> 2] >> ((idx & 3) * 8)) & 0xFFu;
+                    else if (LOAD == kLoadSum16) val = (w[idx >> 1] >> ((idx & 1) * 16)) & 0xFFFFu;
+                    else val = w[idx];
+                    const float yf = LOAD == kLoadSum32 ? (float)val : sum_to_float(val);
+                    s[e] = fmaf(yf, bc.x, bc.y);
+                }
+                tile[swz(u * (kPer / 4) + cc)] = stages01(make_float4(s[0], s[1], s[2], s[3]));
+            }
+        }
+    } else {   // kLoadRaw: second pass, rows 2^14 apart
+        const float *x = static_cast<const float *>(in.p[0]) + (uint64_t)wl * g.d_pad;
+#pragma unroll 4
+        for (int i = 0; i < kTileChunks / kThreads; ++i) {
+            const int c = tid + i * kThreads;
+            const uint64_t j = chunk_coord(g, base, c);
+            tile[swz(c)] = *reinterpret_cast<const float4 *>(x + j);
+        }
+    }
+    __syncthreads();
+
+    // ---- butterflies
+    fwht_rounds(tile, (int)g.lo_cbit, (int)g.hi_cbit, tid);
+
+    // ---- store phase
+    if (STORE == kStoreRaw) {
+        float *ws = static_cast<float *>(out.p[0]) + (uint64_t)wl * g.d_pad;
+#pragma unroll 4
+        for (int i = 0; i < kTileChunks / kThreads; ++i) {
+            const int c = tid + i * kThreads;
+            const uint64_t j = chunk_coord(g, base, c);
+            if (j < g.d_pad) *reinterpret_cast<float4 *>(ws + j) = tile[swz(c)];
+        }
+    } else if (STORE == kStoreQuant) {
+        unsigned char *pk = static_cast<unsigned char *>(out.p[wl]);
+        float *rot = static_cast<float *>(rotated.p[wl]);
+        const float gf = (float)g.granularity;
+        const int lane = tid & 31;
+        const uint2 *my_lut = lut + (g.lut_rep > 1 ? lane : 0);
+#pragma unroll 1
+        for (int i = 0; i < kTileChunks / 2 / kThreads; ++i) {
+            const int u = tid + i * kThreads;
+            const int c = 2 * u;
+            const uint64_t j = chunk_coord(g, base, c);
+            if (j >= g.d_pad) continue;
+            const float4 a = scale4(tile[swz(c)], g.c_block);
+            const float4 b = scale4(tile[swz(c + 1)], g.c_block);
+            if (rot != nullptr) {
+                *reinterpret_cast<float4 *>(rot + j) = a;
+                *reinterpret_cast<float4 *>(rot + j + 4) = b;
+            }
+            const float r[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+            const float2 bc = blk_const[(j >> g.k) - first_blk];
+            const uint4 rnd = round_call(j, g.worker_base + wl, g.round, keys);
+            const uint64_t z = quantize8<BITS, IDENTITY>(r, bc.x, bc.y, gf, rnd, my_lut,
+                                                         (int)g.lut_rep);
+            if constexpr (BITS == 8) *reinterpret_cast<uint2 *>(pk + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
+            else if constexpr (BITS == 4) *reinterpret_cast<uint32_t *>(pk + j / 2) = (uint32_t)z;
+            else if constexpr (BITS == 2) *reinterpret_cast<uint16_t *>(pk + j / 4) = (uint16_t)z;
+            else pk[j / 8] = (unsigned char)z;
+        }
+    } else {   // kStoreOut
+        float *o = static_cast<float *>(out.p[0]);
+#pragma unroll 4
+        for (int i = 0; i < kTileChunks / kThreads; ++i) {
+            const int c = tid + i * kThreads;
+            const uint64_t j = chunk_coord(g, base, c);
+            if (j >= g.d) continue;
+            float4 v = scale4(tile[swz(c)], g.c_block);
+            v = flip4(v, sign_bits_of_chunk(sw, g, c, j));
+            if (j + 4 <= g.d) {
+                *reinterpret_cast<float4 *>(o + j) = v;
+            } else {
+                o[j] = v.x;
+                if (j + 1 < g.d) o[j + 1] = v.y;
+                if (j + 2 < g.d) o[j + 2] = v.z;
+            }
+        }
+    }
+}
+
+// Quantise + pack coordinates that are already rotated (the epilogue of compress alone).
+template <int BITS, bool IDENTITY>
+__global__ void __launch_bounds__(kThreads)
+quantize_rotated_kernel(PtrArray rotated, MutPtrArray packed, uint64_t d_pad, uint32_t k,
+                        uint32_t granularity, uint32_t round, uint32_t worker_base,
+                        const float *__restrict__ scales, const DeviceBlock *dev, PhiloxKeys keys)
+{
+    __shared__ uint2 lut[256];
+    for (int f = threadIdx.x; f <= (int)granularity; f += kThreads)
+        lut[f] = make_uint2(dev->lut_tz[f], __float_as_uint(dev->lut_r16[f]));
+    __syncthreads();
+    const uint32_t wl = blockIdx.y;
+    const float *rot = static_cast<const float *>(rotated.p[wl]);
+    unsigned char *pk = static_cast<unsigned char *>(packed.p[wl]);
+    const float gf = (float)granularity;
+    for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < d_pad / 8;
+         u += (uint64_t)gridDim.x * kThreads) {
+        const uint64_t j = u * 8;
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(rot + j));
+        const float4 b = __ldg(reinterpret_cast<const float4 *>(rot + j + 4));
+        const float r[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        const float M = scales[j >> k];
+        float kappa = 0.f, half_g = 0.f;
+        if (M > 0.0f && isfinite(M)) {
+            kappa = (float)((double)granularity / (2.0 * (double)M));
+            half_g = 0.5f * gf;
+        }
+        const uint4 rnd = round_call(j, worker_base + wl, round, keys);
+        const uint64_t z = quantize8<BITS, IDENTITY>(r, kappa, half_g, gf, rnd, lut, 1);
+        if constexpr (BITS == 8) *reinterpret_cast<uint2 *>(pk + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
+        else if constexpr (BITS == 4) *reinterpret_cast<uint32_t *>(pk + j / 2) = (uint32_t)z;
+        else if constexpr (BITS == 2) *reinterpret_cast<uint16_t *>(pk + j / 4) = (uint16_t)z;
+        else pk[j / 8] = (unsigned char)z;
+    }
+}
+
+// ------------------------------------------------------------------------------ prepare
+// Partial sums of squares in fp64: one CTA per (chunk of 2^chunk_log2 coordinates, worker).
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads)
+prepare_partial_kernel(PtrArray in, uint64_t d, uint32_t chunk_log2, uint64_t chunks_per_worker,
+                       double *__restrict__ partial)
+{
+    const uint64_t chunk = blockIdx.x;
+    const uint32_t wl = blockIdx.y;
+    const uint64_t j0 = chunk << chunk_log2;
+    const int n4 = 1 << (chunk_log2 - 2);
+    double s = 0.0;
+    for (int c = threadIdx.x; c < n4; c += kThreads) {
+        const uint64_t j = j0 + (uint64_t)c * 4;
+        if (j >= d) break;
+        float4 v;
+        if (BF16) {
+            const uint16_t *x = static_cast<const uint16_t *>(in.p[wl]);
+            uint32_t w0 = 0, w1 = 0;
+            if (j + 4 <= d) {
+                const uint2 q = __ldg(reinterpret_cast<const uint2 *>(x + j));
+                w0 = q.x; w1 = q.y;
+            } else {
+                for (int e = 0; e < 4; ++e)
+                    if (j + e < d) {
+                        const uint32_t h = (uint32_t)__ldg(x + j + e) << ((e & 1) * 16);
+                        if (e < 2) w0 |= h; else w1 |= h;
+                    }
+            }
+            v = make_float4(__uint_as_float(w0 << 16), __uint_as_float(w0 & 0xFFFF0000u),
+                            __uint_as_float(w1 << 16), __uint_as_float(w1 & 0xFFFF0000u));
+        } else {
+            v = load_f32x4_masked(static_cast<const float *>(in.p[wl]), j, d);
+        }
+        s = fma((double)v.x, (double)v.x, s);
+        s = fma((double)v.y, (double)v.y, s);
+        s = fma((double)v.z, (double)v.z, s);
+        s = fma((double)v.w, (double)v.w, s);
+    }
+    __shared__ double red[kThreads / 32];
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_down_sync(0xFFFFFFFFu, s, off);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < kThreads / 32; ++w) t += red[w];
+        partial[(uint64_t)wl * chunks_per_worker + chunk] = t;
+    }
+}
+
+// M per block from the partial sums (Section 5.3: M = t_p * max_i ||x_i|| / sqrt(B)).
+__global__ void prepare_final_kernel(const double *__restrict__ partial, uint32_t n,
+                                     uint64_t nblocks, uint64_t chunks_per_block,
+                                     uint64_t chunks_per_worker, double t_p, uint32_t k,
+                                     float *__restrict__ scales, DeviceBlock *dev)
+{
+    const uint64_t blk = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (blk >= nblocks) return;
+    double ell = 0.0;
+    for (uint32_t i = 0; i < n; ++i) {
+        double s = 0.0;
+        const double *p = partial + (uint64_t)i * chunks_per_worker + blk * chunks_per_block;
+        for (uint64_t c = 0; c < chunks_per_block; ++c) s += p[c];
+        const double norm = sqrt(s);
+        if (norm > ell || norm != norm) ell = norm;    // a NaN norm sticks
+    }
+    float M = (float)(t_p * ell / sqrt((double)((uint64_t)1 << k)));
+    uint32_t flags = 0;
+    if (!isfinite(M)) { M = 0.0f; flags |= THC_STATUS_NONFINITE; }
+    if (M == 0.0f) flags |= THC_STATUS_ZERO_BLOCK;
+    scales[blk] = M;
+    if (flags) atomicOr(&dev->status, flags);
+}
+
+// ---------------------------------------------------------------------------- aggregate
+// Y[j] = sum_i T[z_i[j]] (Algorithm 2, PS line).  One thread per 32 coordinates.
+template <int BITS, int W>
+__global__ void __launch_bounds__(kThreads)
+aggregate_kernel(PtrArray in, uint32_t n, uint64_t units, uint64_t d_pad, const DeviceBlock *dev,
+                 unsigned char *__restrict__ sum)
+{
+    __shared__ uint32_t T[256];
+    for (int z = threadIdx.x; z < (1 << BITS); z += kThreads) T[z] = dev->table[z];
+    __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        // coordinates past the last whole group of 32 (blocks of 8 or 16 coordinates only)
+        for (uint64_t j = units * 32; j < d_pad; ++j) {
+            uint32_t acc = 0;
+            for (uint32_t i = 0; i < n; ++i) {
+                const unsigned char byte = static_cast<const unsigned char *>(in.p[i])[j * BITS / 8];
+                acc += T[(byte >> ((j % (8 / BITS)) * BITS)) & ((1u << BITS) - 1u)];
+            }
+            if constexpr (W == 8) sum[j] = (unsigned char)acc;
+            else if constexpr (W == 16) reinterpret_cast<uint16_t *>(sum)[j] = (uint16_t)acc;
+            else reinterpret_cast<uint32_t *>(sum)[j] = acc;
+        }
+    }
+    constexpr int kInWords = BITS;                 // 32 indices * BITS bits = BITS words
+    for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < units;
+         u += (uint64_t)gridDim.x * kThreads) {
+        uint32_t acc[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) acc[e] = 0;
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint32_t *src = reinterpret_cast<const uint32_t *>(
+                static_cast<const unsigned char *>(in.p[i]) + u * (4 * BITS));
+            uint32_t w[kInWords];
+            if constexpr (BITS == 8) {
+                const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src));
+                const uint4 b = __ldg(reinterpret_cast<const uint4 *>(src) + 1);
+                w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w;
+                w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
+            } else if constexpr (BITS == 4) {
+                const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src));
+                w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w;
+            } else if constexpr (BITS == 2) {
+                const uint2 a = __ldg(reinterpret_cast<const uint2 *>(src));
+                w[0] = a.x; w[1] = a.y;
+            } else {
+                w[0] = __ldg(src);
+            }
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+                const int bit = e * BITS;
+                const uint32_t z = (w[bit >> 5] >> (bit & 31)) & ((1u << BITS) - 1u);
+                acc[e] += T[z];
+            }
+        }
+        unsigned char *dst = sum + u * (32 * W / 8);
+        if constexpr (W == 8) {
+            uint32_t o[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                o[q] = (acc[4 * q] & 0xFFu) | ((acc[4 * q + 1] & 0xFFu) << 8) |
+                       ((acc[4 * q + 2] & 0xFFu) << 16) | (acc[4 * q + 3] << 24);
+            reinterpret_cast<uint4 *>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
+            reinterpret_cast<uint4 *>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+        } else if constexpr (W == 16) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t o[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t)
+                    o[t] = (acc[8 * q + 2 * t] & 0xFFFFu) | (acc[8 * q + 2 * t + 1] << 16);
+                reinterpret_cast<uint4 *>(dst)[q] = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                reinterpret_cast<uint4 *>(dst)[q] =
+                    make_uint4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+        }
+    }
+}
+
+}  // namespace thc
+
+// =========================================================================== host side
+using namespace thc;
+
+struct thc_ctx {
+    thc_config cfg;
+    uint32_t acc_bits;
+    bool identity;
+    int device;                 // -1: no CUDA device, host-only context
+    DeviceBlock *dev;
+    PhiloxKeys keys;
+    uint32_t lut_rep;
+    int sm_count;
+};
+
+static thread_local cudaError_t g_last_cuda = cudaSuccess;
+static thread_local char g_err_text[256];
+
+static int cuda_fail(cudaError_t e)
+{
+    g_last_cuda = e;
+    return THC_ECUDA;
+}
+
+#define THC_CUDA(call)                                        \
+    do {                                                      \
+        cudaError_t e__ = (call);                             \
+        if (e__ != cudaSuccess) return cuda_fail(e__);        \
+    } while (0)
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+const char *thc_version(void) { return "thc-b200 0.1 (sm_100a)"; }
+
+const char *thc_strerror(int code)
+{
+    switch (code) {
+    case THC_OK: return "ok";
+    case THC_EINVAL: return "invalid configuration or argument";
+    case THC_EUNSUPPORTED: return "unsupported configuration";
+    case THC_EWORKSPACE: return "workspace too small (see thc_sizes)";
+    case THC_ECUDA:
+        if (g_last_cuda == cudaSuccess) return "CUDA error: context has no device";
+        snprintf(g_err_text, sizeof g_err_text, "CUDA error: %s", cudaGetErrorString(g_last_cuda));
+        return g_err_text;
+    default: return "unknown error code";
+    }
+}
+
+static int validate_config(const thc_config *c, uint32_t *acc_bits, bool *identity)
+{
+    if (c == nullptr) return THC_EINVAL;
+    if (!(c->bits == 1 || c->bits == 2 || c->bits == 4 || c->bits == 8)) return THC_EINVAL;
+    const uint32_t levels = 1u << c->bits;
+    if (c->granularity < levels - 1) return THC_EINVAL;
+    if (c->granularity > 255) return THC_EUNSUPPORTED;
+    if (c->table[0] != 0 || c->table[levels - 1] != c->granularity) return THC_EINVAL;
+    for (uint32_t z = 0; z + 1 < levels; ++z)
+        if (c->table[z + 1] <= c->table[z]) return THC_EINVAL;
+    if (!(c->t_p > 0.0) || !isfinite(c->t_p)) return THC_EINVAL;
+    if (c->log2_block < 3 || c->log2_block > 24) return THC_EINVAL;
+    if (c->in_dtype != THC_F32 && c->in_dtype != THC_BF16) return THC_EINVAL;
+    if (c->workers == 0 || c->workers > THC_MAX_WORKERS) return THC_EINVAL;
+    const uint64_t max_sum = (uint64_t)c->workers * c->granularity;
+    uint32_t w = c->acc_bits;
+    if (w == 0) w = max_sum <= 0xFFu ? 8 : max_sum <= 0xFFFFu ? 16 : 32;
+    if (!(w == 8 || w == 16 || w == 32)) return THC_EINVAL;
+    if (w < 32 && max_sum > ((1ull << w) - 1)) return THC_EINVAL;
+    *acc_bits = w;
+    bool id = c->granularity == levels - 1;
+    for (uint32_t z = 0; id && z < levels; ++z) id = c->table[z] == z;
+    *identity = id;
+    return THC_OK;
+}
+
+int thc_create(const thc_config *cfg, thc_ctx **out)
+{
+    if (out == nullptr) return THC_EINVAL;
+    *out = nullptr;
+    uint32_t acc_bits = 0;
+    bool identity = false;
+    const int rc = validate_config(cfg, &acc_bits, &identity);
+    if (rc != THC_OK) return rc;
+    thc_ctx *ctx = new (std::nothrow) thc_ctx;
+    if (ctx == nullptr) return THC_EINVAL;
+    ctx->cfg = *cfg;
+    ctx->acc_bits = acc_bits;
+    ctx->identity = identity;
+    ctx->device = -1;
+    ctx->dev = nullptr;
+    ctx->sm_count = 148;
+    uint32_t k0 = (uint32_t)cfg->seed, k1 = (uint32_t)(cfg->seed >> 32);
+    for (int r = 0; r < 10; ++r) {
+        ctx->keys.k[2 * r] = k0;
+        ctx->keys.k[2 * r + 1] = k1;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    const uint32_t g = cfg->granularity;
+    ctx->lut_rep = ((g + 1) * 32 * 8 <= (uint32_t)kLutRepMaxBytes) ? 32 : 1;
+
+    // host copy of the device block
+    DeviceBlock *h = new (std::nothrow) DeviceBlock;
+    if (h == nullptr) { delete ctx; return THC_EINVAL; }
+    memset(h, 0, sizeof *h);
+    const uint32_t levels = 1u << cfg->bits;
+    for (uint32_t z = 0; z < levels; ++z) h->table[z] = cfg->table[z];
+    for (uint32_t f = 0; f <= g; ++f) {
+        const uint32_t ff = f < g ? f : g - 1;            // y = g falls in the last interval
+        uint32_t z0 = 0;
+        while (z0 + 1 <= levels - 2 && cfg->table[z0 + 1] <= ff) ++z0;
+        const float tz = (float)cfg->table[z0];
+        uint32_t bits;
+        memcpy(&bits, &tz, 4);
+        h->lut_tz[f] = bits | z0;
+        h->lut_r16[f] = 65536.0f / (float)(cfg->table[z0 + 1] - cfg->table[z0]);
+    }
+
+    int count = 0;
+    if (cudaGetDeviceCount(&count) == cudaSuccess && count > 0) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->dev), sizeof(DeviceBlock));
+        if (e == cudaSuccess) e = cudaMemcpy(ctx->dev, h, sizeof(DeviceBlock), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) {
+            if (ctx->dev) cudaFree(ctx->dev);
+            delete h;
+            delete ctx;
+            return cuda_fail(e);
+        }
+        ctx->device = dev;
+    } else {
+        (void)cudaGetLastError();   // no device: host-only context
+    }
+    delete h;
+    *out = ctx;
+    return THC_OK;
+}
+
+int thc_destroy(thc_ctx *ctx)
+{
+    if (ctx == nullptr) return THC_OK;
+    if (ctx->dev != nullptr) cudaFree(ctx->dev);
+    delete ctx;
+    return THC_OK;
+}
+
+static uint64_t round_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+
+int thc_sizes(const thc_ctx *ctx, uint64_t d, uint32_t n_local, thc_sizes_t *s)
+{
+    if (ctx == nullptr || s == nullptr || d == 0 || n_local == 0 || n_local > THC_MAX_WORKERS)
+        return THC_EINVAL;
+    const uint32_t k = ctx->cfg.log2_block;
+    const uint64_t B = 1ull << k;
+    if (d > (1ull << 40)) return THC_EINVAL;
+    memset(s, 0, sizeof *s);
+    s->d_pad = round_up(d, B);
+    s->nblocks = s->d_pad / B;
+    s->packed_bytes = s->d_pad * ctx->cfg.bits / 8;
+    s->sum_bytes = s->d_pad * ctx->acc_bits / 8;
+    s->rotated_bytes = s->d_pad * 4;
+    s->acc_bits = ctx->acc_bits;
+    const uint32_t chunk_log2 = k < (uint32_t)kTileLog2 ? k : (uint32_t)kTileLog2;
+    const uint64_t prepare_ws = (uint64_t)n_local * (s->d_pad >> chunk_log2) * 8;
+    const uint64_t two_pass_ws = k > (uint32_t)kTileLog2 ? (uint64_t)n_local * s->d_pad * 4 : 0;
+    s->workspace_bytes = round_up((prepare_ws > two_pass_ws ? prepare_ws : two_pass_ws) + 256, 256);
+    return THC_OK;
+}
+
+static int check_launch_ctx(const thc_ctx *ctx)
+{
+    if (ctx == nullptr) return THC_EINVAL;
+    if (ctx->device < 0 || ctx->dev == nullptr) { g_last_cuda = cudaSuccess; return THC_ECUDA; }
+    return THC_OK;
+}
+
+static int check_ptr_array(const void *const *arr, uint32_t n)
+{
+    if (arr == nullptr) return THC_EINVAL;
+    for (uint32_t i = 0; i < n; ++i)
+        if (arr[i] == nullptr || !aligned16(arr[i])) return THC_EINVAL;
+    return THC_OK;
+}
+
+int thc_prepare(thc_ctx *ctx, const void *const *grads, uint32_t n, uint64_t d, float *scales,
+                void *workspace, uint64_t workspace_bytes, void *stream)
+{
+    int rc = check_launch_ctx(ctx);
+    if (rc != THC_OK) return rc;
+    thc_sizes_t sz;
+    if ((rc = thc_sizes(ctx, d, n, &sz)) != THC_OK) return rc;
+    if ((rc = check_ptr_array(grads, n)) != THC_OK) return rc;
+    if (scales == nullptr || workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
+    if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint32_t k = ctx->cfg.log2_block;
+    const uint32_t chunk_log2 = k < (uint32_t)kTileLog2 ? k : (uint32_t)kTileLog2;
+    const uint64_t chunks_per_worker = sz.d_pad >> chunk_log2;
+    const uint64_t chunks_per_block = 1ull << (k - chunk_log2);
+    if (chunks_per_worker > 0x7FFFFFFFull) return THC_EUNSUPPORTED;
+    PtrArray in;
+    memset(&in, 0, sizeof in);
+    for (uint32_t i = 0; i < n; ++i) in.p[i] = grads[i];
+    double *partial = static_cast<double *>(workspace);
+    const dim3 grid((unsigned)chunks_per_worker, n);
+    if (ctx->cfg.in_dtype == THC_BF16)
+        prepare_partial_kernel<true><<<grid, kThreads, 0, st>>>(in, d, chunk_log2, chunks_per_worker, partial);
+    else
+        prepare_partial_kernel<false><<<grid, kThreads, 0, st>>>(in, d, chunk_log2, chunks_per_worker, partial);
+    THC_CUDA(cudaGetLastError());
+    prepare_final_kernel<<<(unsigned)((sz.nblocks + 127) / 128), 128, 0, st>>>(
+        partial, n, sz.nblocks, chunks_per_block, chunks_per_worker, ctx->cfg.t_p, k, scales, ctx->dev);
+    THC_CUDA(cudaGetLastError());
+    return THC_OK;
+}
+
+// ---- tile-kernel dispatch
+typedef void (*tile_kernel_t)(TileGeom, PtrArray, MutPtrArray, MutPtrArray, const float *,
+                              DeviceBlock *, PhiloxKeys);
+
+template <int LOAD, int STORE>
+static tile_kernel_t pick_tile_kernel(uint32_t bits, bool identity)
+{
+    if constexpr (STORE != kStoreQuant) {
+        return rht_tile_kernel<LOAD, STORE, 4, true>;
+    } else {
+    switch (bits) {
+    case 1: return identity ? rht_tile_kernel<LOAD, STORE, 1, true> : rht_tile_kernel<LOAD, STORE, 1, false>;
+    case 2: return identity ? rht_tile_kernel<LOAD, STORE, 2, true> : rht_tile_kernel<LOAD, STORE, 2, false>;
+    case 4: return identity ? rht_tile_kernel<LOAD, STORE, 4, true> : rht_tile_kernel<LOAD, STORE, 4, false>;
+    default: return identity ? rht_tile_kernel<LOAD, STORE, 8, true> : rht_tile_kernel<LOAD, STORE, 8, false>;
+    }
+    }
+}
+
+static size_t tile_smem_bytes(const thc_ctx *ctx, const TileGeom &g)
+{
+    return (size_t)kTileElems * 4 + kSignWordsMax * 4 + (size_t)g.blocks_in_tile * 8 +
+           (size_t)(ctx->cfg.granularity + 1) * ctx->lut_rep * 8;
+}
+
+static int launch_tile(const thc_ctx *ctx, tile_kernel_t kern, const TileGeom &g, uint64_t tiles,
+                       uint32_t n_local, const PtrArray &in, const MutPtrArray &out,
+                       const MutPtrArray &rot, const float *scales, cudaStream_t st)
+{
+    if (tiles > 0x7FFFFFFFull) return THC_EUNSUPPORTED;
+    const size_t smem = tile_smem_bytes(ctx, g);
+    THC_CUDA(cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<dim3((unsigned)tiles, n_local), kThreads, smem, st>>>(g, in, out, rot, scales, ctx->dev,
+                                                                 ctx->keys);
+    THC_CUDA(cudaGetLastError());
+    return THC_OK;
+}
+
+static TileGeom base_geom(const thc_ctx *ctx, const thc_sizes_t &sz, uint64_t d, uint32_t round)
+{
+    TileGeom g;
+    memset(&g, 0, sizeof g);
+    g.d = d;
+    g.d_pad = sz.d_pad;
+    g.k = ctx->cfg.log2_block;
+    g.lut_rep = ctx->lut_rep;
+    g.granularity = ctx->cfg.granularity;
+    g.round = round;
+    g.c_block = (float)(1.0 / sqrt((double)(1ull << g.k)));
+    return g;
+}
+
+static void geom_pass_a(TileGeom &g)
+{
+    g.row_log2 = 0;
+    g.col_log2 = kTileLog2;
+    g.row_stride = 0;
+    g.lo_cbit = 0;
+    g.hi_cbit = (g.k < (uint32_t)kTileLog2 ? g.k : (uint32_t)kTileLog2) - 2;
+    g.blocks_in_tile = g.k >= (uint32_t)kTileLog2 ? 1u : 1u << (kTileLog2 - g.k);
+}
+
+static void geom_pass_b(TileGeom &g)
+{
+    g.row_log2 = g.k - kTileLog2;
+    g.col_log2 = kTileLog2 - g.row_log2;
+    g.row_stride = 1ull << kTileLog2;
+    g.lo_cbit = g.col_log2 - 2;
+    g.hi_cbit = kTileLog2 - 2;
+    g.blocks_in_tile = 1;
+}
+
+int thc_compress(thc_ctx *ctx, const void *const *grads, uint32_t n_local, uint32_t worker_base,
+                 uint64_t d, uint32_t round, const float *scales, void *const *packed,
+                 float *const *rotated, void *workspace, uint64_t workspace_bytes, void *stream)
+{
+    int rc = check_launch_ctx(ctx);
+    if (rc != THC_OK) return rc;
+    thc_sizes_t sz;
+    if ((rc = thc_sizes(ctx, d, n_local, &sz)) != THC_OK) return rc;
+    if ((rc = check_ptr_array(grads, n_local)) != THC_OK) return rc;
+    if ((rc = check_ptr_array(packed, n_local)) != THC_OK) return rc;
+    if (scales == nullptr) return THC_EINVAL;
+    if ((uint64_t)worker_base + n_local > 0xFFFFFFFFull) return THC_EINVAL;
+    const uint32_t k = ctx->cfg.log2_block;
+    const bool two_pass = k > (uint32_t)kTileLog2;
+    if (two_pass) {
+        if (workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
+        if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PtrArray in;
+    MutPtrArray out, rot, ws;
+    memset(&in, 0, sizeof in);
+    memset(&out, 0, sizeof out);
+    memset(&rot, 0, sizeof rot);
+    memset(&ws, 0, sizeof ws);
+    for (uint32_t i = 0; i < n_local; ++i) {
+        in.p[i] = grads[i];
+        out.p[i] = packed[i];
+        if (rotated != nullptr && rotated[i] != nullptr) {
+            if (!aligned16(rotated[i])) return THC_EINVAL;
+            rot.p[i] = rotated[i];
+        }
+    }
+    ws.p[0] = workspace;
+    TileGeom g = base_geom(ctx, sz, d, round);
+    g.worker_base = worker_base;
+    const bool bf16 = ctx->cfg.in_dtype == THC_BF16;
+    const uint64_t tiles = (sz.d_pad + kTileElems - 1) / kTileElems;
+    geom_pass_a(g);
+    if (!two_pass) {
+        tile_kernel_t kern = bf16 ? pick_tile_kernel<kLoadGradBF16, kStoreQuant>(ctx->cfg.bits, ctx->identity)
+                                  : pick_tile_kernel<kLoadGradF32, kStoreQuant>(ctx->cfg.bits, ctx->identity);
+        return launch_tile(ctx, kern, g, tiles, n_local, in, out, rot, scales, st);
+    }
+    tile_kernel_t ka = bf16 ? pick_tile_kernel<kLoadGradBF16, kStoreRaw>(ctx->cfg.bits, ctx->identity)
+                            : pick_tile_kernel<kLoadGradF32, kStoreRaw>(ctx->cfg.bits, ctx->identity);
+    if ((rc = launch_tile(ctx, ka, g, tiles, n_local, in, ws, rot, scales, st)) != THC_OK) return rc;
+    geom_pass_b(g);
+    PtrArray wsin;
+    memset(&wsin, 0, sizeof wsin);
+    wsin.p[0] = workspace;
+    tile_kernel_t kb = pick_tile_kernel<kLoadRaw, kStoreQuant>(ctx->cfg.bits, ctx->identity);
+    return launch_tile(ctx, kb, g, tiles, n_local, wsin, out, rot, scales, st);
+}
+
+int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, uint32_t round,
+                   const float *scales, float *outp, void *workspace, uint64_t workspace_bytes,
+                   void *stream)
+{
+    int rc = check_launch_ctx(ctx);
+    if (rc != THC_OK) return rc;
+    thc_sizes_t sz;
+    if ((rc = thc_sizes(ctx, d, 1, &sz)) != THC_OK) return rc;
+    if (sum == nullptr || outp == nullptr || scales == nullptr || divisor == 0) return THC_EINVAL;
+    if (!aligned16(sum) || !aligned16(outp)) return THC_EINVAL;
+    const uint32_t k = ctx->cfg.log2_block;
+    const bool two_pass = k > (uint32_t)kTileLog2;
+    if (two_pass) {
+        if (workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
+        if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PtrArray in;
+    MutPtrArray out, rot, ws;
+    memset(&in, 0, sizeof in);
+    memset(&out, 0, sizeof out);
+    memset(&rot, 0, sizeof rot);
+    memset(&ws, 0, sizeof ws);
+    in.p[0] = sum;
+    out.p[0] = outp;
+    ws.p[0] = workspace;
+    TileGeom g = base_geom(ctx, sz, d, round);
+    g.divisor = divisor;
+    const uint64_t tiles = (sz.d_pad + kTileElems - 1) / kTileElems;
+    geom_pass_a(g);
+    const uint32_t w = ctx->acc_bits;
+    tile_kernel_t k1;
+    if (!two_pass) {
+        k1 = w == 8 ? pick_tile_kernel<kLoadSum8, kStoreOut>(4, true)
+           : w == 16 ? pick_tile_kernel<kLoadSum16, kStoreOut>(4, true)
+                     : pick_tile_kernel<kLoadSum32, kStoreOut>(4, true);
+        return launch_tile(ctx, k1, g, tiles, 1, in, out, rot, scales, st);
+    }
+    k1 = w == 8 ? pick_tile_kernel<kLoadSum8, kStoreRaw>(4, true)
+       : w == 16 ? pick_tile_kernel<kLoadSum16, kStoreRaw>(4, true)
+                 : pick_tile_kernel<kLoadSum32, kStoreRaw>(4, true);
+    if ((rc = launch_tile(ctx, k1, g, tiles, 1, in, ws, rot, scales, st)) != THC_OK) return rc;
+    geom_pass_b(g);
+    PtrArray wsin;
+    memset(&wsin, 0, sizeof wsin);
+    wsin.p[0] = workspace;
+    return launch_tile(ctx, pick_tile_kernel<kLoadRaw, kStoreOut>(4, true), g, tiles, 1, wsin, out,
+                       rot, scales, st);
+}
+
+int thc_quantize_rotated(thc_ctx *ctx, const float *const *rotated, uint32_t n_local,
+                         uint32_t worker_base, uint64_t d, uint32_t round, const float *scales,
+                         void *const *packed, void *stream)
+{
+    int rc = check_launch_ctx(ctx);
+    if (rc != THC_OK) return rc;
+    thc_sizes_t sz;
+    if ((rc = thc_sizes(ctx, d, n_local, &sz)) != THC_OK) return rc;
+    if ((rc = check_ptr_array(reinterpret_cast<const void *const *>(rotated), n_local)) != THC_OK) return rc;
+    if ((rc = check_ptr_array(packed, n_local)) != THC_OK) return rc;
+    if (scales == nullptr) return THC_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PtrArray in;
+    MutPtrArray out;
+    memset(&in, 0, sizeof in);
+    memset(&out, 0, sizeof out);
+    for (uint32_t i = 0; i < n_local; ++i) { in.p[i] = rotated[i]; out.p[i] = packed[i]; }
+    const uint64_t units = sz.d_pad / 8;
+    uint64_t blocks = (units + kThreads - 1) / kThreads;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    const dim3 grid((unsigned)blocks, n_local);
+    const uint32_t k = ctx->cfg.log2_block, g = ctx->cfg.granularity;
+#define THC_QR(B, I) quantize_rotated_kernel<B, I><<<grid, kThreads, 0, st>>>( \
+        in, out, sz.d_pad, k, g, round, worker_base, scales, ctx->dev, ctx->keys)
+    switch (ctx->cfg.bits) {
+    case 1: if (ctx->identity) THC_QR(1, true); else THC_QR(1, false); break;
+    case 2: if (ctx->identity) THC_QR(2, true); else THC_QR(2, false); break;
+    case 4: if (ctx->identity) THC_QR(4, true); else THC_QR(4, false); break;
+    default: if (ctx->identity) THC_QR(8, true); else THC_QR(8, false); break;
+    }
+#undef THC_QR
+    THC_CUDA(cudaGetLastError());
+    return THC_OK;
+}
+
+int thc_aggregate(thc_ctx *ctx, const void *const *packed, uint32_t n, uint64_t d, void *sum,
+                  void *stream)
+{
+    int rc = check_launch_ctx(ctx);
+    if (rc != THC_OK) return rc;
+    if (n == 0 || n > ctx->cfg.workers) return THC_EINVAL;
+    thc_sizes_t sz;
+    if ((rc = thc_sizes(ctx, d, n, &sz)) != THC_OK) return rc;
+    if ((rc = check_ptr_array(packed, n)) != THC_OK) return rc;
+    if (sum == nullptr || !aligned16(sum)) return THC_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PtrArray in;
+    memset(&in, 0, sizeof in);
+    for (uint32_t i = 0; i < n; ++i) in.p[i] = packed[i];
+    const uint64_t units = sz.d_pad / 32;       // the kernel finishes a tail of 8..24 itself
+    uint64_t blocks = (units + kThreads - 1) / kThreads;
+    if (blocks == 0) blocks = 1;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    unsigned char *s = static_cast<unsigned char *>(sum);
+#define THC_AG(B, W) aggregate_kernel<B, W><<<(unsigned)blocks, kThreads, 0, st>>>(in, n, units, sz.d_pad, ctx->dev, s)
+#define THC_AGW(B)                                       \
+    do {                                                 \
+        if (ctx->acc_bits == 8) THC_AG(B, 8);            \
+        else if (ctx->acc_bits == 16) THC_AG(B, 16);     \
+        else THC_AG(B, 32);                              \
+    } while (0)
+    switch (ctx->cfg.bits) {
+    case 1: THC_AGW(1); break;
+    case 2: THC_AGW(2); break;
+    case 4: THC_AGW(4); break;
+    default: THC_AGW(8); break;
+    }
+#undef THC_AGW
+#undef THC_AG
+    THC_CUDA(cudaGetLastError());
+    return THC_OK;
+}
+
+int thc_status(thc_ctx *ctx, uint32_t *flags, void *stream)
+{
+    int rc = check_launch_ctx(ctx);
+    if (rc != THC_OK) return rc;
+    if (flags == nullptr) return THC_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    THC_CUDA(cudaMemcpyAsync(flags, &ctx->dev->status, 4, cudaMemcpyDeviceToHost, st));
+    THC_CUDA(cudaMemsetAsync(&ctx->dev->status, 0, 4, st));
+    THC_CUDA(cudaStreamSynchronize(st));
+    return THC_OK;
+}

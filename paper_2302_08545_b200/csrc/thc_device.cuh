@@ -1,0 +1,215 @@
+// Device-side building blocks of libthc: counter RNG, packed-fp32 butterflies, the
+// swizzled shared-memory Hadamard rounds and the per-coordinate quantiser.
+//
+// Arithmetic contract (what makes results reproducible bit for bit):
+//   * every fp32 operation is a single IEEE round-to-nearest operation; the file is
+//     compiled with -fmad=false, so only the fmaf() calls written here are fused;
+//   * the Hadamard transform is radix-2 with stages in ascending stride order and one
+//     multiplication by (float)(1/sqrt(B)) at the end (THC paper, Section 5.1: the RHT is
+//     (1/sqrt d) H D x; the paper fixes no evaluation order, this is the library's);
+//   * random bits come from Philox4x32-10 keyed by the shared seed.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace thc {
+
+constexpr int kTileLog2 = 14;                  // a CTA transforms 2^14 coordinates at a time
+constexpr int kTileElems = 1 << kTileLog2;
+constexpr int kTileChunks = kTileElems / 4;    // 16-byte chunks
+constexpr int kThreads = 256;
+constexpr int kSignWordsMax = 1024;            // sign words a tile can need
+constexpr int kLutRepMaxBytes = 16384;
+
+// Lives in the context's device block.
+struct DeviceBlock {
+    uint32_t status;             // THC_STATUS_* bits
+    uint32_t counters[31];       // scheduling counters (self-resetting)
+    uint32_t lut_tz[256];        // by floor(y): float bits of T[z0] | z0
+    float    lut_r16[256];       // by floor(y): 65536 / (T[z0+1] - T[z0])
+    uint32_t table[256];         // T
+};
+
+struct PhiloxKeys { uint32_t k[20]; };         // the ten round keys, precomputed on the host
+
+// Philox4x32-10 (Salmon et al., SC'11).
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               const PhiloxKeys &keys)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ keys.k[2 * r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ keys.k[2 * r + 1];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// Sign diagonal D of the RHT (Section 5.1; "D^r" in Algorithm 3): one Philox call covers
+// 128 consecutive padded coordinates, counter = (j/128 lo, j/128 hi, 0xFFFFFFFF, round).
+__device__ __forceinline__ uint4 sign_call(uint64_t j, uint32_t round, const PhiloxKeys &keys)
+{
+    const uint64_t call = j >> 7;
+    return philox4x32_10((uint32_t)call, (uint32_t)(call >> 32), 0xFFFFFFFFu, round, keys);
+}
+
+// Rounding variates (Section 4.1 needs one uniform per coordinate; Appendix A.2 asks that
+// workers draw independently): one call covers 8 consecutive coordinates, 16 bits each,
+// counter = (j/8 lo, j/8 hi, worker, round).
+__device__ __forceinline__ uint4 round_call(uint64_t j, uint32_t worker, uint32_t round,
+                                            const PhiloxKeys &keys)
+{
+    const uint64_t call = j >> 3;
+    return philox4x32_10((uint32_t)call, (uint32_t)(call >> 32), worker, round, keys);
+}
+
+// ---------------------------------------------------------------- packed fp32 arithmetic
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
+
+__device__ __forceinline__ float2 sub2(float2 a, float2 b)
+{
+    uint64_t ra, rb, rc;
+    asm("mov.b64 %0, {%1,%2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1,%2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(rc) : "l"(ra), "l"(rb));
+    float2 c;
+    asm("mov.b64 {%0,%1}, %2;" : "=f"(c.x), "=f"(c.y) : "l"(rc));
+    return c;
+}
+
+// One radix-2 butterfly on four independent columns: (a, b) <- (a + b, a - b).
+__device__ __forceinline__ void butterfly(float4 &a, float4 &b)
+{
+    const float2 alo = make_float2(a.x, a.y), ahi = make_float2(a.z, a.w);
+    const float2 blo = make_float2(b.x, b.y), bhi = make_float2(b.z, b.w);
+    const float2 slo = add2(alo, blo), shi = add2(ahi, bhi);
+    const float2 dlo = sub2(alo, blo), dhi = sub2(ahi, bhi);
+    a = make_float4(slo.x, slo.y, shi.x, shi.y);
+    b = make_float4(dlo.x, dlo.y, dhi.x, dhi.y);
+}
+
+// Stages of stride 1 and 2 inside one 16-byte chunk (coordinates 4q .. 4q+3).
+__device__ __forceinline__ float4 stages01(float4 v)
+{
+    const float x = v.x + v.y, y = v.x - v.y, z = v.z + v.w, w = v.z - v.w;
+    const float2 s = add2(make_float2(x, y), make_float2(z, w));
+    const float2 d = sub2(make_float2(x, y), make_float2(z, w));
+    return make_float4(s.x, s.y, d.x, d.y);
+}
+
+__device__ __forceinline__ float4 scale4(float4 v, float c)
+{
+    const float2 c2 = make_float2(c, c);
+    const float2 lo = __fmul2_rn(make_float2(v.x, v.y), c2);
+    const float2 hi = __fmul2_rn(make_float2(v.z, v.w), c2);
+    return make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+
+// Flip the signs of a chunk by bits [0,4) of `bits` (bit e set -> element e negated).
+__device__ __forceinline__ float4 flip4(float4 v, uint32_t bits)
+{
+    v.x = __uint_as_float(__float_as_uint(v.x) ^ ((bits << 31) & 0x80000000u));
+    v.y = __uint_as_float(__float_as_uint(v.y) ^ ((bits << 30) & 0x80000000u));
+    v.z = __uint_as_float(__float_as_uint(v.z) ^ ((bits << 29) & 0x80000000u));
+    v.w = __uint_as_float(__float_as_uint(v.w) ^ ((bits << 28) & 0x80000000u));
+    return v;
+}
+
+// ------------------------------------------------------------------- shared-memory tile
+// The tile holds 4096 chunks.  Chunk c is stored at c ^ ((c >> 4) & 7): with this XOR every
+// access pattern below (consecutive chunks per lane, or one chunk per lane at any
+// power-of-two stride) touches eight distinct 16-byte bank groups per quarter warp.
+__device__ __forceinline__ int swz(int c) { return c ^ ((c >> 4) & 7); }
+
+// Butterfly stages on chunk-index bits [sp, sp+E) of the tile, ascending.  Each thread owns
+// whole groups of 2^E chunks, so the update is in place; callers separate rounds by a
+// block barrier.
+template <int E>
+__device__ __forceinline__ void fwht_round(float4 *tile, int sp, int tid)
+{
+    constexpr int N = 1 << E;
+    constexpr int kGroups = kTileChunks >> E;
+#pragma unroll 1
+    for (int G = tid; G < kGroups; G += kThreads) {
+        const int low = G & ((1 << sp) - 1);
+        const int base = ((G >> sp) << (sp + E)) | low;
+        float4 v[N];
+#pragma unroll
+        for (int m = 0; m < N; ++m) v[m] = tile[swz(base + (m << sp))];
+#pragma unroll
+        for (int t = 0; t < E; ++t) {
+#pragma unroll
+            for (int m = 0; m < N; ++m) {
+                if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < N; ++m) tile[swz(base + (m << sp))] = v[m];
+    }
+}
+
+// All stages on chunk bits [lo, hi), in rounds of at most four bits.
+__device__ __forceinline__ void fwht_rounds(float4 *tile, int lo, int hi, int tid)
+{
+    int sp = lo;
+    while (sp < hi) {
+        const int e = min(4, hi - sp);
+        switch (e) {
+        case 4: fwht_round<4>(tile, sp, tid); break;
+        case 3: fwht_round<3>(tile, sp, tid); break;
+        case 2: fwht_round<2>(tile, sp, tid); break;
+        default: fwht_round<1>(tile, sp, tid); break;
+        }
+        sp += e;
+        __syncthreads();
+    }
+}
+
+// --------------------------------------------------------------------------- quantiser
+// Stochastic quantisation of eight consecutive rotated coordinates to table indices
+// (Algorithm 2, worker lines; Section 4.1 for the rounding rule):
+//   y = clamp(fma(r, kappa, g/2), 0, g)        position on the grid <g+1>, truncated
+//   z0 = index of the table value at or below y, up iff u16 < RN(2^16 (y - T[z0]) / gap)
+// kappa = 0 and half_g = 0 encode a degenerate block (every index 0).
+// `lut` points at this lane's copy of the (T[z0] | z0, 65536/gap) pairs, `lut_stride`
+// entries apart per floor value.  Returns the indices packed BITS apiece, coordinate 0 in
+// the low bits.
+template <int BITS, bool IDENTITY>
+__device__ __forceinline__ uint64_t quantize8(const float (&r)[8], float kappa, float half_g,
+                                              float gf, uint4 rnd, const uint2 *lut,
+                                              int lut_stride)
+{
+    const uint32_t words[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+    uint64_t out = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        float y = fmaf(r[e], kappa, half_g);
+        y = fminf(fmaxf(y, 0.0f), gf);
+        const float t = __fadd_rd(y, 8388608.0f);              // 2^23 + floor(y)
+        const uint32_t u16 = (e & 1) ? (words[e >> 1] >> 16) : (words[e >> 1] & 0xFFFFu);
+        const uint32_t ub = u16 | 0x4B000000u;                 // bits of 2^23 + u16
+        uint32_t z0;
+        float tau;
+        if (IDENTITY) {
+            z0 = __float_as_uint(t) & 0xFFu;
+            const float delta = y - (t - 8388608.0f);
+            tau = fmaf(delta, 65536.0f, 8388608.0f);
+        } else {
+            const uint32_t f = __float_as_uint(t) & 0xFFu;
+            const uint2 entry = lut[f * lut_stride];
+            z0 = entry.x & 0xFFu;
+            const float delta = y - __uint_as_float(entry.x & 0xFFFFFF00u);
+            tau = fmaf(delta, __uint_as_float(entry.y), 8388608.0f);
+        }
+        const uint32_t z = z0 + (ub < __float_as_uint(tau) ? 1u : 0u);
+        out |= (uint64_t)z << (e * BITS);
+    }
+    return out;
+}
+
+}  // namespace thc

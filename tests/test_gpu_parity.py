@@ -1,0 +1,234 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, on the same seeded inputs.
+
+Bars (stated by the benchmark definition):
+  * packed indices and aggregated sums: bit-exact when both sides quantise the same rotated
+    input;
+  * end to end: max |err| <= 1e-5 * M of the coordinate's block, at most 1e-6 of the
+    indices differing.
+Both sides are always given the same `scales` array (the GPU's), so a last-bit difference
+in M cannot pass for index flips; thc_prepare is tested on its own.
+"""
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from paper_2302_08545_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+T4_30 = W.TABLES[(4, 30)]
+
+
+def _mk(n, d, k, bits=4, g=30, table=T4_30, in_dtype="f32", name="cfg1_x", t_p=W.T_P["1/32"]):
+    return W.Workload(name, n=n, d=d, log2_block=k, bits=bits, granularity=g, table=tuple(table),
+                      in_dtype=in_dtype, data_seed=4242 + d % 97 + k, t_p=t_p)
+
+
+def _ocfg(w):
+    return O.Config(bits=w.bits, granularity=w.granularity, table=tuple(w.table), t_p=w.t_p,
+                    log2_block=w.log2_block, seed=w.seed)
+
+
+def _inputs(w):
+    x = W.generate(w)
+    xf = O.bf16_to_f32(x) if w.in_dtype == "bf16" else x
+    return x, xf
+
+
+def _gpu_round(w, x, rnd=0, acc_bits=0, want_rotated=True):
+    import torch
+    from paper_2302_08545_b200 import runner
+    ctx = runner.context_for(w, acc_bits=acc_bits)
+    r = runner.Round(ctx, w.n, w.d, w.in_dtype, want_rotated=want_rotated)
+    r.upload(x)
+    r.run(rnd)
+    torch.cuda.synchronize()
+    return ctx, r
+
+
+def _block_scale_per_coord(scl, w, count):
+    return np.repeat(scl.astype(np.float64), w.block)[:count]
+
+
+def check_round(w, rnd=0, acc_bits=0, expect_exact_rotation=True):
+    x, xf = _inputs(w)
+    ctx, r = _gpu_round(w, x, rnd, acc_bits)
+    c = _ocfg(w)
+    sz = r.sz
+    scl = r.scales.cpu().numpy()
+
+    # thc_prepare on its own: equal as fp32 up to summation order (<= 1 ulp, rare)
+    scl_ref = O.scales(xf, c)
+    ulp = np.abs(scl.view(np.int32).astype(np.int64) - scl_ref.view(np.int32).astype(np.int64))
+    assert ulp.max() <= 1, "scale differs by more than one ulp"
+    assert (ulp > 0).mean() <= max(1e-3, 1.0 / scl.size) or scl.size < 1000
+
+    flips = 0
+    total_idx = 0
+    packed_gpu = np.stack([p.cpu().numpy() for p in r.packed])
+    for i in range(w.n):
+        rot_gpu = r.rotated[i].cpu().numpy()
+        rot_ref = O.rht_forward(xf[i], c, rnd)
+        if expect_exact_rotation:
+            assert np.array_equal(rot_gpu.view(np.uint32), rot_ref.view(np.uint32)), \
+                f"worker {i}: rotated coordinates differ from the oracle's"
+        # T1: same rotated input on both sides -> packed bytes identical
+        z_from_gpu_rot = O.pack(O.quantize(rot_gpu, scl, c, rnd, i), w.bits)
+        assert np.array_equal(packed_gpu[i], z_from_gpu_rot), f"worker {i}: packed indices differ"
+        z_ref = O.quantize(rot_ref, scl, c, rnd, i)
+        z_gpu = O.unpack(packed_gpu[i], sz.d_pad, w.bits)
+        flips += int((z_ref != z_gpu).sum())
+        total_idx += z_ref.size
+    assert flips <= 1e-6 * total_idx, f"{flips} of {total_idx} indices differ"
+
+    # aggregate: exact integers
+    wbits = sz.acc_bits
+    sum_ref = O.aggregate(packed_gpu, sz.d_pad, c, wbits)
+    sum_gpu = r.sum_numpy()
+    assert np.array_equal(sum_gpu, sum_ref), "aggregated sums differ"
+
+    # decompress of the same sums
+    out_gpu = r.out.cpu().numpy()
+    out_ref = O.decompress(sum_gpu, w.n, w.d, scl, c, rnd)
+    M = _block_scale_per_coord(scl, w, w.d)
+    err = np.abs(out_gpu.astype(np.float64) - out_ref.astype(np.float64))
+    assert np.all(err <= 1e-5 * M + 0.0), f"decompress error {err.max()} vs bound"
+    # end to end against the oracle's own round
+    if flips == 0:
+        assert np.array_equal(out_gpu.view(np.uint32), out_ref.view(np.uint32)) or np.all(err <= 1e-5 * M)
+    return ctx, r
+
+
+@pytest.mark.parametrize("k,d,n", [
+    (3, 8, 1), (3, 200, 3), (4, 1000, 2), (5, 4096 + 32, 2), (8, 5000, 4), (10, 33_000, 3),
+    (13, 20_000, 2), (14, 16_384, 2), (14, 70_001, 3),
+])
+def test_single_pass_blocks(k, d, n):
+    check_round(_mk(n, d, k))
+
+
+@pytest.mark.parametrize("k,d,n", [
+    (15, 32_768, 2), (15, 100_000, 2), (16, 65_536 * 2 + 5, 3), (18, 300_000, 2),
+    (20, (1 << 20) + 777, 2), (22, (1 << 22), 1),
+])
+def test_two_pass_blocks(k, d, n):
+    check_round(_mk(n, d, k))
+
+
+@pytest.mark.parametrize("bits,g,table", [
+    (1, 1, (0, 1)), (1, 30, (0, 30)), (2, 3, (0, 1, 2, 3)), (2, 4, (0, 1, 3, 4)),
+    (4, 15, tuple(range(16))), (4, 30, T4_30), (8, 255, tuple(range(256))),
+    (4, 200, tuple(int(round(v)) for v in np.linspace(0, 200, 16))),
+])
+@pytest.mark.parametrize("k", [10, 16])
+def test_bit_budgets_and_tables(bits, g, table, k):
+    check_round(_mk(3, 70_000, k, bits=bits, g=g, table=table))
+
+
+@pytest.mark.parametrize("n,acc", [(8, 0), (9, 0), (16, 16), (3, 32), (40, 0)])
+def test_accumulator_widths(n, acc):
+    w = _mk(n, 40_000, 12)
+    ctx, r = check_round(w, acc_bits=acc)
+    assert r.sz.acc_bits == (acc if acc else O.acc_bits(n, 30))
+
+
+def test_bf16_gradients():
+    w = _mk(3, 150_000, 16, in_dtype="bf16", name="cfg4_x")
+    check_round(w)
+
+
+def test_other_round_and_seed_change_the_result():
+    w = _mk(2, 50_000, 12)
+    x, _ = _inputs(w)
+    _, r0 = _gpu_round(w, x, rnd=0)
+    _, r1 = _gpu_round(w, x, rnd=1)
+    assert not np.array_equal(r0.packed[0].cpu().numpy(), r1.packed[0].cpu().numpy())
+    check_round(w, rnd=7)
+
+
+def test_config1_full_size():
+    """Benchmark configuration 1 at full size (n=4, d=65536, one block of 2^16)."""
+    check_round(W.config1())
+
+
+def test_degenerate_and_nonfinite_blocks():
+    import torch
+    from paper_2302_08545_b200 import runner, thc
+    w = _mk(2, 4 * 1024, 10)
+    x, _ = _inputs(w)
+    x[:, 1024:2048] = 0.0                 # an all-zero block
+    x[1, 2048 + 5] = np.inf               # a non-finite block
+    x[0, 3072 + 9] = np.nan
+    ctx = runner.context_for(w)
+    r = runner.Round(ctx, w.n, w.d, want_rotated=False)
+    r.upload(x)
+    r.run(0)
+    torch.cuda.synchronize()
+    flags = ctx.status()
+    assert flags & thc.STATUS_NONFINITE and flags & thc.STATUS_ZERO_BLOCK
+    assert ctx.status() == 0              # read-and-clear
+    scl = r.scales.cpu().numpy()
+    assert scl[0] > 0 and scl[1] == 0 and scl[2] == 0 and scl[3] == 0
+    out = r.out.cpu().numpy()
+    assert np.all(out[1024:] == 0.0)
+    packed = np.stack([p.cpu().numpy() for p in r.packed])
+    assert np.all(packed[:, 1024 // 2:] == 0)
+    c = _ocfg(w)
+    ref = O.thc_round(x, c, 0, scl=scl)
+    assert np.array_equal(packed, ref["packed"])
+    assert np.array_equal(out.view(np.uint32), ref["out"].view(np.uint32))
+
+
+def test_workers_can_be_compressed_in_separate_calls():
+    """n_local = 1 calls with worker_base = i give the same bytes as one batched call."""
+    import torch
+    from paper_2302_08545_b200 import runner
+    w = _mk(3, 90_000, 16)
+    x, _ = _inputs(w)
+    ctx, r = _gpu_round(w, x, 0, want_rotated=False)
+    batched = [p.cpu().numpy().copy() for p in r.packed]
+    for p in r.packed:
+        p.zero_()
+    for i in range(w.n):
+        ctx.compress([r.grads[i]], w.d, 0, r.scales, [r.packed[i]], r.workspace, worker_base=i)
+    torch.cuda.synchronize()
+    for i in range(w.n):
+        assert np.array_equal(batched[i], r.packed[i].cpu().numpy())
+
+
+def test_quantize_rotated_entry_matches_oracle_on_oracle_rotation():
+    import torch
+    from paper_2302_08545_b200 import runner
+    w = _mk(2, 40_000, 13)
+    x, xf = _inputs(w)
+    c = _ocfg(w)
+    ctx = runner.context_for(w)
+    r = runner.Round(ctx, w.n, w.d, want_rotated=True)
+    scl = O.scales(xf, c)
+    r.scales.copy_(torch.from_numpy(scl))
+    for i in range(w.n):
+        r.rotated[i].copy_(torch.from_numpy(O.rht_forward(xf[i], c, 3)))
+    ctx.quantize_rotated(r.rotated, w.d, 3, r.scales, r.packed)
+    torch.cuda.synchronize()
+    for i in range(w.n):
+        ref = O.pack(O.quantize(r.rotated[i].cpu().numpy(), scl, c, 3, i), w.bits)
+        assert np.array_equal(r.packed[i].cpu().numpy(), ref)
+
+
+def test_partial_aggregation_uses_the_count_as_divisor():
+    import torch
+    from paper_2302_08545_b200 import runner
+    w = _mk(5, 30_000, 12)
+    x, _ = _inputs(w)
+    ctx, r = _gpu_round(w, x, 0, want_rotated=False)
+    c = _ocfg(w)
+    scl = r.scales.cpu().numpy()
+    subset = [0, 2, 3]
+    ctx.aggregate([r.packed[i] for i in subset], w.d, r.total)
+    ctx.decompress(r.total, len(subset), w.d, 0, r.scales, r.out, r.workspace)
+    torch.cuda.synchronize()
+    packed = np.stack([r.packed[i].cpu().numpy() for i in subset])
+    sum_ref = O.aggregate(packed, r.sz.d_pad, c, r.sz.acc_bits)
+    assert np.array_equal(r.sum_numpy(), sum_ref)
+    out_ref = O.decompress(sum_ref, len(subset), w.d, scl, c, 0)
+    assert np.array_equal(r.out.cpu().numpy().view(np.uint32), out_ref.view(np.uint32))

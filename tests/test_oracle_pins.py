@@ -467,7 +467,7 @@ def test_homomorphic_identity():
 
 def test_whole_round_error_falls_with_workers_and_bits():
     """Independent unbiased rounding: NMSE of the average ~ 1/n (Appendix A.2), and 4 bits
-    beat 2 bits by a wide margin (Appendix D.2: about an order of magnitude per bit)."""
+    beat 2 bits by a wide margin (Appendix D.4: roughly an order of magnitude per extra bit)."""
     k, d = 10, 4096
     rng = np.random.default_rng(9)
     base = rng.standard_normal(d).astype(np.float32)
@@ -504,3 +504,15 @@ def test_bf16_upcast_is_exact():
     f = O.bf16_to_f32(bits)
     assert f[0] == 1.0 and f[1] == -1.0 and f[4] == 0.0 and np.signbit(f[4])
     assert f[2] > 0 and f[3] == np.float32(3.3895314e38)
+
+
+def test_nonfinite_norm_of_any_worker_makes_the_block_degenerate():
+    c = cfg(k=4)
+    x = np.ones((3, 32), dtype=np.float32)
+    x[0, 3] = np.nan          # first worker: must not be overwritten by later finite norms
+    x[2, 20] = np.inf         # last worker
+    M = O.scales(x, c)
+    assert M[0] == 0.0 and M[1] == 0.0
+    x = np.ones((3, 32), dtype=np.float32)
+    x[1, 16:] = 0
+    assert np.all(O.scales(x, c) > 0)
