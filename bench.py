@@ -35,6 +35,10 @@ KERNELS_PER_STEP = {"prepare": 2, "compress": 2, "aggregate": 1, "decompress": 2
 
 
 def pick_workload(name: str) -> W.Workload:
+    """cfg1..cfg4, or 'sweep:<log2 d>:<bits>:<n>' for a point of the cfg5 sweep."""
+    if name.startswith("sweep:"):
+        log2d, bits, n = (int(v) for v in name.split(":")[1:4])
+        return W.sweep_point(1 << log2d, bits, n)
     return {"cfg1": W.config1, "cfg2": W.config2, "cfg3": lambda: W.config3(4),
             "cfg3b2": lambda: W.config3(2), "cfg4": W.config4}[name]()
 
