@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libthc.so")
 SOURCES = ["thc.cu"]
-HEADERS = ["thc_device.cuh", os.path.join("..", "..", "include", "thc.h")]
+HEADERS = ["thc_device.cuh", "thc_pipeline.cuh", os.path.join("..", "..", "include", "thc.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

@@ -499,6 +499,8 @@ aggregate_kernel(PtrArray in, uint32_t n, uint64_t units, uint64_t d_pad, const 
 
 }  // namespace thc
 
+#include "thc_pipeline.cuh"
+
 // =========================================================================== host side
 using namespace thc;
 
@@ -648,6 +650,31 @@ int thc_destroy(thc_ctx *ctx)
 
 static uint64_t round_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 
+// Schedule of the persistent pipeline for `wb_count` worker-blocks of 2^k coordinates:
+// how far pass B trails pass A (lag, in worker-blocks) and how many ring slots that needs.
+struct PipePlan { uint32_t grid, lag, ring; };
+
+static PipePlan plan_pipeline(const thc_ctx *ctx, uint64_t wb_count)
+{
+    const uint32_t k = ctx->cfg.log2_block;
+    const uint64_t T = 1ull << (k - kTileLog2);
+    const uint64_t resident = (uint64_t)ctx->sm_count * 2;
+    PipePlan p;
+    const uint64_t tasks = wb_count * T * 2;
+    p.grid = (uint32_t)(tasks < resident ? tasks : resident);
+    uint64_t lag = (resident + T - 1) / T + 1;
+    uint64_t ring = lag + (resident + 2 * T - 1) / (2 * T) + 1;
+    if (lag > wb_count) lag = wb_count;
+    if (ring > wb_count) ring = wb_count;
+    if (ring > (uint64_t)kMaxRing) {           // tiny blocks on a huge grid: shrink the window
+        ring = kMaxRing;
+        if (lag > ring - 2) lag = ring - 2;
+    }
+    p.lag = (uint32_t)lag;
+    p.ring = (uint32_t)ring;
+    return p;
+}
+
 int thc_sizes(const thc_ctx *ctx, uint64_t d, uint32_t n_local, thc_sizes_t *s)
 {
     if (ctx == nullptr || s == nullptr || d == 0 || n_local == 0 || n_local > THC_MAX_WORKERS)
@@ -664,7 +691,11 @@ int thc_sizes(const thc_ctx *ctx, uint64_t d, uint32_t n_local, thc_sizes_t *s)
     s->acc_bits = ctx->acc_bits;
     const uint32_t chunk_log2 = k < (uint32_t)kTileLog2 ? k : (uint32_t)kTileLog2;
     const uint64_t prepare_ws = (uint64_t)n_local * (s->d_pad >> chunk_log2) * 8;
-    const uint64_t two_pass_ws = k > (uint32_t)kTileLog2 ? (uint64_t)n_local * s->d_pad * 4 : 0;
+    uint64_t two_pass_ws = 0;
+    if (k > (uint32_t)kTileLog2) {
+        const PipePlan pl = plan_pipeline(ctx, s->nblocks * n_local);
+        two_pass_ws = (uint64_t)pl.ring * B * 4;
+    }
     s->workspace_bytes = round_up((prepare_ws > two_pass_ws ? prepare_ws : two_pass_ws) + 256, 256);
     return THC_OK;
 }
@@ -789,6 +820,62 @@ static void geom_pass_b(TileGeom &g)
     g.blocks_in_tile = 1;
 }
 
+// ---- persistent pipeline dispatch (RHT blocks of 2^15 .. 2^24 coordinates)
+typedef void (*pipe_kernel_t)(PipeParams, PtrArrayP, MutPtrArrayP, MutPtrArrayP, PhiloxKeys);
+
+template <int MODE>
+static pipe_kernel_t pick_pipe_kernel(uint32_t bits, bool identity)
+{
+    if constexpr (MODE != kCompressF32 && MODE != kCompressBF16) {
+        return thc_pipeline_kernel<MODE, 4, true>;
+    } else {
+        switch (bits) {
+        case 1: return identity ? thc_pipeline_kernel<MODE, 1, true> : thc_pipeline_kernel<MODE, 1, false>;
+        case 2: return identity ? thc_pipeline_kernel<MODE, 2, true> : thc_pipeline_kernel<MODE, 2, false>;
+        case 4: return identity ? thc_pipeline_kernel<MODE, 4, true> : thc_pipeline_kernel<MODE, 4, false>;
+        default: return identity ? thc_pipeline_kernel<MODE, 8, true> : thc_pipeline_kernel<MODE, 8, false>;
+        }
+    }
+}
+
+static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, const thc_sizes_t &sz, uint64_t d,
+                           uint32_t n_local, uint32_t worker_base, uint32_t round, uint32_t divisor,
+                           const float *scales, void *workspace, const PtrArrayP &in,
+                           const MutPtrArrayP &out, const MutPtrArrayP &rot, cudaStream_t st)
+{
+    const uint32_t k = ctx->cfg.log2_block;
+    PipeParams P;
+    memset(&P, 0, sizeof P);
+    P.d = d;
+    P.d_pad = sz.d_pad;
+    P.wb_count = sz.nblocks * n_local;
+    const uint64_t T = 1ull << (k - kTileLog2);
+    P.total_tasks = P.wb_count * T * 2;
+    if (P.wb_count >= 0x7FFFFFFFull || P.total_tasks >= 0x7FFFFFFFull) return THC_EUNSUPPORTED;
+    const PipePlan pl = plan_pipeline(ctx, P.wb_count);
+    P.ring = static_cast<float *>(workspace);
+    P.scales = scales;
+    P.dev = ctx->dev;
+    P.k = k;
+    P.kb = k - kTileLog2;
+    P.n_local = n_local;
+    P.lag = pl.lag;
+    P.ring_slots = pl.ring;
+    P.granularity = ctx->cfg.granularity;
+    P.divisor = divisor;
+    P.round = round;
+    P.worker_base = worker_base;
+    P.lut_rep = ctx->lut_rep;
+    P.c_block = (float)(1.0 / sqrt((double)(1ull << k)));
+    const size_t smem = (size_t)kTileElems * 4 + kSignWordsMax * 4 +
+                        (size_t)(ctx->cfg.granularity + 1) * ctx->lut_rep * 8;
+    THC_CUDA(cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<pl.grid, kThreads, smem, st>>>(P, in, out, rot, ctx->keys);
+    THC_CUDA(cudaGetLastError());
+    return THC_OK;
+}
+
 int thc_compress(thc_ctx *ctx, const void *const *grads, uint32_t n_local, uint32_t worker_base,
                  uint64_t d, uint32_t round, const float *scales, void *const *packed,
                  float *const *rotated, void *workspace, uint64_t workspace_bytes, void *stream)
@@ -833,15 +920,15 @@ int thc_compress(thc_ctx *ctx, const void *const *grads, uint32_t n_local, uint3
                                   : pick_tile_kernel<kLoadGradF32, kStoreQuant>(ctx->cfg.bits, ctx->identity);
         return launch_tile(ctx, kern, g, tiles, n_local, in, out, rot, scales, st);
     }
-    tile_kernel_t ka = bf16 ? pick_tile_kernel<kLoadGradBF16, kStoreRaw>(ctx->cfg.bits, ctx->identity)
-                            : pick_tile_kernel<kLoadGradF32, kStoreRaw>(ctx->cfg.bits, ctx->identity);
-    if ((rc = launch_tile(ctx, ka, g, tiles, n_local, in, ws, rot, scales, st)) != THC_OK) return rc;
-    geom_pass_b(g);
-    PtrArray wsin;
-    memset(&wsin, 0, sizeof wsin);
-    wsin.p[0] = workspace;
-    tile_kernel_t kb = pick_tile_kernel<kLoadRaw, kStoreQuant>(ctx->cfg.bits, ctx->identity);
-    return launch_tile(ctx, kb, g, tiles, n_local, wsin, out, rot, scales, st);
+    PtrArrayP pin;
+    MutPtrArrayP pout, prot;
+    memcpy(&pin, &in, sizeof pin);
+    memcpy(&pout, &out, sizeof pout);
+    memcpy(&prot, &rot, sizeof prot);
+    pipe_kernel_t kern = bf16 ? pick_pipe_kernel<kCompressBF16>(ctx->cfg.bits, ctx->identity)
+                              : pick_pipe_kernel<kCompressF32>(ctx->cfg.bits, ctx->identity);
+    return launch_pipeline(ctx, kern, sz, d, n_local, worker_base, round, 1, scales, workspace, pin,
+                           pout, prot, st);
 }
 
 int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, uint32_t round,
@@ -882,16 +969,15 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
                      : pick_tile_kernel<kLoadSum32, kStoreOut>(4, true);
         return launch_tile(ctx, k1, g, tiles, 1, in, out, rot, scales, st);
     }
-    k1 = w == 8 ? pick_tile_kernel<kLoadSum8, kStoreRaw>(4, true)
-       : w == 16 ? pick_tile_kernel<kLoadSum16, kStoreRaw>(4, true)
-                 : pick_tile_kernel<kLoadSum32, kStoreRaw>(4, true);
-    if ((rc = launch_tile(ctx, k1, g, tiles, 1, in, ws, rot, scales, st)) != THC_OK) return rc;
-    geom_pass_b(g);
-    PtrArray wsin;
-    memset(&wsin, 0, sizeof wsin);
-    wsin.p[0] = workspace;
-    return launch_tile(ctx, pick_tile_kernel<kLoadRaw, kStoreOut>(4, true), g, tiles, 1, wsin, out,
-                       rot, scales, st);
+    PtrArrayP pin;
+    MutPtrArrayP pout, prot;
+    memcpy(&pin, &in, sizeof pin);
+    memcpy(&pout, &out, sizeof pout);
+    memcpy(&prot, &rot, sizeof prot);
+    pipe_kernel_t kern = w == 8 ? pick_pipe_kernel<kDecompress8>(4, true)
+                       : w == 16 ? pick_pipe_kernel<kDecompress16>(4, true)
+                                 : pick_pipe_kernel<kDecompress32>(4, true);
+    return launch_pipeline(ctx, kern, sz, d, 1, 0, round, divisor, scales, workspace, pin, pout, prot, st);
 }
 
 int thc_quantize_rotated(thc_ctx *ctx, const float *const *rotated, uint32_t n_local,

@@ -24,7 +24,7 @@ constexpr int kLutRepMaxBytes = 16384;
 // Lives in the context's device block.
 struct DeviceBlock {
     uint32_t status;             // THC_STATUS_* bits
-    uint32_t counters[31];       // scheduling counters (self-resetting)
+    uint32_t counters[127];      // scheduling counters (self-resetting)
     uint32_t lut_tz[256];        // by floor(y): float bits of T[z0] | z0
     float    lut_r16[256];       // by floor(y): 65536 / (T[z0+1] - T[z0])
     uint32_t table[256];         // T
