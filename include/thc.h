@@ -67,7 +67,7 @@ typedef struct thc_ctx thc_ctx;   /* opaque */
  *   table        T[0 .. 2^b - 1], 0 = T[0] < T[1] < ... < T[2^b - 1] = g (Section 4.3);
  *                the identity table with g = 2^b - 1 is Uniform THC (Section 4.2)
  *   t_p          truncation threshold Phi^-1(1 - p/2) (Section 5.2), > 0
- *   log2_block   k in [3, 24]: the RHT acts on blocks of B = 2^k coordinates (Section 5.1
+ *   log2_block   k in [3, 22]: the RHT acts on blocks of B = 2^k coordinates (Section 5.1
  *                applied per partition)
  *   seed         shared by all workers: the diagonal D of the RHT must be common
  *   in_dtype     THC_F32 or THC_BF16 (bf16 gradients are widened exactly on load)

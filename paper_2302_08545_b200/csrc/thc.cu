@@ -14,6 +14,7 @@
 #include <math.h>
 #include <new>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 namespace thc {
@@ -62,14 +63,15 @@ __device__ __forceinline__ uint64_t chunk_coord(const TileGeom &g, uint64_t base
 
 // Sign words of every row of the tile, 32 coordinates per word.
 __device__ __forceinline__ void fill_sign_words(uint32_t *sw, const TileGeom &g, uint64_t base,
-                                                const PhiloxKeys &keys, int tid)
+                                                const PhiloxKeys &keys, int tid,
+                                                int nthreads = kThreads)
 {
     const int cols = 1 << g.col_log2;
     const int words_per_row = max(1, cols >> 5);
     const int calls_per_row = max(1, cols >> 7);
     const int rows = 1 << g.row_log2;
     const int words_per_call = min(4, words_per_row);
-    for (int q = tid; q < rows * calls_per_row; q += kThreads) {
+    for (int q = tid; q < rows * calls_per_row; q += nthreads) {
         const int row = q / calls_per_row;
         const int cr = q - row * calls_per_row;
         const uint64_t j0 = base + (uint64_t)row * g.row_stride + (uint64_t)cr * 128;
@@ -560,7 +562,7 @@ static int validate_config(const thc_config *c, uint32_t *acc_bits, bool *identi
     for (uint32_t z = 0; z + 1 < levels; ++z)
         if (c->table[z + 1] <= c->table[z]) return THC_EINVAL;
     if (!(c->t_p > 0.0) || !isfinite(c->t_p)) return THC_EINVAL;
-    if (c->log2_block < 3 || c->log2_block > 24) return THC_EINVAL;
+    if (c->log2_block < 3 || c->log2_block > 22) return THC_EINVAL;
     if (c->in_dtype != THC_F32 && c->in_dtype != THC_BF16) return THC_EINVAL;
     if (c->workers == 0 || c->workers > THC_MAX_WORKERS) return THC_EINVAL;
     const uint64_t max_sum = (uint64_t)c->workers * c->granularity;
@@ -657,19 +659,23 @@ struct PipePlan { uint32_t grid, lag, ring; };
 static PipePlan plan_pipeline(const thc_ctx *ctx, uint64_t wb_count)
 {
     const uint32_t k = ctx->cfg.log2_block;
-    const uint64_t T = 1ull << (k - kTileLog2);
-    const uint64_t resident = (uint64_t)ctx->sm_count * 2;
+    const uint64_t T = 1ull << (k - kPLog2);
+    const uint64_t resident = (uint64_t)ctx->sm_count * 3;
     PipePlan p;
     const uint64_t tasks = wb_count * T * 2;
     p.grid = (uint32_t)(tasks < resident ? tasks : resident);
-    uint64_t lag = (resident + T - 1) / T + 1;
-    uint64_t ring = lag + (resident + 2 * T - 1) / (2 * T) + 1;
+    // tasks in flight: per CTA one running, one handed over, and at times one being claimed
+    const uint64_t inflight = resident * 5 / 2;
+    uint64_t lag = (inflight + 2 * T - 1) / (2 * T) + 1;
+    uint64_t ring = lag + (inflight + 2 * T - 1) / (2 * T) + 1;
     if (lag > wb_count) lag = wb_count;
     if (ring > wb_count) ring = wb_count;
     if (ring > (uint64_t)kMaxRing) {           // tiny blocks on a huge grid: shrink the window
         ring = kMaxRing;
         if (lag > ring - 2) lag = ring - 2;
     }
+    if (const char *e = getenv("THC_EXP_LAG")) { lag = strtoull(e, nullptr, 10); if (lag > wb_count) lag = wb_count; }
+    if (const char *e = getenv("THC_EXP_RING")) { ring = strtoull(e, nullptr, 10); if (ring > wb_count) ring = wb_count; if (ring > (uint64_t)kMaxRing) ring = kMaxRing; }
     p.lag = (uint32_t)lag;
     p.ring = (uint32_t)ring;
     return p;
@@ -810,32 +816,30 @@ static void geom_pass_a(TileGeom &g)
     g.blocks_in_tile = g.k >= (uint32_t)kTileLog2 ? 1u : 1u << (kTileLog2 - g.k);
 }
 
-static void geom_pass_b(TileGeom &g)
-{
-    g.row_log2 = g.k - kTileLog2;
-    g.col_log2 = kTileLog2 - g.row_log2;
-    g.row_stride = 1ull << kTileLog2;
-    g.lo_cbit = g.col_log2 - 2;
-    g.hi_cbit = kTileLog2 - 2;
-    g.blocks_in_tile = 1;
-}
-
 // ---- persistent pipeline dispatch (RHT blocks of 2^15 .. 2^24 coordinates)
 typedef void (*pipe_kernel_t)(PipeParams, PtrArrayP, MutPtrArrayP, MutPtrArrayP, PhiloxKeys);
 
-template <int MODE>
-static pipe_kernel_t pick_pipe_kernel(uint32_t bits, bool identity)
+template <int MODE, int KB>
+static pipe_kernel_t pick_pipe_kernel_kb(uint32_t bits, bool identity)
 {
     if constexpr (MODE != kCompressF32 && MODE != kCompressBF16) {
-        return thc_pipeline_kernel<MODE, 4, true>;
+        return thc_pipeline_kernel<MODE, 4, true, KB>;
     } else {
         switch (bits) {
-        case 1: return identity ? thc_pipeline_kernel<MODE, 1, true> : thc_pipeline_kernel<MODE, 1, false>;
-        case 2: return identity ? thc_pipeline_kernel<MODE, 2, true> : thc_pipeline_kernel<MODE, 2, false>;
-        case 4: return identity ? thc_pipeline_kernel<MODE, 4, true> : thc_pipeline_kernel<MODE, 4, false>;
-        default: return identity ? thc_pipeline_kernel<MODE, 8, true> : thc_pipeline_kernel<MODE, 8, false>;
+        case 1: return identity ? thc_pipeline_kernel<MODE, 1, true, KB> : thc_pipeline_kernel<MODE, 1, false, KB>;
+        case 2: return identity ? thc_pipeline_kernel<MODE, 2, true, KB> : thc_pipeline_kernel<MODE, 2, false, KB>;
+        case 4: return identity ? thc_pipeline_kernel<MODE, 4, true, KB> : thc_pipeline_kernel<MODE, 4, false, KB>;
+        default: return identity ? thc_pipeline_kernel<MODE, 8, true, KB> : thc_pipeline_kernel<MODE, 8, false, KB>;
         }
     }
+}
+
+// The 2^20-coordinate block (the paper's 4 MB partition) gets the compile-time geometry.
+template <int MODE>
+static pipe_kernel_t pick_pipe_kernel(uint32_t bits, bool identity, uint32_t k)
+{
+    return k == 20 ? pick_pipe_kernel_kb<MODE, 7>(bits, identity)
+                   : pick_pipe_kernel_kb<MODE, 0>(bits, identity);
 }
 
 static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, const thc_sizes_t &sz, uint64_t d,
@@ -849,7 +853,7 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, const thc_siz
     P.d = d;
     P.d_pad = sz.d_pad;
     P.wb_count = sz.nblocks * n_local;
-    const uint64_t T = 1ull << (k - kTileLog2);
+    const uint64_t T = 1ull << (k - kPLog2);
     P.total_tasks = P.wb_count * T * 2;
     if (P.wb_count >= 0x7FFFFFFFull || P.total_tasks >= 0x7FFFFFFFull) return THC_EUNSUPPORTED;
     const PipePlan pl = plan_pipeline(ctx, P.wb_count);
@@ -857,7 +861,7 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, const thc_siz
     P.scales = scales;
     P.dev = ctx->dev;
     P.k = k;
-    P.kb = k - kTileLog2;
+    P.kb = k - kPLog2;
     P.n_local = n_local;
     P.lag = pl.lag;
     P.ring_slots = pl.ring;
@@ -865,13 +869,13 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, const thc_siz
     P.divisor = divisor;
     P.round = round;
     P.worker_base = worker_base;
-    P.lut_rep = ctx->lut_rep;
     P.c_block = (float)(1.0 / sqrt((double)(1ull << k)));
-    const size_t smem = (size_t)kTileElems * 4 + kSignWordsMax * 4 +
-                        (size_t)(ctx->cfg.granularity + 1) * ctx->lut_rep * 8;
+    const uint64_t nblk_cached = sz.nblocks < (uint64_t)kBlockConstMax ? sz.nblocks : (uint64_t)kBlockConstMax;
+    const size_t smem = (size_t)2 * kPElems * 4 + kPSignWords * 4 +
+                        (size_t)(ctx->cfg.granularity + 1) * kPLutRep * 8 + (size_t)nblk_cached * 8;
     THC_CUDA(cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<pl.grid, kThreads, smem, st>>>(P, in, out, rot, ctx->keys);
+    kern<<<pl.grid, kPCtaThreads, smem, st>>>(P, in, out, rot, ctx->keys);
     THC_CUDA(cudaGetLastError());
     return THC_OK;
 }
@@ -925,8 +929,8 @@ int thc_compress(thc_ctx *ctx, const void *const *grads, uint32_t n_local, uint3
     memcpy(&pin, &in, sizeof pin);
     memcpy(&pout, &out, sizeof pout);
     memcpy(&prot, &rot, sizeof prot);
-    pipe_kernel_t kern = bf16 ? pick_pipe_kernel<kCompressBF16>(ctx->cfg.bits, ctx->identity)
-                              : pick_pipe_kernel<kCompressF32>(ctx->cfg.bits, ctx->identity);
+    pipe_kernel_t kern = bf16 ? pick_pipe_kernel<kCompressBF16>(ctx->cfg.bits, ctx->identity, k)
+                              : pick_pipe_kernel<kCompressF32>(ctx->cfg.bits, ctx->identity, k);
     return launch_pipeline(ctx, kern, sz, d, n_local, worker_base, round, 1, scales, workspace, pin,
                            pout, prot, st);
 }
@@ -974,9 +978,9 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
     memcpy(&pin, &in, sizeof pin);
     memcpy(&pout, &out, sizeof pout);
     memcpy(&prot, &rot, sizeof prot);
-    pipe_kernel_t kern = w == 8 ? pick_pipe_kernel<kDecompress8>(4, true)
-                       : w == 16 ? pick_pipe_kernel<kDecompress16>(4, true)
-                                 : pick_pipe_kernel<kDecompress32>(4, true);
+    pipe_kernel_t kern = w == 8 ? pick_pipe_kernel<kDecompress8>(4, true, k)
+                       : w == 16 ? pick_pipe_kernel<kDecompress16>(4, true, k)
+                                 : pick_pipe_kernel<kDecompress32>(4, true, k);
     return launch_pipeline(ctx, kern, sz, d, 1, 0, round, divisor, scales, workspace, pin, pout, prot, st);
 }
 

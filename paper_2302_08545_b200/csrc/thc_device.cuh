@@ -65,26 +65,29 @@ __device__ __forceinline__ uint4 round_call(uint64_t j, uint32_t worker, uint32_
                                             const PhiloxKeys &keys)
 {
     const uint64_t call = j >> 3;
+#ifdef THC_EXP_NOPHILOX
+    return make_uint4((uint32_t)call, worker, round, keys.k[0]);
+#endif
     return philox4x32_10((uint32_t)call, (uint32_t)(call >> 32), worker, round, keys);
 }
 
 // ---------------------------------------------------------------- packed fp32 arithmetic
 __device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
 
+// a - b as fma(b, -1, a): one rounding of the exact difference, i.e. the same result as a
+// subtraction, expressed with the packed intrinsic so that the compiler keeps operands in
+// register pairs.
 __device__ __forceinline__ float2 sub2(float2 a, float2 b)
 {
-    uint64_t ra, rb, rc;
-    asm("mov.b64 %0, {%1,%2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
-    asm("mov.b64 %0, {%1,%2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(rc) : "l"(ra), "l"(rb));
-    float2 c;
-    asm("mov.b64 {%0,%1}, %2;" : "=f"(c.x), "=f"(c.y) : "l"(rc));
-    return c;
+    return __ffma2_rn(b, make_float2(-1.0f, -1.0f), a);
 }
 
 // One radix-2 butterfly on four independent columns: (a, b) <- (a + b, a - b).
 __device__ __forceinline__ void butterfly(float4 &a, float4 &b)
 {
+#ifdef THC_EXP_NOBFLY
+    return;
+#endif
     const float2 alo = make_float2(a.x, a.y), ahi = make_float2(a.z, a.w);
     const float2 blo = make_float2(b.x, b.y), bhi = make_float2(b.z, b.w);
     const float2 slo = add2(alo, blo), shi = add2(ahi, bhi);
@@ -113,6 +116,9 @@ __device__ __forceinline__ float4 scale4(float4 v, float c)
 // Flip the signs of a chunk by bits [0,4) of `bits` (bit e set -> element e negated).
 __device__ __forceinline__ float4 flip4(float4 v, uint32_t bits)
 {
+#ifdef THC_EXP_NOFLIP
+    return v;
+#endif
     v.x = __uint_as_float(__float_as_uint(v.x) ^ ((bits << 31) & 0x80000000u));
     v.y = __uint_as_float(__float_as_uint(v.y) ^ ((bits << 30) & 0x80000000u));
     v.z = __uint_as_float(__float_as_uint(v.z) ^ ((bits << 29) & 0x80000000u));
@@ -186,6 +192,9 @@ __device__ __forceinline__ uint64_t quantize8(const float (&r)[8], float kappa, 
 {
     const uint32_t words[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
     uint64_t out = 0;
+#ifdef THC_EXP_NOQUANT
+    return (uint64_t)(__float_as_uint(r[0]) ^ __float_as_uint(r[5]) ^ rnd.x ^ rnd.z) + __float_as_uint(kappa);
+#endif
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
         float y = fmaf(r[e], kappa, half_g);

@@ -1,17 +1,21 @@
 // Persistent dataflow kernel for RHT blocks larger than one shared-memory tile (k >= 15).
 //
-// Work is cut into tasks of one 2^14-coordinate tile each:
+// Work is cut into tasks of one 2^13-coordinate tile each, run by CTAs of 128 threads:
 //   A(wb, t)  pass A of tile t of worker-block wb: consecutive coordinates, stages of
-//             stride 1 .. 2^13, result written to slot (wb mod R) of a ring in the workspace;
-//   B(wb, p)  pass B of panel p: 2^(k-14) rows (2^14 apart) x 2^(28-k) columns read back from
-//             the slot, stages 2^14 .. 2^(k-1), then the fused epilogue.
+//             stride 1 .. 2^12, result written to slot (wb mod R) of a ring in the workspace;
+//   B(wb, p)  pass B of panel p: 2^(k-13) rows (2^13 apart) x 2^(26-k) columns read back from
+//             the slot, stages 2^13 .. 2^(k-1), then the fused epilogue.
 // A worker-block is (RHT block r, local worker i), wb = r * n_local + i.  Tasks are claimed
 // from one queue in the order  A(0) .. A(L-1), [A(s), B(s-L)] for s = L .., B(..) : pass B
 // follows its pass A by L worker-blocks, close enough for the ring (R slots of 2^k floats) to
 // stay in L2, far enough that the tiles it needs are normally finished.  Dependencies only
-// point backwards in the queue, so a CTA that waits never waits for work that has not been
-// claimed by a running CTA.  Every wait is bounded: on expiry the kernel sets
-// THC_STATUS_WAIT_TIMEOUT, raises an abort flag that ends all CTAs, and returns.
+// point backwards in the queue, and a task waits only before it starts, so a CTA that waits
+// never waits for work that is not already claimed by a running CTA.  Every wait is bounded:
+// on expiry the kernel sets THC_STATUS_WAIT_TIMEOUT, raises an abort flag that ends all CTAs,
+// and returns.
+//
+// Each CTA keeps two tile buffers: while it computes task i from one, the tile of task i+1
+// (claimed one task ahead, dependency polled early) streams into the other with cp.async.
 //
 // Counters (in the context's device block, all zero between launches; the last CTA to leave
 // clears them):  head, exited, abort, a_done[R], b_done[R].  a_done[s] counts finished A tiles
@@ -22,7 +26,15 @@
 
 namespace thc {
 
-constexpr int kMaxRing = 40;
+constexpr int kPLog2 = 13;                  // coordinates per pipeline tile
+constexpr int kPElems = 1 << kPLog2;
+constexpr int kPChunks = kPElems / 4;
+constexpr int kPThreads = 128;                // compute threads of a CTA
+constexpr int kPCtaThreads = 160;             // plus one control warp that runs the queue
+constexpr int kPSignWords = 512;            // sign words a tile can need
+constexpr int kPLutRep = 16;                // lane replication of the quantiser table
+constexpr int kMaxRing = 56;
+constexpr int kBlockConstMax = 256;         // per-block constants cached in shared memory
 constexpr uint32_t kMaxPolls = 1u << 21;
 
 enum PipeMode { kCompressF32, kCompressBF16, kDecompress8, kDecompress16, kDecompress32 };
@@ -45,7 +57,7 @@ struct PipeParams {
     const float *scales;
     DeviceBlock *dev;
     uint32_t k;
-    uint32_t kb;               // k - 14: log2 rows of a pass-B tile
+    uint32_t kb;               // k - 13: log2 rows of a pass-B tile
     uint32_t n_local;
     uint32_t lag;              // L
     uint32_t ring_slots;       // R
@@ -53,12 +65,22 @@ struct PipeParams {
     uint32_t divisor;
     uint32_t round;
     uint32_t worker_base;
-    uint32_t lut_rep;
     float    c_block;
 };
 
 struct PtrArrayP { const void *p[THC_MAX_WORKERS]; };
 struct MutPtrArrayP { void *p[THC_MAX_WORKERS]; };
+
+struct TaskInfo {              // published by thread 0 for the whole CTA
+    uint32_t idx;              // tile / panel index; 0xFFFFFFFF = no task
+    uint32_t is_b;
+    uint32_t wl;               // local worker
+    uint32_t r;                // RHT block
+    uint32_t slot;             // ring slot
+    uint32_t gen;              // generation of the slot
+    uint32_t loaded;           // dependency satisfied: its tile load may be / has been issued
+    uint32_t pad;
+};
 
 // ------------------------------------------------------------------------ small helpers
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
@@ -97,23 +119,48 @@ __device__ __forceinline__ uint64_t make_evict_first_policy()
     return pol;
 }
 
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc, uint32_t src_bytes,
-                                           uint64_t policy)
+__device__ __forceinline__ void cp_async16_hint(void *smem_dst, const void *gsrc,
+                                                uint32_t src_bytes, uint64_t policy)
 {
     const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;"
                  :: "r"(dst), "l"(gsrc), "r"(src_bytes), "l"(policy) : "memory");
 }
 
-__device__ __forceinline__ void cp_async_wait_all()
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
 {
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst), "l"(gsrc) : "memory");
 }
 
-__device__ __forceinline__ float4 ld_cg_f4(const float *p)      // L2 only: written by other CTAs
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+
+// Named barriers: 1,2 = task slot full; 3,4 = task slot consumed; 5 = compute warps only.
+__device__ __forceinline__ void bar_sync(int id, int count)
 {
-    return __ldcg(reinterpret_cast<const float4 *>(p));
+    asm volatile("bar.sync %0, %1;" :: "r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(int id, int count)
+{
+    asm volatile("bar.arrive %0, %1;" :: "r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void compute_barrier() { bar_sync(5, kPThreads); }
+
+// Barrier over the compute warps that also ORs a predicate: every thread gets the same answer.
+__device__ __forceinline__ bool compute_barrier_or(bool pred)
+{
+    uint32_t out;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\t"
+                 "barrier.cta.red.or.pred q, 5, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                 : "=r"(out) : "r"((uint32_t)pred), "r"(kPThreads) : "memory");
+    return out != 0;
+}
+
+__device__ __forceinline__ void red_release_add(uint32_t *p, uint32_t v)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
 }
 
 // Lane <-> unit permutation (swap bits 2 and 3): makes pairs of adjacent chunks per lane
@@ -123,16 +170,104 @@ __device__ __forceinline__ int swap_bits_2_3(int t)
     return (t & ~12) | ((t & 4) << 1) | ((t & 8) >> 1);
 }
 
+struct TaskId { uint32_t wb, idx, is_b, slot, gen; };
+
+// Queue position -> task.  Order: A(0..L-1), then [A(s), B(s-L)] per worker-block, then the
+// trailing B's.  T = tiles (= panels) per worker-block = 2^kb.
+__device__ __forceinline__ TaskId decode_task(uint32_t q, const PipeParams &P)
+{
+    TaskId t;
+    const uint32_t T = 1u << P.kb;
+    const uint32_t wbc = (uint32_t)P.wb_count;
+    const uint32_t head_tasks = P.lag << P.kb;
+    const uint32_t mid_tasks = (wbc - P.lag) << (P.kb + 1);
+    if (q < head_tasks) {
+        t.wb = q >> P.kb; t.idx = q & (T - 1); t.is_b = 0;
+    } else if (q - head_tasks < mid_tasks) {
+        const uint32_t q1 = q - head_tasks;
+        const uint32_t s = P.lag + (q1 >> (P.kb + 1));
+        const uint32_t off = q1 & (2 * T - 1);
+        t.is_b = off >= T;
+        t.idx = off & (T - 1);
+        t.wb = t.is_b ? s - P.lag : s;
+    } else {
+        const uint32_t q2 = q - head_tasks - mid_tasks;
+        t.wb = wbc - P.lag + (q2 >> P.kb); t.idx = q2 & (T - 1); t.is_b = 1;
+    }
+    t.gen = t.wb / P.ring_slots;
+    t.slot = t.wb - t.gen * P.ring_slots;
+    return t;
+}
+
+template <bool COMPRESS>
+__device__ __forceinline__ float2 block_constants(float M, uint32_t g, uint32_t divisor)
+{
+    float2 c = make_float2(0.f, 0.f);
+    if (M > 0.0f && isfinite(M)) {
+        if (COMPRESS) {
+            c.x = (float)((double)g / (2.0 * (double)M));
+            c.y = 0.5f * (float)g;
+        } else {
+            c.x = (float)(2.0 * (double)M / ((double)g * (double)divisor));
+            c.y = -M;
+        }
+    }
+    return c;
+}
+
+// ------------------------------------------------------------------ in-place tile rounds
+// Butterfly stages on chunk-index bits [sp, sp+E) of a 2048-chunk tile (see fwht_round).
+template <int E>
+__device__ __forceinline__ void p_round(float4 *tile, int sp, int tid)
+{
+    constexpr int N = 1 << E;
+    constexpr int kGroups = kPChunks >> E;
+#pragma unroll 1
+    for (int G = tid; G < kGroups; G += kPThreads) {
+        const int low = G & ((1 << sp) - 1);
+        const int base = ((G >> sp) << (sp + E)) | low;
+        float4 v[N];
+#pragma unroll
+        for (int m = 0; m < N; ++m) v[m] = tile[swz(base + (m << sp))];
+#pragma unroll
+        for (int t = 0; t < E; ++t) {
+#pragma unroll
+            for (int m = 0; m < N; ++m)
+                if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
+        }
+#pragma unroll
+        for (int m = 0; m < N; ++m) tile[swz(base + (m << sp))] = v[m];
+    }
+}
+
+__device__ __forceinline__ void p_rounds(float4 *tile, int lo, int hi, int tid)
+{
+    int sp = lo;
+    while (sp < hi) {
+        const int e = min(4, hi - sp);
+        switch (e) {
+        case 4: p_round<4>(tile, sp, tid); break;
+        case 3: p_round<3>(tile, sp, tid); break;
+        case 2: p_round<2>(tile, sp, tid); break;
+        default: p_round<1>(tile, sp, tid); break;
+        }
+        sp += e;
+        compute_barrier();
+    }
+}
+
 // ------------------------------------------------------------------------------- pass A
-// First round of a pass-A tile, in place: sign flip (compress), stages of stride 1 and 2
-// inside each chunk, then stride 4 .. 32 across the thread's 16 consecutive chunks.
+// First round, in place: sign flip (compress), stages of stride 1 and 2 inside each chunk,
+// then stride 4 .. 32 across the thread's 16 consecutive chunks.  Chunk 16*tid + m lives at
+// 16*tid + (m ^ (tid & 7)).
 template <bool FLIP>
 __device__ __forceinline__ void pass_a_round1(float4 *tile, const uint32_t *sw, int tid)
 {
-    const int base = tid * 16;
+    float4 *mine = tile + tid * 16;
+    const int x = tid & 7;
     float4 v[16];
 #pragma unroll
-    for (int m = 0; m < 16; ++m) v[m] = tile[swz(base + m)];
+    for (int m = 0; m < 16; ++m) v[m] = mine[m ^ x];
     if (FLIP) {
         const uint2 w = *reinterpret_cast<const uint2 *>(sw + 2 * tid);
 #pragma unroll
@@ -148,15 +283,19 @@ __device__ __forceinline__ void pass_a_round1(float4 *tile, const uint32_t *sw, 
             if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
     }
 #pragma unroll
-    for (int m = 0; m < 16; ++m) tile[swz(base + m)] = v[m];
+    for (int m = 0; m < 16; ++m) mine[m ^ x] = v[m];
 }
 
-// Last round of a pass-A tile (chunk bits 8..11) with the result stored straight to the ring.
-__device__ __forceinline__ void pass_a_round3_store(const float4 *tile, float *dst, int tid)
+// Round on chunk bits 4..7 (also the first pass-B round when a row has 16 chunks): thread
+// tid owns chunks hi*256 + 16*m + low (low = tid & 15, hi = tid >> 4), stored with the low
+// three bits XORed by m & 7.
+__device__ __forceinline__ void round_bits_4_7(float4 *tile, int tid)
 {
+    float4 *mine = tile + ((tid >> 4) << 8);
+    const int low = tid & 15;
     float4 v[16];
 #pragma unroll
-    for (int m = 0; m < 16; ++m) v[m] = tile[swz(tid + (m << 8))];
+    for (int m = 0; m < 16; ++m) v[m] = mine[16 * m + (low ^ (m & 7))];
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
 #pragma unroll
@@ -164,43 +303,36 @@ __device__ __forceinline__ void pass_a_round3_store(const float4 *tile, float *d
             if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
     }
 #pragma unroll
-    for (int m = 0; m < 16; ++m)
-        *reinterpret_cast<float4 *>(dst + 4 * (tid + (m << 8))) = v[m];
+    for (int m = 0; m < 16; ++m) mine[16 * m + (low ^ (m & 7))] = v[m];
 }
 
-// ------------------------------------------------------------------------------- pass B
-// First round of a pass-B tile: E row bits (the lowest), operands loaded straight from the
-// ring (L2), result stored to the tile.
-template <int E>
-__device__ __forceinline__ void pass_b_round1(float4 *tile, const float *src, int ccl, int tid)
+// Last round of a pass-A tile (chunk bits 8..10) with the result stored straight to the ring.
+__device__ __forceinline__ void pass_a_round3_store(const float4 *tile, float *dst, int tid)
 {
-    constexpr int N = 1 << E;
-    const int cmask = (1 << ccl) - 1;                  // chunks per row - 1
-#pragma unroll 1
-    for (int i = 0; i < 16 / N; ++i) {
-        const int G = tid + i * kThreads;
-        const int cc = G & cmask;
-        const int rbase = (G >> ccl) << E;
-        float4 v[N];
 #pragma unroll
-        for (int m = 0; m < N; ++m)
-            v[m] = ld_cg_f4(src + ((size_t)(rbase + m) << kTileLog2) + 4 * cc);
+    for (int i = 0; i < 2; ++i) {
+        const int low = tid + i * kPThreads;
+        const float4 *mine = tile + (low ^ ((low >> 4) & 7));
+        float4 v[8];
 #pragma unroll
-        for (int t = 0; t < E; ++t) {
+        for (int m = 0; m < 8; ++m) v[m] = mine[m << 8];
 #pragma unroll
-            for (int m = 0; m < N; ++m)
+        for (int t = 0; t < 3; ++t) {
+#pragma unroll
+            for (int m = 0; m < 8; ++m)
                 if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
         }
+        float4 *out = reinterpret_cast<float4 *>(dst) + low;
 #pragma unroll
-        for (int m = 0; m < N; ++m) tile[swz(((rbase + m) << ccl) + cc)] = v[m];
+        for (int m = 0; m < 8; ++m) out[m << 8] = v[m];
     }
 }
 
+// ------------------------------------------------------------------------------- pass B
 struct EpilogueCtx {
     uint64_t j_tile;        // coordinate of (row 0, column 0) of the tile in the worker's vector
     float kappa, half_g, gf, c_block;
     const uint2 *lut;
-    int lut_stride;
     uint32_t worker, round;
     unsigned char *packed;
     float *rotated;
@@ -210,8 +342,46 @@ struct EpilogueCtx {
     int words_per_row;
 };
 
-// Last round of a pass-B tile: the top E row bits, each thread owning 2^E rows of one
-// 8-coordinate unit, followed by the epilogue on the registers.
+template <bool COMPRESS, int BITS, bool IDENTITY>
+__device__ __forceinline__ void epilogue_unit(const float4 &va, const float4 &vb, uint64_t j, int row,
+                                              int uu, const EpilogueCtx &ep, const PhiloxKeys &keys)
+{
+    const float4 ra = scale4(va, ep.c_block);
+    const float4 rb = scale4(vb, ep.c_block);
+    if (COMPRESS) {
+        if (ep.rotated != nullptr) {
+            *reinterpret_cast<float4 *>(ep.rotated + j) = ra;
+            *reinterpret_cast<float4 *>(ep.rotated + j + 4) = rb;
+        }
+        const float r[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+        const uint4 rnd = round_call(j, ep.worker, ep.round, keys);
+        const uint64_t z = quantize8<BITS, IDENTITY>(r, ep.kappa, ep.half_g, ep.gf, rnd, ep.lut, kPLutRep);
+        if constexpr (BITS == 8)
+            *reinterpret_cast<uint2 *>(ep.packed + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
+        else if constexpr (BITS == 4)
+            *reinterpret_cast<uint32_t *>(ep.packed + j / 2) = (uint32_t)z;
+        else if constexpr (BITS == 2)
+            *reinterpret_cast<uint16_t *>(ep.packed + j / 4) = (uint16_t)z;
+        else
+            ep.packed[j / 8] = (unsigned char)z;
+    } else {
+        if (j >= ep.d) return;
+        const uint32_t bits = ep.sw[row * ep.words_per_row + (uu >> 2)] >> (uint32_t)(j & 31);
+        const float4 oa = flip4(ra, bits);
+        const float4 ob = flip4(rb, bits >> 4);
+        if (j + 8 <= ep.d) {
+            *reinterpret_cast<float4 *>(ep.out + j) = oa;
+            *reinterpret_cast<float4 *>(ep.out + j + 4) = ob;
+        } else {
+            const float o[8] = {oa.x, oa.y, oa.z, oa.w, ob.x, ob.y, ob.z, ob.w};
+            for (int e = 0; e < 8; ++e)
+                if (j + e < ep.d) ep.out[j + e] = o[e];
+        }
+    }
+}
+
+// Last round of a pass-B tile, any geometry: the top E row bits, each thread owning 2^E rows
+// of one 8-coordinate unit, followed by the epilogue on the registers.
 template <int E, bool COMPRESS, int BITS, bool IDENTITY>
 __device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, int ccl, int tid,
                                                   const EpilogueCtx &ep, const PhiloxKeys &keys)
@@ -221,7 +391,7 @@ __device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, in
     const int rl = kb - E;                             // log2 of the row stride of this round
 #pragma unroll 1
     for (int i = 0; i < 8 / N; ++i) {
-        const int gg = swap_bits_2_3(tid) + i * kThreads;
+        const int gg = swap_bits_2_3(tid) + i * kPThreads;
         const int uu = gg & ((1 << ul) - 1);
         const int row_low = gg >> ul;
         float4 a[N], b[N];
@@ -243,153 +413,122 @@ __device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, in
 #pragma unroll
         for (int m = 0; m < N; ++m) {
             const int row = row_low + (m << rl);
-            const uint64_t j = ep.j_tile + ((uint64_t)row << kTileLog2) + 8 * uu;
-            const float4 ra = scale4(a[m], ep.c_block);
-            const float4 rb = scale4(b[m], ep.c_block);
-            if (COMPRESS) {
-                if (ep.rotated != nullptr) {
-                    *reinterpret_cast<float4 *>(ep.rotated + j) = ra;
-                    *reinterpret_cast<float4 *>(ep.rotated + j + 4) = rb;
-                }
-                const float r[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
-                const uint4 rnd = round_call(j, ep.worker, ep.round, keys);
-                const uint64_t z = quantize8<BITS, IDENTITY>(r, ep.kappa, ep.half_g, ep.gf, rnd,
-                                                             ep.lut, ep.lut_stride);
-                if constexpr (BITS == 8)
-                    *reinterpret_cast<uint2 *>(ep.packed + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
-                else if constexpr (BITS == 4)
-                    *reinterpret_cast<uint32_t *>(ep.packed + j / 2) = (uint32_t)z;
-                else if constexpr (BITS == 2)
-                    *reinterpret_cast<uint16_t *>(ep.packed + j / 4) = (uint16_t)z;
-                else
-                    ep.packed[j / 8] = (unsigned char)z;
-            } else {
-                if (j >= ep.d) continue;
-                const uint32_t bits = ep.sw[row * ep.words_per_row + (uu >> 2)] >> (uint32_t)(j & 31);
-                const float4 oa = flip4(ra, bits);
-                const float4 ob = flip4(rb, bits >> 4);
-                if (j + 8 <= ep.d) {
-                    *reinterpret_cast<float4 *>(ep.out + j) = oa;
-                    *reinterpret_cast<float4 *>(ep.out + j + 4) = ob;
-                } else {
-                    const float o[8] = {oa.x, oa.y, oa.z, oa.w, ob.x, ob.y, ob.z, ob.w};
-                    for (int e = 0; e < 8; ++e)
-                        if (j + e < ep.d) ep.out[j + e] = o[e];
-                }
-            }
+            const uint64_t j = ep.j_tile + ((uint64_t)row << kPLog2) + 8 * uu;
+            epilogue_unit<COMPRESS, BITS, IDENTITY>(a[m], b[m], j, row, uu, ep, keys);
         }
     }
 }
 
+// The same for the 128-row x 16-chunk tile (k = 20): rows row_low + 16 m, m = 0..7; lanes
+// 0-7 of a quarter warp cover four units of two adjacent rows, which is conflict-free.
+template <bool COMPRESS, int BITS, bool IDENTITY>
+__device__ __forceinline__ void pass_b_last_round_kb7(const float4 *tile, int tid,
+                                                      const EpilogueCtx &ep, const PhiloxKeys &keys)
+{
+    const int uu = (tid & 3) | ((tid >> 1) & 4);
+    const int row_low = ((tid >> 2) & 1) | ((tid >> 4) << 1);
+    const int x = row_low & 7;
+    const float4 *pa = tile + row_low * 16 + ((2 * uu) ^ x);
+    const float4 *pb = tile + row_low * 16 + ((2 * uu + 1) ^ x);
+    float4 a[8], b[8];
+#pragma unroll
+    for (int m = 0; m < 8; ++m) { a[m] = pa[m << 8]; b[m] = pb[m << 8]; }
+#pragma unroll
+    for (int t = 0; t < 3; ++t) {
+#pragma unroll
+        for (int m = 0; m < 8; ++m)
+            if (!(m & (1 << t))) {
+                butterfly(a[m], a[m | (1 << t)]);
+                butterfly(b[m], b[m | (1 << t)]);
+            }
+    }
+    const uint64_t j0 = ep.j_tile + ((uint64_t)row_low << kPLog2) + 8 * uu;
+#pragma unroll
+    for (int m = 0; m < 8; ++m)
+        epilogue_unit<COMPRESS, BITS, IDENTITY>(a[m], b[m], j0 + ((uint64_t)m << (kPLog2 + 4)),
+                                                row_low + 16 * m, uu, ep, keys);
+}
+
 // ------------------------------------------------------------------------------ the kernel
-template <int MODE, int BITS, bool IDENTITY>
-__global__ void __launch_bounds__(kThreads, 2)
+// KB = 7 specialises the k = 20 geometry at compile time; KB = 0 reads it from the params.
+template <int MODE, int BITS, bool IDENTITY, int KB>
+__global__ void __launch_bounds__(kPCtaThreads, 3)
 thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP rotated,
                     PhiloxKeys keys)
 {
     constexpr bool kCompress = MODE == kCompressF32 || MODE == kCompressBF16;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    float4 *tile = reinterpret_cast<float4 *>(smem_raw);
-    uint32_t *sw = reinterpret_cast<uint32_t *>(smem_raw + kTileElems * 4);
-    uint2 *lut = reinterpret_cast<uint2 *>(smem_raw + kTileElems * 4 + kSignWordsMax * 4);
-    __shared__ uint32_t s_task[2];
-    __shared__ float s_const[2];
+    constexpr bool kAsyncA = MODE == kCompressF32;
+    extern __shared__ __align__(1024) unsigned char pipe_smem[];
+    float4 *bufs[2] = {reinterpret_cast<float4 *>(pipe_smem),
+                       reinterpret_cast<float4 *>(pipe_smem + kPElems * 4)};
+    uint32_t *sw = reinterpret_cast<uint32_t *>(pipe_smem + 2 * kPElems * 4);
+    uint2 *lut = reinterpret_cast<uint2 *>(pipe_smem + 2 * kPElems * 4 + kPSignWords * 4);
+    float2 *blk_const = reinterpret_cast<float2 *>(pipe_smem + 2 * kPElems * 4 + kPSignWords * 4 +
+                                                   (size_t)(P.granularity + 1) * kPLutRep * 8);
+    __shared__ TaskInfo s_info[2];
+    __shared__ uint32_t s_published;       // tasks the control warp has handed over so far
 
     const int tid = threadIdx.x;
+    if (tid == 0) s_published = 0;
     PipeCounters *pc = reinterpret_cast<PipeCounters *>(P.dev->counters);
-    const uint32_t T = 1u << P.kb;                    // tiles (= panels) per worker-block
+    const int kb = KB ? KB : (int)P.kb;
+    const uint32_t T = 1u << kb;                      // tiles (= panels) per worker-block
     const uint64_t B = 1ull << P.k;
-    const int ccl = 12 - (int)P.kb;                   // log2 chunks per pass-B row
+    const int ccl = 11 - kb;                          // log2 chunks per pass-B row
     const uint64_t policy = make_evict_first_policy();
 
     if (kCompress && !IDENTITY) {
-        const int rep = (int)P.lut_rep;
-        for (int idx = tid; idx < (int)(P.granularity + 1) * rep; idx += kThreads) {
-            const int f = idx / rep;
+        for (int idx = tid; idx < (int)(P.granularity + 1) * kPLutRep; idx += kPThreads) {
+            const int f = idx / kPLutRep;
             lut[idx] = make_uint2(P.dev->lut_tz[f], __float_as_uint(P.dev->lut_r16[f]));
         }
     }
+    const uint32_t nblk_total = (uint32_t)(P.d_pad >> P.k);
+    const uint32_t nblk_cached = nblk_total < (uint32_t)kBlockConstMax ? nblk_total : (uint32_t)kBlockConstMax;
+    for (uint32_t b = tid; b < nblk_cached; b += kPThreads)
+        blk_const[b] = block_constants<kCompress>(P.scales[b], P.granularity, P.divisor);
+    __syncthreads();
 
-    for (;;) {
-        // ---- claim a task; thread 0 also resolves its dependency and per-block constants
-        __syncthreads();                              // previous task done with smem
-        if (tid == 0) {
-            uint32_t q = 0xFFFFFFFFu, ok = 1;
-            if (ld_relaxed_u32(&pc->abort) == 0) q = atomicAdd(&pc->head, 1u);
-            if ((uint64_t)q >= P.total_tasks) {
-                ok = 0;
-            } else {
-                // decode
-                const uint64_t head_tasks = (uint64_t)P.lag * T;
-                const uint64_t mid_tasks = (P.wb_count - P.lag) * 2ull * T;
-                uint64_t wb;
-                uint32_t idx, is_b;
-                if (q < head_tasks) {
-                    wb = q >> P.kb; idx = q & (T - 1); is_b = 0;
-                } else if (q - head_tasks < mid_tasks) {
-                    const uint64_t q1 = q - head_tasks;
-                    const uint64_t s = P.lag + (q1 >> (P.kb + 1));
-                    const uint32_t off = (uint32_t)(q1 & (2 * T - 1));
-                    is_b = off >= T;
-                    idx = off & (T - 1);
-                    wb = is_b ? s - P.lag : s;
-                } else {
-                    const uint64_t q2 = q - head_tasks - mid_tasks;
-                    wb = P.wb_count - P.lag + (q2 >> P.kb); idx = (uint32_t)(q2 & (T - 1)); is_b = 1;
-                }
-                const uint32_t slot = (uint32_t)(wb % P.ring_slots);
-                const uint32_t gen = (uint32_t)(wb / P.ring_slots);
-                if (is_b) ok = wait_at_least(&pc->a_done[slot], (gen + 1) * T, pc, P.dev);
-                else if (gen > 0) ok = wait_at_least(&pc->b_done[slot], gen * T, pc, P.dev);
-                // constants of the RHT block this task belongs to
-                const uint64_t r = wb / P.n_local;
-                const float M = P.scales[r];
-                float c0 = 0.f, c1 = 0.f;
-                if (M > 0.0f && isfinite(M)) {
-                    if (kCompress) {
-                        c0 = (float)((double)P.granularity / (2.0 * (double)M));
-                        c1 = 0.5f * (float)P.granularity;
-                    } else {
-                        c0 = (float)(2.0 * (double)M / ((double)P.granularity * (double)P.divisor));
-                        c1 = -M;
-                    }
-                }
-                s_const[0] = c0;
-                s_const[1] = c1;
-                s_task[1] = (uint32_t)(wb & 0x7FFFFFFFu) | (is_b << 31);
-                q = idx;
-            }
-            s_task[0] = ok ? q : 0xFFFFFFFFu;
-        }
-        __syncthreads();
-        const uint32_t idx = s_task[0];
-        if (idx == 0xFFFFFFFFu) break;
-        const uint32_t wbw = s_task[1];
-        const bool is_b = (wbw >> 31) != 0;
-        const uint64_t wb = wbw & 0x7FFFFFFFu;
-        const uint32_t wl = (uint32_t)(wb % P.n_local);
-        const uint64_t r = wb / P.n_local;
-        const uint32_t slot = (uint32_t)(wb % P.ring_slots);
-        float *slot_base = P.ring + (size_t)slot * B;
-        const float c0 = s_const[0], c1 = s_const[1];
-
-        if (!is_b) {
-            // ================================ pass A: tile idx of worker-block wb
-            const uint64_t j0 = r * B + ((uint64_t)idx << kTileLog2);
-            if (MODE == kCompressF32) {
-                const float *x = static_cast<const float *>(in.p[wl]);
+    // ---- issue the tile load of a task into a buffer (all threads)
+    auto issue_load = [&](const TaskInfo &ti, float4 *tile) {
+        const bool is_b = ti.is_b != 0;
+        const uint32_t wl = ti.wl;
+        const uint64_t r = ti.r;
+        const uint32_t slot = ti.slot;
+        if (is_b) {
+            // panel idx: rows 2^13 apart in the ring slot, 2^(13-kb) columns each
+            const float *src = P.ring + (size_t)slot * B + ((size_t)ti.idx << (kPLog2 - kb));
 #pragma unroll 4
-                for (int i = 0; i < kTileChunks / kThreads; ++i) {
-                    const int c = tid + i * kThreads;
-                    const uint64_t j = j0 + 4ull * c;
-                    const uint32_t nbytes = j + 4 <= P.d ? 16u : j < P.d ? (uint32_t)(P.d - j) * 4u : 0u;
-                    cp_async16(&tile[swz(c)], nbytes ? (const void *)(x + j) : (const void *)x, nbytes, policy);
+            for (int i = 0; i < kPChunks / kPThreads; ++i) {
+                const int c = tid + i * kPThreads;
+                const int row = c >> ccl, cc = c & ((1 << ccl) - 1);
+                cp_async16(&tile[swz(c)], src + ((size_t)row << kPLog2) + 4 * cc);
+            }
+        } else {
+            const uint64_t j0 = r * B + ((uint64_t)ti.idx << kPLog2);
+            if (kAsyncA) {
+                const float *x = static_cast<const float *>(in.p[wl]);
+                if (j0 + kPElems <= P.d) {
+                    const float *xs = x + j0 + 4 * tid;
+                    float4 *dst = tile + (tid ^ ((tid >> 4) & 7));
+#pragma unroll
+                    for (int i = 0; i < kPChunks / kPThreads; ++i)
+                        cp_async16_hint(dst + i * kPThreads, xs + 4 * i * kPThreads, 16u, policy);
+                } else {
+#pragma unroll 4
+                    for (int i = 0; i < kPChunks / kPThreads; ++i) {
+                        const int c = tid + i * kPThreads;
+                        const uint64_t j = j0 + 4ull * c;
+                        const uint32_t nbytes = j + 4 <= P.d ? 16u : j < P.d ? (uint32_t)(P.d - j) * 4u : 0u;
+                        cp_async16_hint(&tile[swz(c)], nbytes ? (const void *)(x + j) : (const void *)x,
+                                        nbytes, policy);
+                    }
                 }
             } else if (MODE == kCompressBF16) {
                 const uint16_t *x = static_cast<const uint16_t *>(in.p[wl]);
 #pragma unroll 2
-                for (int i = 0; i < kTileChunks / 2 / kThreads; ++i) {
-                    const int u = tid + i * kThreads;
+                for (int i = 0; i < kPChunks / 2 / kPThreads; ++i) {
+                    const int u = tid + i * kPThreads;
                     const uint64_t j = j0 + 8ull * u;
                     uint32_t w[4] = {0, 0, 0, 0};
                     if (j + 8 <= P.d) {
@@ -407,9 +546,11 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
             } else {
                 constexpr int kPer = MODE == kDecompress8 ? 16 : MODE == kDecompress16 ? 8 : 4;
                 const unsigned char *y = static_cast<const unsigned char *>(in.p[0]);
+                const float2 bc = r < nblk_cached ? blk_const[r]
+                                                  : block_constants<false>(P.scales[r], P.granularity, P.divisor);
 #pragma unroll 2
-                for (int i = 0; i < kTileElems / kPer / kThreads; ++i) {
-                    const int u = tid + i * kThreads;
+                for (int i = 0; i < kPElems / kPer / kPThreads; ++i) {
+                    const int u = tid + i * kPThreads;
                     const uint64_t j = j0 + (uint64_t)u * kPer;
                     const uint4 q = __ldg(reinterpret_cast<const uint4 *>(y + j * (16 / kPer)));
                     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
@@ -425,75 +566,164 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
                             else val = w[ix];
                             const float yf = MODE == kDecompress32 ? (float)val
                                              : __uint_as_float(0x4B000000u | val) - 8388608.0f;
-                            s[e] = fmaf(yf, c0, c1);
+                            s[e] = fmaf(yf, bc.x, bc.y);
                         }
                         tile[swz(u * (kPer / 4) + cc)] = make_float4(s[0], s[1], s[2], s[3]);
                     }
                 }
             }
-            if (kCompress) {
-                if (tid < 128) {                       // sign words of the tile: 128 calls
-                    const uint4 ph = sign_call(j0 + 128ull * tid, P.round, keys);
-                    *reinterpret_cast<uint4 *>(sw + 4 * tid) = ph;
+        }
+    };
+
+    // ================================================================ control warp
+    // Lane 0 claims tasks, waits (bounded) for their dependency and hands them to the compute
+    // warps through s_info[0/1]; it runs at most two tasks ahead of them.
+    if (tid >= kPThreads) {
+        const int lane = tid - kPThreads;
+        for (uint32_t i = 0;; ++i) {
+            const int s = (int)(i & 1);
+            TaskInfo ti;
+            ti.idx = 0xFFFFFFFFu; ti.is_b = 0; ti.wl = 0; ti.r = 0; ti.slot = 0; ti.gen = 0; ti.loaded = 0; ti.pad = 0;
+            // claim task i only once the compute warps have picked up task i-1: a deeper
+            // look-ahead would stretch every task's claim-to-completion time, which is what
+            // dependent tasks wait for
+            if (i >= 1) bar_sync(3 + (s ^ 1), kPCtaThreads);
+            if (lane == 0) {
+                const uint32_t q = atomicAdd(&pc->head, 1u);
+                if ((uint64_t)q < P.total_tasks) {
+                    const TaskId t = decode_task(q, P);
+                    const uint32_t *ctr = t.is_b ? &pc->a_done[t.slot] : &pc->b_done[t.slot];
+                    const uint32_t target = t.is_b ? (t.gen + 1) * T : t.gen * T;
+                    if (target == 0 || wait_at_least(ctr, target, pc, P.dev)) {
+                        ti.idx = t.idx;
+                        ti.is_b = t.is_b;
+                        ti.r = t.wb / P.n_local;
+                        ti.wl = t.wb - ti.r * P.n_local;
+                        ti.slot = t.slot;
+                        ti.gen = t.gen;
+                        ti.loaded = 1;
+                    }
                 }
             }
-            if (MODE == kCompressF32) cp_async_wait_all();
-            __syncthreads();
-            pass_a_round1<kCompress>(tile, sw, tid);
-            __syncthreads();
-            fwht_round<4>(tile, 4, tid);
-            __syncthreads();
-            pass_a_round3_store(tile, slot_base + ((size_t)idx << kTileLog2), tid);
-            __syncthreads();
-            if (tid == 0) {
-                __threadfence();
-                atomicAdd(&pc->a_done[slot], 1u);
+            __syncwarp();
+            if (lane == 0) {
+                s_info[s] = ti;
+                __threadfence_block();
+                *reinterpret_cast<volatile uint32_t *>(&s_published) = i + 1;
             }
+            __syncwarp();
+            bar_arrive(1 + s, kPCtaThreads);                  // slot s is full
+            if (__shfl_sync(0xFFFFFFFFu, ti.idx, 0) == 0xFFFFFFFFu) break;
+        }
+    } else {
+    // ================================================================ compute warps
+    bar_sync(1, kPCtaThreads);
+    TaskInfo me = s_info[0];
+    bar_arrive(3, kPCtaThreads);
+    bool me_loaded = false;
+
+    for (uint32_t it = 0; me.idx != 0xFFFFFFFFu; ++it) {
+        const int cur = (int)(it & 1);
+        const int s1 = cur ^ 1;
+        if (!me_loaded) issue_load(me, bufs[cur]);
+        cp_async_commit();
+        // Is the next task already handed over?  Then its tile streams in while this one is
+        // computed.  A task is never waited for before the current one is finished and
+        // signalled: it may depend on it.
+        const bool have_next = compute_barrier_or(
+            *reinterpret_cast<volatile uint32_t *>(&s_published) >= it + 2);
+        TaskInfo nxt = me;
+        if (have_next) {
+            bar_sync(1 + s1, kPCtaThreads);
+            nxt = s_info[s1];
+            bar_arrive(3 + s1, kPCtaThreads);
+            if (nxt.idx != 0xFFFFFFFFu) issue_load(nxt, bufs[s1]);
+        }
+        cp_async_commit();
+        cp_async_wait_but_one();
+
+        const bool is_b = me.is_b != 0;
+        const uint32_t wl = me.wl;
+        const uint64_t r = me.r;
+        const uint32_t slot = me.slot;
+        const uint32_t idx = me.idx;
+        float4 *tile = bufs[cur];
+        const float2 bc = r < nblk_cached ? blk_const[r]
+                                          : block_constants<kCompress>(P.scales[r], P.granularity, P.divisor);
+
+        if (!is_b) {
+            // ================================ pass A: tile idx of worker-block wb
+            const uint64_t j0 = r * B + ((uint64_t)idx << kPLog2);
+            if (kCompress && tid < 64) {               // sign words of the tile: 64 calls
+                const uint4 ph = sign_call(j0 + 128ull * tid, P.round, keys);
+                *reinterpret_cast<uint4 *>(sw + 4 * tid) = ph;
+            }
+            compute_barrier();                        // tile and sign words visible
+            pass_a_round1<kCompress>(tile, sw, tid);
+            compute_barrier();
+            round_bits_4_7(tile, tid);
+            compute_barrier();
+            pass_a_round3_store(tile, P.ring + (size_t)slot * B + ((size_t)idx << kPLog2), tid);
         } else {
             // ================================ pass B: panel idx of worker-block wb
-            const int kb = (int)P.kb;
-            const uint64_t j_tile = r * B + ((uint64_t)idx << (kTileLog2 - kb));
-            const float *src = slot_base + ((size_t)idx << (kTileLog2 - kb));
+            const uint64_t j_tile = r * B + ((uint64_t)idx << (kPLog2 - kb));
             EpilogueCtx ep;
             ep.j_tile = j_tile;
-            ep.kappa = c0; ep.half_g = c1; ep.gf = (float)P.granularity; ep.c_block = P.c_block;
-            ep.lut = lut + (P.lut_rep > 1 ? (tid & 31) : 0);
-            ep.lut_stride = (int)P.lut_rep;
+            ep.kappa = bc.x; ep.half_g = bc.y; ep.gf = (float)P.granularity; ep.c_block = P.c_block;
+            ep.lut = lut + (tid & (kPLutRep - 1));
             ep.worker = P.worker_base + wl; ep.round = P.round;
             ep.packed = kCompress ? static_cast<unsigned char *>(outp.p[wl]) : nullptr;
             ep.rotated = kCompress ? static_cast<float *>(rotated.p[wl]) : nullptr;
             ep.out = kCompress ? nullptr : static_cast<float *>(outp.p[0]);
             ep.d = P.d;
             ep.sw = sw;
-            ep.words_per_row = max(1, (1 << (kTileLog2 - kb)) >> 5);
+            ep.words_per_row = max(1, (1 << (kPLog2 - kb)) >> 5);
             if (!kCompress) {
-                // sign words of the panel's rows
                 TileGeom g;
-                g.row_log2 = (uint32_t)kb; g.col_log2 = (uint32_t)(kTileLog2 - kb);
-                g.row_stride = 1ull << kTileLog2; g.round = P.round;
-                fill_sign_words(sw, g, j_tile, keys, tid);
+                g.row_log2 = (uint32_t)kb; g.col_log2 = (uint32_t)(kPLog2 - kb);
+                g.row_stride = 1ull << kPLog2; g.round = P.round;
+                fill_sign_words(sw, g, j_tile, keys, tid, kPThreads);
             }
+            compute_barrier();                        // tile (and sign words) visible
             const int e1 = kb < 4 ? kb : 4;
-            switch (e1) {
-            case 4: pass_b_round1<4>(tile, src, ccl, tid); break;
-            case 3: pass_b_round1<3>(tile, src, ccl, tid); break;
-            case 2: pass_b_round1<2>(tile, src, ccl, tid); break;
-            default: pass_b_round1<1>(tile, src, ccl, tid); break;
+            if (KB == 7) {
+                round_bits_4_7(tile, tid);
+            } else {
+                switch (e1) {
+                case 4: p_round<4>(tile, ccl, tid); break;
+                case 3: p_round<3>(tile, ccl, tid); break;
+                default: p_round<2>(tile, ccl, tid); break;
+                }
             }
-            __syncthreads();
-            const int rem = kb - e1;
-            const int e_last = rem < 3 ? rem : 3;
-            if (rem > e_last) fwht_rounds(tile, ccl + e1, ccl + kb - e_last, tid);
-            switch (e_last) {
-            case 3: pass_b_last_round<3, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
-            case 2: pass_b_last_round<2, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
-            case 1: pass_b_last_round<1, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
-            default: pass_b_last_round<0, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
+            compute_barrier();
+            if (KB == 7) {
+                pass_b_last_round_kb7<kCompress, BITS, IDENTITY>(tile, tid, ep, keys);
+            } else {
+                const int rem = kb - e1;
+                const int e_last = rem < 3 ? rem : 3;
+                if (rem > e_last) p_rounds(tile, ccl + e1, ccl + kb - e_last, tid);
+                switch (e_last) {
+                case 3: pass_b_last_round<3, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
+                case 2: pass_b_last_round<2, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
+                case 1: pass_b_last_round<1, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
+                default: pass_b_last_round<0, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
+                }
             }
-            __syncthreads();
-            if (tid == 0) atomicAdd(&pc->b_done[slot], 1u);
         }
+        // every compute warp has issued its stores and is done with the tile and sign words
+        compute_barrier();
+        if (tid == 0) red_release_add(is_b ? &pc->b_done[slot] : &pc->a_done[slot], 1u);
+        if (!have_next) {
+            bar_sync(1 + s1, kPCtaThreads);
+            nxt = s_info[s1];
+            bar_arrive(3 + s1, kPCtaThreads);
+        }
+        me_loaded = have_next;
+        me = nxt;
     }
+    cp_async_wait_all();
+    }
+    __syncthreads();
 
     // ---- leave: the last CTA clears the counters for the next launch
     if (tid == 0) {
