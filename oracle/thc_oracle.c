@@ -32,13 +32,15 @@
  *       counter = (j/128 lo, j/128 hi, 0xFFFFFFFF, round)).
  *   R4  The uniform variate of coordinate j at worker i is the 16-bit field (j mod 8)
  *       of Philox4x32-10(key = seed, counter = (j/8 lo, j/8 hi, i, round)).
- *   R5  Position on the grid in fp32: y = clamp(fma(r, kappa, g/2), 0, g) with
- *       kappa = (float)(g / (2 M)).  Clamping y to [0, g] is the truncation of r to
- *       [-M, M] carried through the (monotone) affine map of Algorithm 2.
- *   R6  Rounding decision: z0 = the largest index <= 2^b - 2 with T[z0] <= floor(y)
- *       (capped so that y = g falls in the last interval);
- *       up iff u16 < RN(2^16 * (y - T[z0]) / (T[z0+1] - T[z0])), the product taken as
- *       one fused multiply-add of (y - T[z0]) with R16[z0] = 65536 / (T[z0+1]-T[z0]).
+ *   R5  Position in the range, in fp32 on the unit interval:
+ *       u = clamp(fma(r, kappa, 1/2), 0, 1) with kappa = (float)(1 / (2 M)), i.e.
+ *       (r - m)/(M - m) of Algorithm 2.  Clamping u to [0, 1] is the truncation of r to
+ *       [-M, M] carried through the (monotone) affine map; the position on the grid
+ *       <g+1> is the real number u*g, which is never rounded on its own.
+ *   R6  Rounding decision: z0 = the largest index <= 2^b - 2 with T[z0] <= floor(u*g)
+ *       (capped so that u = 1 falls in the last interval); delta = fma(u, g, -T[z0]);
+ *       up iff u16 < RN(2^16 * delta / (T[z0+1] - T[z0])), the product taken as one fused
+ *       multiply-add of delta with R16[z0] = 65536 / (T[z0+1]-T[z0]).
  *       So P(up) is the paper's (a - q0)/(q1 - q0) rounded to a multiple of 2^-16.
  *   R7  Packing: index j occupies bits [(j mod 8/b) * b, +b) of byte j*b/8; sums are
  *       little-endian unsigned w-bit integers in coordinate order.
@@ -218,18 +220,17 @@ void thc_oracle_quantize(const float *r, uint64_t d_pad, uint32_t k, const float
         uint64_t j = (uint64_t)jj;
         float M = scales[j / B];
         if (!(M > 0.0f) || !isfinite(M)) { z[j] = 0; continue; }          /* R8 */
-        float kappa = (float)((double)g / (2.0 * (double)M));
-        float half_g = 0.5f * (float)g;
-        float y = fmaf(r[j], kappa, half_g);                              /* R5 */
-        if (!(y >= 0.0f)) y = 0.0f;                                       /* NaN -> 0 */
-        if (y > (float)g) y = (float)g;
-        int f = (int)floorf(y);
+        float kappa = (float)(1.0 / (2.0 * (double)M));
+        float pos = fmaf(r[j], kappa, 0.5f);                              /* R5 */
+        if (!(pos >= 0.0f)) pos = 0.0f;                                   /* NaN -> 0 */
+        if (pos > 1.0f) pos = 1.0f;
+        int f = (int)floor((double)pos * (double)g);                      /* exact product */
         if (f > (int)g - 1) f = (int)g - 1;
         uint32_t z0 = 0;                                                  /* R6 */
         while (z0 + 1 <= levels - 2 && (int)table[z0 + 1] <= f) ++z0;
         float gap = (float)((int)table[z0 + 1] - (int)table[z0]);
         float r16 = 65536.0f / gap;
-        float delta = y - (float)table[z0];
+        float delta = fmaf(pos, (float)g, -(float)table[z0]);
         float tau = fmaf(delta, r16, 8388608.0f);                         /* RN to integer */
         uint32_t threshold = (uint32_t)(tau - 8388608.0f);
         uint32_t u = thc_oracle_u16(seed, round, worker, j);

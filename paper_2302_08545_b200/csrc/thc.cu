@@ -121,8 +121,8 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
     float4 *tile = reinterpret_cast<float4 *>(smem_raw);
     uint32_t *sw = reinterpret_cast<uint32_t *>(smem_raw + kTileElems * 4);
     float2 *blk_const = reinterpret_cast<float2 *>(smem_raw + kTileElems * 4 + kSignWordsMax * 4);
-    uint2 *lut = reinterpret_cast<uint2 *>(smem_raw + kTileElems * 4 + kSignWordsMax * 4 +
-                                           (size_t)g.blocks_in_tile * 8);
+    uint4 *lut = reinterpret_cast<uint4 *>(smem_raw + kTileElems * 4 + kSignWordsMax * 4 +
+                                           (((size_t)g.blocks_in_tile * 8 + 15) & ~(size_t)15));
 
     const int tid = threadIdx.x;
     const uint32_t wl = blockIdx.y;
@@ -134,24 +134,21 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
     if (LOAD == kLoadGradF32 || LOAD == kLoadGradBF16 || STORE == kStoreOut)
         fill_sign_words(sw, g, base, keys, tid);
     if (STORE == kStoreQuant) {
-        // (kappa, g/2) per block; (0, 0) for a degenerate block
+        // (1/(2M), 1/2) per block; (0, 0) for a degenerate block
         for (uint32_t b = tid; b < g.blocks_in_tile; b += kThreads) {
             float2 c = make_float2(0.f, 0.f);
             if (first_blk + b < nblocks) {
                 const float M = scales[first_blk + b];
                 if (M > 0.0f && isfinite(M)) {
-                    c.x = (float)((double)g.granularity / (2.0 * (double)M));
-                    c.y = 0.5f * (float)g.granularity;
+                    c.x = (float)(1.0 / (2.0 * (double)M));
+                    c.y = 0.5f;
                 }
             }
             blk_const[b] = c;
         }
         if (!IDENTITY) {
-            const int rep = (int)g.lut_rep;
-            for (int idx = tid; idx < (int)(g.granularity + 1) * rep; idx += kThreads) {
-                const int f = idx / rep;
-                lut[idx] = make_uint2(dev->lut_tz[f], __float_as_uint(dev->lut_r16[f]));
-            }
+            for (int idx = tid; idx < (int)(g.granularity + 1) * kLutRep; idx += kThreads)
+                lut[idx] = dev->lut[idx / kLutRep];
         }
     }
     if (LOAD == kLoadSum8 || LOAD == kLoadSum16 || LOAD == kLoadSum32) {
@@ -264,8 +261,7 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
         unsigned char *pk = static_cast<unsigned char *>(out.p[wl]);
         float *rot = static_cast<float *>(rotated.p[wl]);
         const float gf = (float)g.granularity;
-        const int lane = tid & 31;
-        const uint2 *my_lut = lut + (g.lut_rep > 1 ? lane : 0);
+        const uint4 *my_lut = lut + (tid & (kLutRep - 1));
 #pragma unroll 1
         for (int i = 0; i < kTileChunks / 2 / kThreads; ++i) {
             const int u = tid + i * kThreads;
@@ -281,8 +277,7 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
             const float r[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
             const float2 bc = blk_const[(j >> g.k) - first_blk];
             const uint4 rnd = round_call(j, g.worker_base + wl, g.round, keys);
-            const uint64_t z = quantize8<BITS, IDENTITY>(r, bc.x, bc.y, gf, rnd, my_lut,
-                                                         (int)g.lut_rep);
+            const uint64_t z = quantize8<BITS, IDENTITY>(r, bc.x, bc.y, gf, rnd, my_lut, kLutRep);
             if constexpr (BITS == 8) *reinterpret_cast<uint2 *>(pk + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
             else if constexpr (BITS == 4) *reinterpret_cast<uint32_t *>(pk + j / 2) = (uint32_t)z;
             else if constexpr (BITS == 2) *reinterpret_cast<uint16_t *>(pk + j / 4) = (uint16_t)z;
@@ -315,9 +310,8 @@ quantize_rotated_kernel(PtrArray rotated, MutPtrArray packed, uint64_t d_pad, ui
                         uint32_t granularity, uint32_t round, uint32_t worker_base,
                         const float *__restrict__ scales, const DeviceBlock *dev, PhiloxKeys keys)
 {
-    __shared__ uint2 lut[256];
-    for (int f = threadIdx.x; f <= (int)granularity; f += kThreads)
-        lut[f] = make_uint2(dev->lut_tz[f], __float_as_uint(dev->lut_r16[f]));
+    __shared__ uint4 lut[256];
+    for (int f = threadIdx.x; f <= (int)granularity; f += kThreads) lut[f] = dev->lut[f];
     __syncthreads();
     const uint32_t wl = blockIdx.y;
     const float *rot = static_cast<const float *>(rotated.p[wl]);
@@ -330,13 +324,13 @@ quantize_rotated_kernel(PtrArray rotated, MutPtrArray packed, uint64_t d_pad, ui
         const float4 b = __ldg(reinterpret_cast<const float4 *>(rot + j + 4));
         const float r[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
         const float M = scales[j >> k];
-        float kappa = 0.f, half_g = 0.f;
+        float kappa = 0.f, offset = 0.f;
         if (M > 0.0f && isfinite(M)) {
-            kappa = (float)((double)granularity / (2.0 * (double)M));
-            half_g = 0.5f * gf;
+            kappa = (float)(1.0 / (2.0 * (double)M));
+            offset = 0.5f;
         }
         const uint4 rnd = round_call(j, worker_base + wl, round, keys);
-        const uint64_t z = quantize8<BITS, IDENTITY>(r, kappa, half_g, gf, rnd, lut, 1);
+        const uint64_t z = quantize8<BITS, IDENTITY>(r, kappa, offset, gf, rnd, lut, 1);
         if constexpr (BITS == 8) *reinterpret_cast<uint2 *>(pk + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
         else if constexpr (BITS == 4) *reinterpret_cast<uint32_t *>(pk + j / 2) = (uint32_t)z;
         else if constexpr (BITS == 2) *reinterpret_cast<uint16_t *>(pk + j / 4) = (uint16_t)z;
@@ -601,7 +595,7 @@ int thc_create(const thc_config *cfg, thc_ctx **out)
         k1 += 0xBB67AE85u;
     }
     const uint32_t g = cfg->granularity;
-    ctx->lut_rep = ((g + 1) * 32 * 8 <= (uint32_t)kLutRepMaxBytes) ? 32 : 1;
+    ctx->lut_rep = kLutRep;
 
     // host copy of the device block
     DeviceBlock *h = new (std::nothrow) DeviceBlock;
@@ -610,14 +604,15 @@ int thc_create(const thc_config *cfg, thc_ctx **out)
     const uint32_t levels = 1u << cfg->bits;
     for (uint32_t z = 0; z < levels; ++z) h->table[z] = cfg->table[z];
     for (uint32_t f = 0; f <= g; ++f) {
-        const uint32_t ff = f < g ? f : g - 1;            // y = g falls in the last interval
+        const uint32_t ff = f < g ? f : g - 1;            // u = 1 falls in the last interval
         uint32_t z0 = 0;
         while (z0 + 1 <= levels - 2 && cfg->table[z0 + 1] <= ff) ++z0;
-        const float tz = (float)cfg->table[z0];
-        uint32_t bits;
-        memcpy(&bits, &tz, 4);
-        h->lut_tz[f] = bits | z0;
-        h->lut_r16[f] = 65536.0f / (float)(cfg->table[z0 + 1] - cfg->table[z0]);
+        const float ntf = -(float)cfg->table[z0];
+        const float r16 = 65536.0f / (float)(cfg->table[z0 + 1] - cfg->table[z0]);
+        uint32_t b0, b1;
+        memcpy(&b0, &ntf, 4);
+        memcpy(&b1, &r16, 4);
+        h->lut[f] = make_uint4(b0, b1, z0, 0u);
     }
 
     int count = 0;
@@ -774,8 +769,9 @@ static tile_kernel_t pick_tile_kernel(uint32_t bits, bool identity)
 
 static size_t tile_smem_bytes(const thc_ctx *ctx, const TileGeom &g)
 {
-    return (size_t)kTileElems * 4 + kSignWordsMax * 4 + (size_t)g.blocks_in_tile * 8 +
-           (size_t)(ctx->cfg.granularity + 1) * ctx->lut_rep * 8;
+    return (size_t)kTileElems * 4 + kSignWordsMax * 4 +
+           (((size_t)g.blocks_in_tile * 8 + 15) & ~(size_t)15) +
+           (size_t)(ctx->cfg.granularity + 1) * kLutRep * 16;
 }
 
 static int launch_tile(const thc_ctx *ctx, tile_kernel_t kern, const TileGeom &g, uint64_t tiles,
@@ -872,7 +868,7 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, const thc_siz
     P.c_block = (float)(1.0 / sqrt((double)(1ull << k)));
     const uint64_t nblk_cached = sz.nblocks < (uint64_t)kBlockConstMax ? sz.nblocks : (uint64_t)kBlockConstMax;
     const size_t smem = (size_t)2 * kPElems * 4 + kPSignWords * 4 +
-                        (size_t)(ctx->cfg.granularity + 1) * kPLutRep * 8 + (size_t)nblk_cached * 8;
+                        (size_t)(ctx->cfg.granularity + 1) * kLutRep * 16 + (size_t)nblk_cached * 8;
     THC_CUDA(cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     kern<<<pl.grid, kPCtaThreads, smem, st>>>(P, in, out, rot, ctx->keys);

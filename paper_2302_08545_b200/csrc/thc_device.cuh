@@ -19,14 +19,13 @@ constexpr int kTileElems = 1 << kTileLog2;
 constexpr int kTileChunks = kTileElems / 4;    // 16-byte chunks
 constexpr int kThreads = 256;
 constexpr int kSignWordsMax = 1024;            // sign words a tile can need
-constexpr int kLutRepMaxBytes = 16384;
+constexpr int kLutRep = 8;                     // lane replication of the quantiser table
 
 // Lives in the context's device block.
 struct DeviceBlock {
     uint32_t status;             // THC_STATUS_* bits
     uint32_t counters[127];      // scheduling counters (self-resetting)
-    uint32_t lut_tz[256];        // by floor(y): float bits of T[z0] | z0
-    float    lut_r16[256];       // by floor(y): 65536 / (T[z0+1] - T[z0])
+    uint4    lut[256];           // by floor(u*g): (-T[z0] as float, 65536/(T[z0+1]-T[z0]), z0, 0)
     uint32_t table[256];         // T
 };
 
@@ -179,15 +178,17 @@ __device__ __forceinline__ void fwht_rounds(float4 *tile, int lo, int hi, int ti
 // --------------------------------------------------------------------------- quantiser
 // Stochastic quantisation of eight consecutive rotated coordinates to table indices
 // (Algorithm 2, worker lines; Section 4.1 for the rounding rule):
-//   y = clamp(fma(r, kappa, g/2), 0, g)        position on the grid <g+1>, truncated
-//   z0 = index of the table value at or below y, up iff u16 < RN(2^16 (y - T[z0]) / gap)
-// kappa = 0 and half_g = 0 encode a degenerate block (every index 0).
-// `lut` points at this lane's copy of the (T[z0] | z0, 65536/gap) pairs, `lut_stride`
+//   u = sat(fma(r, kappa, offset))          position in [m, M] on the unit interval, truncated
+//   f = floor(u * g)                         (one round-down fma onto 2^23; exact)
+//   z0 = index of the table value at or below u*g, delta = fma(u, g, -T[z0])
+//   up iff u16 < RN(2^16 delta / gap)        (one fma onto 2^23, integer compare)
+// kappa = 1/(2M) and offset = 1/2; kappa = offset = 0 encodes a degenerate block (index 0).
+// `lut` points at this lane's copy of the (-T[z0], 65536/gap, z0) entries, `lut_stride`
 // entries apart per floor value.  Returns the indices packed BITS apiece, coordinate 0 in
 // the low bits.
 template <int BITS, bool IDENTITY>
-__device__ __forceinline__ uint64_t quantize8(const float (&r)[8], float kappa, float half_g,
-                                              float gf, uint4 rnd, const uint2 *lut,
+__device__ __forceinline__ uint64_t quantize8(const float (&r)[8], float kappa, float offset,
+                                              float gf, uint4 rnd, const uint4 *lut,
                                               int lut_stride)
 {
     const uint32_t words[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
@@ -197,22 +198,21 @@ __device__ __forceinline__ uint64_t quantize8(const float (&r)[8], float kappa, 
 #endif
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-        float y = fmaf(r[e], kappa, half_g);
-        y = fminf(fmaxf(y, 0.0f), gf);
-        const float t = __fadd_rd(y, 8388608.0f);              // 2^23 + floor(y)
+        float u;
+        asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(u) : "f"(r[e]), "f"(kappa), "f"(offset));
+        const float t = __fmaf_rd(u, gf, 8388608.0f);          // 2^23 + floor(u * g)
         const uint32_t u16 = (e & 1) ? (words[e >> 1] >> 16) : (words[e >> 1] & 0xFFFFu);
         const uint32_t ub = u16 | 0x4B000000u;                 // bits of 2^23 + u16
         uint32_t z0;
         float tau;
         if (IDENTITY) {
             z0 = __float_as_uint(t) & 0xFFu;
-            const float delta = y - (t - 8388608.0f);
+            const float delta = fmaf(u, gf, 8388608.0f - t);
             tau = fmaf(delta, 65536.0f, 8388608.0f);
         } else {
-            const uint32_t f = __float_as_uint(t) & 0xFFu;
-            const uint2 entry = lut[f * lut_stride];
-            z0 = entry.x & 0xFFu;
-            const float delta = y - __uint_as_float(entry.x & 0xFFFFFF00u);
+            const uint4 entry = lut[(__float_as_uint(t) & 0xFFu) * lut_stride];
+            z0 = entry.z;
+            const float delta = fmaf(u, gf, __uint_as_float(entry.x));
             tau = fmaf(delta, __uint_as_float(entry.y), 8388608.0f);
         }
         const uint32_t z = z0 + (ub < __float_as_uint(tau) ? 1u : 0u);

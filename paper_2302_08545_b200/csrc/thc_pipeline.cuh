@@ -32,7 +32,6 @@ constexpr int kPChunks = kPElems / 4;
 constexpr int kPThreads = 128;                // compute threads of a CTA
 constexpr int kPCtaThreads = 160;             // plus one control warp that runs the queue
 constexpr int kPSignWords = 512;            // sign words a tile can need
-constexpr int kPLutRep = 16;                // lane replication of the quantiser table
 constexpr int kMaxRing = 56;
 constexpr int kBlockConstMax = 256;         // per-block constants cached in shared memory
 constexpr uint32_t kMaxPolls = 1u << 21;
@@ -205,8 +204,8 @@ __device__ __forceinline__ float2 block_constants(float M, uint32_t g, uint32_t 
     float2 c = make_float2(0.f, 0.f);
     if (M > 0.0f && isfinite(M)) {
         if (COMPRESS) {
-            c.x = (float)((double)g / (2.0 * (double)M));
-            c.y = 0.5f * (float)g;
+            c.x = (float)(1.0 / (2.0 * (double)M));
+            c.y = 0.5f;
         } else {
             c.x = (float)(2.0 * (double)M / ((double)g * (double)divisor));
             c.y = -M;
@@ -332,7 +331,7 @@ __device__ __forceinline__ void pass_a_round3_store(const float4 *tile, float *d
 struct EpilogueCtx {
     uint64_t j_tile;        // coordinate of (row 0, column 0) of the tile in the worker's vector
     float kappa, half_g, gf, c_block;
-    const uint2 *lut;
+    const uint4 *lut;
     uint32_t worker, round;
     unsigned char *packed;
     float *rotated;
@@ -355,7 +354,7 @@ __device__ __forceinline__ void epilogue_unit(const float4 &va, const float4 &vb
         }
         const float r[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
         const uint4 rnd = round_call(j, ep.worker, ep.round, keys);
-        const uint64_t z = quantize8<BITS, IDENTITY>(r, ep.kappa, ep.half_g, ep.gf, rnd, ep.lut, kPLutRep);
+        const uint64_t z = quantize8<BITS, IDENTITY>(r, ep.kappa, ep.half_g, ep.gf, rnd, ep.lut, kLutRep);
         if constexpr (BITS == 8)
             *reinterpret_cast<uint2 *>(ep.packed + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
         else if constexpr (BITS == 4)
@@ -422,30 +421,35 @@ __device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, in
 // The same for the 128-row x 16-chunk tile (k = 20): rows row_low + 16 m, m = 0..7; lanes
 // 0-7 of a quarter warp cover four units of two adjacent rows, which is conflict-free.
 template <bool COMPRESS, int BITS, bool IDENTITY>
-__device__ __forceinline__ void pass_b_last_round_kb7(const float4 *tile, int tid,
+__device__ __forceinline__ void pass_b_last_round_kb7(float4 *tile, int tid,
                                                       const EpilogueCtx &ep, const PhiloxKeys &keys)
 {
     const int uu = (tid & 3) | ((tid >> 1) & 4);
     const int row_low = ((tid >> 2) & 1) | ((tid >> 4) << 1);
     const int x = row_low & 7;
-    const float4 *pa = tile + row_low * 16 + ((2 * uu) ^ x);
-    const float4 *pb = tile + row_low * 16 + ((2 * uu + 1) ^ x);
-    float4 a[8], b[8];
+    float4 *pa = tile + row_low * 16 + ((2 * uu) ^ x);
+    float4 *pb = tile + row_low * 16 + ((2 * uu + 1) ^ x);
+    {
+        float4 a[8], b[8];
 #pragma unroll
-    for (int m = 0; m < 8; ++m) { a[m] = pa[m << 8]; b[m] = pb[m << 8]; }
+        for (int m = 0; m < 8; ++m) { a[m] = pa[m << 8]; b[m] = pb[m << 8]; }
 #pragma unroll
-    for (int t = 0; t < 3; ++t) {
+        for (int t = 0; t < 3; ++t) {
 #pragma unroll
-        for (int m = 0; m < 8; ++m)
-            if (!(m & (1 << t))) {
-                butterfly(a[m], a[m | (1 << t)]);
-                butterfly(b[m], b[m | (1 << t)]);
-            }
+            for (int m = 0; m < 8; ++m)
+                if (!(m & (1 << t))) {
+                    butterfly(a[m], a[m | (1 << t)]);
+                    butterfly(b[m], b[m | (1 << t)]);
+                }
+        }
+        // back to the thread's own slots: the epilogue below is a compact loop (code size)
+#pragma unroll
+        for (int m = 0; m < 8; ++m) { pa[m << 8] = a[m]; pb[m << 8] = b[m]; }
     }
     const uint64_t j0 = ep.j_tile + ((uint64_t)row_low << kPLog2) + 8 * uu;
-#pragma unroll
+#pragma unroll 1
     for (int m = 0; m < 8; ++m)
-        epilogue_unit<COMPRESS, BITS, IDENTITY>(a[m], b[m], j0 + ((uint64_t)m << (kPLog2 + 4)),
+        epilogue_unit<COMPRESS, BITS, IDENTITY>(pa[m << 8], pb[m << 8], j0 + ((uint64_t)m << (kPLog2 + 4)),
                                                 row_low + 16 * m, uu, ep, keys);
 }
 
@@ -462,9 +466,9 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
     float4 *bufs[2] = {reinterpret_cast<float4 *>(pipe_smem),
                        reinterpret_cast<float4 *>(pipe_smem + kPElems * 4)};
     uint32_t *sw = reinterpret_cast<uint32_t *>(pipe_smem + 2 * kPElems * 4);
-    uint2 *lut = reinterpret_cast<uint2 *>(pipe_smem + 2 * kPElems * 4 + kPSignWords * 4);
+    uint4 *lut = reinterpret_cast<uint4 *>(pipe_smem + 2 * kPElems * 4 + kPSignWords * 4);
     float2 *blk_const = reinterpret_cast<float2 *>(pipe_smem + 2 * kPElems * 4 + kPSignWords * 4 +
-                                                   (size_t)(P.granularity + 1) * kPLutRep * 8);
+                                                   (size_t)(P.granularity + 1) * kLutRep * 16);
     __shared__ TaskInfo s_info[2];
     __shared__ uint32_t s_published;       // tasks the control warp has handed over so far
 
@@ -478,10 +482,8 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
     const uint64_t policy = make_evict_first_policy();
 
     if (kCompress && !IDENTITY) {
-        for (int idx = tid; idx < (int)(P.granularity + 1) * kPLutRep; idx += kPThreads) {
-            const int f = idx / kPLutRep;
-            lut[idx] = make_uint2(P.dev->lut_tz[f], __float_as_uint(P.dev->lut_r16[f]));
-        }
+        for (int idx = tid; idx < (int)(P.granularity + 1) * kLutRep; idx += kPThreads)
+            lut[idx] = P.dev->lut[idx / kLutRep];
     }
     const uint32_t nblk_total = (uint32_t)(P.d_pad >> P.k);
     const uint32_t nblk_cached = nblk_total < (uint32_t)kBlockConstMax ? nblk_total : (uint32_t)kBlockConstMax;
@@ -670,7 +672,7 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
             EpilogueCtx ep;
             ep.j_tile = j_tile;
             ep.kappa = bc.x; ep.half_g = bc.y; ep.gf = (float)P.granularity; ep.c_block = P.c_block;
-            ep.lut = lut + (tid & (kPLutRep - 1));
+            ep.lut = lut + (tid & (kLutRep - 1));
             ep.worker = P.worker_base + wl; ep.round = P.round;
             ep.packed = kCompress ? static_cast<unsigned char *>(outp.p[wl]) : nullptr;
             ep.rotated = kCompress ? static_cast<float *>(rotated.p[wl]) : nullptr;
