@@ -192,10 +192,12 @@ __device__ __forceinline__ uint64_t quantize8(const float (&r)[8], float kappa, 
                                               int lut_stride)
 {
     const uint32_t words[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
-    uint64_t out = 0;
 #ifdef THC_EXP_NOQUANT
     return (uint64_t)(__float_as_uint(r[0]) ^ __float_as_uint(r[5]) ^ rnd.x ^ rnd.z) + __float_as_uint(kappa);
 #endif
+    // Indices are accumulated as z * 2^(BITS*slot) with multiply-adds into two 32-bit halves
+    // (coordinates 0-3 and 4-7 for BITS = 8, otherwise everything in the low half).
+    uint32_t acc[2] = {0u, 0u};
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
         float u;
@@ -215,10 +217,14 @@ __device__ __forceinline__ uint64_t quantize8(const float (&r)[8], float kappa, 
             const float delta = fmaf(u, gf, __uint_as_float(entry.x));
             tau = fmaf(delta, __uint_as_float(entry.y), 8388608.0f);
         }
-        const uint32_t z = z0 + (ub < __float_as_uint(tau) ? 1u : 0u);
-        out |= (uint64_t)z << (e * BITS);
+        constexpr int half = BITS == 8 ? 1 : 0;
+        const int slot = BITS == 8 ? (e & 3) : e;
+        const int h = half ? (e >> 2) : 0;
+        const uint32_t weight = 1u << (BITS * slot);
+        acc[h] = z0 * weight + acc[h];
+        if (ub < __float_as_uint(tau)) acc[h] += weight;
     }
-    return out;
+    return (uint64_t)acc[0] | ((uint64_t)acc[1] << 32);
 }
 
 }  // namespace thc

@@ -292,9 +292,12 @@ __device__ __forceinline__ void round_bits_4_7(float4 *tile, int tid)
 {
     float4 *mine = tile + ((tid >> 4) << 8);
     const int low = tid & 15;
+    float4 *q[8];
+#pragma unroll
+    for (int x = 0; x < 8; ++x) q[x] = mine + (low ^ x);
     float4 v[16];
 #pragma unroll
-    for (int m = 0; m < 16; ++m) v[m] = mine[16 * m + (low ^ (m & 7))];
+    for (int m = 0; m < 16; ++m) v[m] = q[m & 7][16 * m];
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
 #pragma unroll
@@ -302,7 +305,7 @@ __device__ __forceinline__ void round_bits_4_7(float4 *tile, int tid)
             if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
     }
 #pragma unroll
-    for (int m = 0; m < 16; ++m) mine[16 * m + (low ^ (m & 7))] = v[m];
+    for (int m = 0; m < 16; ++m) q[m & 7][16 * m] = v[m];
 }
 
 // Last round of a pass-A tile (chunk bits 8..10) with the result stored straight to the ring.
@@ -447,7 +450,7 @@ __device__ __forceinline__ void pass_b_last_round_kb7(float4 *tile, int tid,
         for (int m = 0; m < 8; ++m) { pa[m << 8] = a[m]; pb[m << 8] = b[m]; }
     }
     const uint64_t j0 = ep.j_tile + ((uint64_t)row_low << kPLog2) + 8 * uu;
-#pragma unroll 1
+#pragma unroll 2
     for (int m = 0; m < 8; ++m)
         epilogue_unit<COMPRESS, BITS, IDENTITY>(pa[m << 8], pb[m << 8], j0 + ((uint64_t)m << (kPLog2 + 4)),
                                                 row_low + 16 * m, uu, ep, keys);
@@ -493,6 +496,9 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
 
     // ---- issue the tile load of a task into a buffer (all threads)
     auto issue_load = [&](const TaskInfo &ti, float4 *tile) {
+#ifdef THC_EXP_NO_LOAD
+        return;
+#endif
         const bool is_b = ti.is_b != 0;
         const uint32_t wl = ti.wl;
         const uint64_t r = ti.r;
@@ -500,6 +506,14 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
         if (is_b) {
             // panel idx: rows 2^13 apart in the ring slot, 2^(13-kb) columns each
             const float *src = P.ring + (size_t)slot * B + ((size_t)ti.idx << (kPLog2 - kb));
+            if (KB == 7) {
+                // chunk tid + 128 i is (row (tid >> 4) + 8 i, column chunk tid & 15)
+                const float *xs = src + ((size_t)(tid >> 4) << kPLog2) + 4 * (tid & 15);
+                float4 *dst = tile + (tid ^ ((tid >> 4) & 7));
+#pragma unroll
+                for (int i = 0; i < kPChunks / kPThreads; ++i)
+                    cp_async16(dst + i * kPThreads, xs + ((size_t)i << (kPLog2 + 3)));
+            } else
 #pragma unroll 4
             for (int i = 0; i < kPChunks / kPThreads; ++i) {
                 const int c = tid + i * kPThreads;
@@ -661,11 +675,17 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
                 *reinterpret_cast<uint4 *>(sw + 4 * tid) = ph;
             }
             compute_barrier();                        // tile and sign words visible
+#ifndef THC_EXP_NO_A_R1
             pass_a_round1<kCompress>(tile, sw, tid);
+#endif
             compute_barrier();
+#ifndef THC_EXP_NO_A_R2
             round_bits_4_7(tile, tid);
+#endif
             compute_barrier();
+#ifndef THC_EXP_NO_A_R3
             pass_a_round3_store(tile, P.ring + (size_t)slot * B + ((size_t)idx << kPLog2), tid);
+#endif
         } else {
             // ================================ pass B: panel idx of worker-block wb
             const uint64_t j_tile = r * B + ((uint64_t)idx << (kPLog2 - kb));
@@ -689,7 +709,9 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
             compute_barrier();                        // tile (and sign words) visible
             const int e1 = kb < 4 ? kb : 4;
             if (KB == 7) {
+#ifndef THC_EXP_NO_B_R1
                 round_bits_4_7(tile, tid);
+#endif
             } else {
                 switch (e1) {
                 case 4: p_round<4>(tile, ccl, tid); break;
@@ -699,7 +721,9 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
             }
             compute_barrier();
             if (KB == 7) {
+#ifndef THC_EXP_NO_B_LAST
                 pass_b_last_round_kb7<kCompress, BITS, IDENTITY>(tile, tid, ep, keys);
+#endif
             } else {
                 const int rem = kb - e1;
                 const int e_last = rem < 3 ? rem : 3;
