@@ -14,7 +14,6 @@
 #include <math.h>
 #include <new>
 #include <stdio.h>
-#include <stdlib.h>
 #include <string.h>
 
 namespace thc {
@@ -335,6 +334,47 @@ quantize_rotated_kernel(PtrArray rotated, MutPtrArray packed, uint64_t d_pad, ui
         else if constexpr (BITS == 4) *reinterpret_cast<uint32_t *>(pk + j / 2) = (uint32_t)z;
         else if constexpr (BITS == 2) *reinterpret_cast<uint16_t *>(pk + j / 4) = (uint16_t)z;
         else pk[j / 8] = (unsigned char)z;
+    }
+}
+
+// Fast path of the PS sum for 4-bit indices, 8-bit sums and table values below 128 (the
+// paper's prototype: 4-bit indices, 8-bit table values and sums, Section 3).  The 16 table
+// bytes sit in four registers; `prmt` looks four indices up at once.  A selector nibble with
+// bit 3 set makes prmt return the sign of the selected byte, i.e. 0 for values < 128, so the
+// low half of the table answers indices 0-7 and, with bit 3 flipped, the high half answers
+// 8-15; the two results are disjoint and are added into packed byte accumulators (no byte
+// can overflow because workers * g <= 255).
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+__global__ void __launch_bounds__(kThreads)
+aggregate_b4w8_kernel(PtrArray in, uint32_t n, uint64_t units16, const DeviceBlock *dev,
+                      uint4 *__restrict__ sum)
+{
+    uint32_t t[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        t[q] = dev->table[4 * q] | (dev->table[4 * q + 1] << 8) | (dev->table[4 * q + 2] << 16) |
+               (dev->table[4 * q + 3] << 24);
+    for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < units16;
+         u += (uint64_t)gridDim.x * kThreads) {
+        uint32_t acc[4] = {0u, 0u, 0u, 0u};                  // 16 sums of 8 bits
+#pragma unroll 4
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint2 w = __ldg(reinterpret_cast<const uint2 *>(in.p[i]) + u);   // 16 indices
+            const uint32_t words[2] = {w.x, w.y};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t a = words[h], b = a ^ 0x88888888u;
+                acc[2 * h] += prmt(t[0], t[1], a) + prmt(t[2], t[3], b);
+                acc[2 * h + 1] += prmt(t[0], t[1], a >> 16) + prmt(t[2], t[3], b >> 16);
+            }
+        }
+        sum[u] = make_uint4(acc[0], acc[1], acc[2], acc[3]);
     }
 }
 
@@ -669,8 +709,6 @@ static PipePlan plan_pipeline(const thc_ctx *ctx, uint64_t wb_count)
         ring = kMaxRing;
         if (lag > ring - 2) lag = ring - 2;
     }
-    if (const char *e = getenv("THC_EXP_LAG")) { lag = strtoull(e, nullptr, 10); if (lag > wb_count) lag = wb_count; }
-    if (const char *e = getenv("THC_EXP_RING")) { ring = strtoull(e, nullptr, 10); if (ring > wb_count) ring = wb_count; if (ring > (uint64_t)kMaxRing) ring = kMaxRing; }
     p.lag = (uint32_t)lag;
     p.ring = (uint32_t)ring;
     return p;
@@ -1036,6 +1074,16 @@ int thc_aggregate(thc_ctx *ctx, const void *const *packed, uint32_t n, uint64_t 
     const uint64_t cap = (uint64_t)ctx->sm_count * 16;
     if (blocks > cap) blocks = cap;
     unsigned char *s = static_cast<unsigned char *>(sum);
+    if (ctx->cfg.bits == 4 && ctx->acc_bits == 8 && ctx->cfg.granularity < 128 && sz.d_pad % 16 == 0) {
+        const uint64_t units16 = sz.d_pad / 16;
+        uint64_t nb = (units16 + kThreads - 1) / kThreads;
+        const uint64_t cap16 = (uint64_t)ctx->sm_count * 8;
+        if (nb > cap16) nb = cap16;
+        aggregate_b4w8_kernel<<<(unsigned)nb, kThreads, 0, st>>>(in, n, units16, ctx->dev,
+                                                                  reinterpret_cast<uint4 *>(s));
+        THC_CUDA(cudaGetLastError());
+        return THC_OK;
+    }
 #define THC_AG(B, W) aggregate_kernel<B, W><<<(unsigned)blocks, kThreads, 0, st>>>(in, n, units, sz.d_pad, ctx->dev, s)
 #define THC_AGW(B)                                       \
     do {                                                 \
@@ -1066,3 +1114,4 @@ int thc_status(thc_ctx *ctx, uint32_t *flags, void *stream)
     THC_CUDA(cudaStreamSynchronize(st));
     return THC_OK;
 }
+

@@ -64,9 +64,6 @@ __device__ __forceinline__ uint4 round_call(uint64_t j, uint32_t worker, uint32_
                                             const PhiloxKeys &keys)
 {
     const uint64_t call = j >> 3;
-#ifdef THC_EXP_NOPHILOX
-    return make_uint4((uint32_t)call, worker, round, keys.k[0]);
-#endif
     return philox4x32_10((uint32_t)call, (uint32_t)(call >> 32), worker, round, keys);
 }
 
@@ -84,9 +81,6 @@ __device__ __forceinline__ float2 sub2(float2 a, float2 b)
 // One radix-2 butterfly on four independent columns: (a, b) <- (a + b, a - b).
 __device__ __forceinline__ void butterfly(float4 &a, float4 &b)
 {
-#ifdef THC_EXP_NOBFLY
-    return;
-#endif
     const float2 alo = make_float2(a.x, a.y), ahi = make_float2(a.z, a.w);
     const float2 blo = make_float2(b.x, b.y), bhi = make_float2(b.z, b.w);
     const float2 slo = add2(alo, blo), shi = add2(ahi, bhi);
@@ -115,9 +109,6 @@ __device__ __forceinline__ float4 scale4(float4 v, float c)
 // Flip the signs of a chunk by bits [0,4) of `bits` (bit e set -> element e negated).
 __device__ __forceinline__ float4 flip4(float4 v, uint32_t bits)
 {
-#ifdef THC_EXP_NOFLIP
-    return v;
-#endif
     v.x = __uint_as_float(__float_as_uint(v.x) ^ ((bits << 31) & 0x80000000u));
     v.y = __uint_as_float(__float_as_uint(v.y) ^ ((bits << 30) & 0x80000000u));
     v.z = __uint_as_float(__float_as_uint(v.z) ^ ((bits << 29) & 0x80000000u));
@@ -192,9 +183,6 @@ __device__ __forceinline__ uint64_t quantize8(const float (&r)[8], float kappa, 
                                               int lut_stride)
 {
     const uint32_t words[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
-#ifdef THC_EXP_NOQUANT
-    return (uint64_t)(__float_as_uint(r[0]) ^ __float_as_uint(r[5]) ^ rnd.x ^ rnd.z) + __float_as_uint(kappa);
-#endif
     // Indices are accumulated as z * 2^(BITS*slot) with multiply-adds into two 32-bit halves
     // (coordinates 0-3 and 4-7 for BITS = 8, otherwise everything in the low half).
     uint32_t acc[2] = {0u, 0u};

@@ -496,9 +496,6 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
 
     // ---- issue the tile load of a task into a buffer (all threads)
     auto issue_load = [&](const TaskInfo &ti, float4 *tile) {
-#ifdef THC_EXP_NO_LOAD
-        return;
-#endif
         const bool is_b = ti.is_b != 0;
         const uint32_t wl = ti.wl;
         const uint64_t r = ti.r;
@@ -643,20 +640,25 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
         const int s1 = cur ^ 1;
         if (!me_loaded) issue_load(me, bufs[cur]);
         cp_async_commit();
-        // Is the next task already handed over?  Then its tile streams in while this one is
-        // computed.  A task is never waited for before the current one is finished and
+        cp_async_wait_all();
+        // Every barrier of the task doubles as a look at the hand-over flag: as soon as the
+        // control warp has published the next task, its tile starts streaming into the other
+        // buffer.  A task is never waited for before the current one is finished and
         // signalled: it may depend on it.
-        const bool have_next = compute_barrier_or(
-            *reinterpret_cast<volatile uint32_t *>(&s_published) >= it + 2);
+        bool have_next = false;
         TaskInfo nxt = me;
-        if (have_next) {
-            bar_sync(1 + s1, kPCtaThreads);
-            nxt = s_info[s1];
-            bar_arrive(3 + s1, kPCtaThreads);
-            if (nxt.idx != 0xFFFFFFFFu) issue_load(nxt, bufs[s1]);
-        }
-        cp_async_commit();
-        cp_async_wait_but_one();
+        auto barrier_and_prefetch = [&]() {
+            const bool pub = compute_barrier_or(
+                !have_next && *reinterpret_cast<volatile uint32_t *>(&s_published) >= it + 2);
+            if (pub) {
+                bar_sync(1 + s1, kPCtaThreads);
+                nxt = s_info[s1];
+                bar_arrive(3 + s1, kPCtaThreads);
+                if (nxt.idx != 0xFFFFFFFFu) issue_load(nxt, bufs[s1]);
+                cp_async_commit();
+                have_next = true;
+            }
+        };
 
         const bool is_b = me.is_b != 0;
         const uint32_t wl = me.wl;
@@ -674,18 +676,12 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
                 const uint4 ph = sign_call(j0 + 128ull * tid, P.round, keys);
                 *reinterpret_cast<uint4 *>(sw + 4 * tid) = ph;
             }
-            compute_barrier();                        // tile and sign words visible
-#ifndef THC_EXP_NO_A_R1
+            barrier_and_prefetch();                   // tile and sign words visible
             pass_a_round1<kCompress>(tile, sw, tid);
-#endif
-            compute_barrier();
-#ifndef THC_EXP_NO_A_R2
+            barrier_and_prefetch();
             round_bits_4_7(tile, tid);
-#endif
-            compute_barrier();
-#ifndef THC_EXP_NO_A_R3
+            barrier_and_prefetch();
             pass_a_round3_store(tile, P.ring + (size_t)slot * B + ((size_t)idx << kPLog2), tid);
-#endif
         } else {
             // ================================ pass B: panel idx of worker-block wb
             const uint64_t j_tile = r * B + ((uint64_t)idx << (kPLog2 - kb));
@@ -706,12 +702,10 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
                 g.row_stride = 1ull << kPLog2; g.round = P.round;
                 fill_sign_words(sw, g, j_tile, keys, tid, kPThreads);
             }
-            compute_barrier();                        // tile (and sign words) visible
+            barrier_and_prefetch();                   // tile (and sign words) visible
             const int e1 = kb < 4 ? kb : 4;
             if (KB == 7) {
-#ifndef THC_EXP_NO_B_R1
                 round_bits_4_7(tile, tid);
-#endif
             } else {
                 switch (e1) {
                 case 4: p_round<4>(tile, ccl, tid); break;
@@ -719,11 +713,9 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
                 default: p_round<2>(tile, ccl, tid); break;
                 }
             }
-            compute_barrier();
+            barrier_and_prefetch();
             if (KB == 7) {
-#ifndef THC_EXP_NO_B_LAST
                 pass_b_last_round_kb7<kCompress, BITS, IDENTITY>(tile, tid, ep, keys);
-#endif
             } else {
                 const int rem = kb - e1;
                 const int e_last = rem < 3 ? rem : 3;

@@ -11,7 +11,7 @@ import os
 from dataclasses import dataclass
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.environ.get("THC_LIB", os.path.join(_HERE, "libthc.so"))
+_LIB_PATH = os.path.join(_HERE, "libthc.so")
 _lib = None
 
 THC_OK, THC_EINVAL, THC_EUNSUPPORTED, THC_ECUDA, THC_EWORKSPACE = 0, -1, -2, -3, -4
