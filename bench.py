@@ -31,7 +31,11 @@ from paper_2302_08545_b200 import workloads as W  # noqa: E402
 
 METRIC = "gradient GB/s per compress+aggregate+decompress round; % of HBM roofline"
 UNIT = "GB/s"
-KERNELS_PER_STEP = {"prepare": 2, "compress": 2, "aggregate": 1, "decompress": 2}
+KERNELS_PER_STEP = {"prepare": 2, "compress": 1, "aggregate": 1, "decompress": 1}
+# DRAM bytes per (worker, padded coordinate) of the compress kernel, measured with ncu on the
+# d=2^24, n=4, b=4 sweep point (profiles/thc_pipeline_kernel_sweep_d2p24_b4_n4.md); traffic
+# grows in proportion to n*d_pad, so a full launch is this times n*d_pad.
+NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.315}
 
 
 def pick_workload(name: str) -> W.Workload:
@@ -52,45 +56,68 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Streams SM clocks and throttle reasons from one nvidia-smi process (loop mode) and
+    keeps the samples that arrive between mark_start() and mark_end()."""
     QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index = index
-        self.samples = []
-        self._stop = threading.Event()
+    def __init__(self, index: int, period_ms: int = 20):
+        self.samples = []          # (host time, fields)
+        self.t0 = self.t1 = None
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", str(period_ms)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
         self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
 
     def _run(self):
-        while not self._stop.is_set():
+        if self.proc is None:
+            return
+        for line in self.proc.stdout:
+            fields = [f.strip() for f in line.strip().split(",")]
+            if len(fields) >= 6:
+                self.samples.append((time.perf_counter(), fields))
+
+    def wait_ready(self, timeout=3.0):
+        t = time.perf_counter()
+        while not self.samples and time.perf_counter() - t < timeout:
+            time.sleep(0.01)
+
+    def mark_start(self):
+        self.t0 = time.perf_counter()
+
+    def mark_end(self):
+        self.t1 = time.perf_counter()
+
+    def close(self):
+        if self.proc is not None:
+            self.proc.terminate()
             try:
-                out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
-                                      "--format=csv,noheader,nounits"], capture_output=True,
-                                     text=True, timeout=5).stdout.strip()
-                if out:
-                    self.samples.append([s.strip() for s in out.splitlines()[0].split(",")])
+                self.proc.wait(timeout=3)
             except Exception:
-                pass
-            self._stop.wait(0.1)
-
-    def __enter__(self):
-        self._thread.start()
-        return self
-
-    def __exit__(self, *a):
-        self._stop.set()
-        self._thread.join(timeout=6)
+                self.proc.kill()
 
     def summary(self):
-        if not self.samples:
+        inside = [f for (t, f) in self.samples if self.t0 is not None and self.t0 <= t <= self.t1]
+        note = "during the timed region"
+        if not inside and self.samples:
+            # region shorter than the sampling period: take the samples closest to it
+            mid = 0.5 * (self.t0 + self.t1)
+            inside = [min(self.samples, key=lambda s: abs(s[0] - mid))[1]]
+            note = "nearest sample (timed region shorter than the sampling period)"
+        if not inside:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
-        sm = sorted(float(s[0]) for s in self.samples)
+        sm = sorted(float(f[0]) for f in inside)
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names) if any(s[2 + i] == "Active" for s in self.samples)]
-        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(self.samples[0][1]),
-                "reasons": reasons, "samples": len(sm)}
+        reasons = [n for i, n in enumerate(names) if any(f[2 + i] == "Active" for f in inside)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(inside[0][1]), "reasons": reasons,
+                "samples": len(sm), "note": note}
 
 
 def visible_gpu_index(local_rank: int) -> int:
@@ -234,12 +261,17 @@ def run_gpu(args):
     torch.cuda.synchronize()
     events = []
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(visible_gpu_index(local_rank)) as clocks:
-        start.record(stream)
-        for _ in range(args.steps):
-            step(events)
-        end.record(stream)
-        torch.cuda.synchronize()
+    clocks = ClockSampler(visible_gpu_index(local_rank))
+    clocks.wait_ready()
+    torch.cuda.synchronize()
+    clocks.mark_start()
+    start.record(stream)
+    for _ in range(args.steps):
+        step(events)
+    end.record(stream)
+    torch.cuda.synchronize()
+    clocks.mark_end()
+    clocks.close()
     if world > 1:
         dist.barrier()
     ms_local = start.elapsed_time(end) / args.steps
@@ -288,6 +320,8 @@ def run_gpu(args):
     comp_ms = per_call_ms["compress"]
     achieved = ab["compress"] / (comp_ms * 1e-3) / 1e9
     in_bytes = w.n * w.d * (4 if w.in_dtype == "f32" else 2)
+    per_coord = NCU_COMPRESS_DRAM_BYTES_PER_COORD.get((w.in_dtype, w.bits))
+    traffic = None if per_coord is None or w.log2_block < 15 else per_coord * w.n * w.d_pad
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
@@ -298,10 +332,13 @@ def run_gpu(args):
                 "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": w.d * 4,
                 "ms_per_step": e2e_ms, "steps": e2e_steps},
         "gpu_launches": args.steps * sum(KERNELS_PER_STEP.values()),
-        "roofline": {"kernel": "thc_compress (RHT + quantise + pack kernels)", "bound": "hbm",
-                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_source": peak_src, "algorithmic_bytes_per_launch": ab["compress"],
-                     "ms_per_launch": comp_ms, "traffic": None},
+        "roofline": {"kernel": "thc_compress: one persistent RHT + quantise + pack kernel per call",
+                     "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": peak_src,
+                     "algorithmic_bytes_per_launch": ab["compress"], "ms_per_launch": comp_ms,
+                     "traffic": traffic,
+                     "traffic_source": "ncu dram bytes on the d=2^24 n=4 b=4 sweep point, scaled by n*d_pad"
+                                       if traffic is not None else None},
         "per_call_ms": per_call_ms,
         "round_excl_prepare": {
             "ms": round_ms, "gradient_gbs": grad_bytes / (round_ms * 1e-3) / 1e9,
@@ -321,7 +358,7 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="thc", choices=["thc", "reference"])
     ap.add_argument("--workload", default="cfg2")

@@ -428,22 +428,27 @@ prepare_partial_kernel(PtrArray in, uint64_t d, uint32_t chunk_log2, uint64_t ch
     }
 }
 
-// M per block from the partial sums (Section 5.3: M = t_p * max_i ||x_i|| / sqrt(B)).
-__global__ void prepare_final_kernel(const double *__restrict__ partial, uint32_t n,
-                                     uint64_t nblocks, uint64_t chunks_per_block,
-                                     uint64_t chunks_per_worker, double t_p, uint32_t k,
-                                     float *__restrict__ scales, DeviceBlock *dev)
+// M per block from the partial sums (Section 5.3: M = t_p * max_i ||x_i|| / sqrt(B)).  One warp
+// per RHT block; the summation order is fixed (strided per lane, then a butterfly of
+// shuffles), so the result does not depend on timing.
+__global__ void __launch_bounds__(128)
+prepare_final_kernel(const double *__restrict__ partial, uint32_t n, uint64_t nblocks,
+                     uint64_t chunks_per_block, uint64_t chunks_per_worker, double t_p, uint32_t k,
+                     float *__restrict__ scales, DeviceBlock *dev)
 {
-    const uint64_t blk = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint64_t blk = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
     if (blk >= nblocks) return;
     double ell = 0.0;
     for (uint32_t i = 0; i < n; ++i) {
         double s = 0.0;
         const double *p = partial + (uint64_t)i * chunks_per_worker + blk * chunks_per_block;
-        for (uint64_t c = 0; c < chunks_per_block; ++c) s += p[c];
+        for (uint64_t c = lane; c < chunks_per_block; c += 32) s += p[c];
+        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
         const double norm = sqrt(s);
         if (norm > ell || norm != norm) ell = norm;    // a NaN norm sticks
     }
+    if (lane != 0) return;
     float M = (float)(t_p * ell / sqrt((double)((uint64_t)1 << k)));
     uint32_t flags = 0;
     if (!isfinite(M)) { M = 0.0f; flags |= THC_STATUS_NONFINITE; }
@@ -780,7 +785,7 @@ int thc_prepare(thc_ctx *ctx, const void *const *grads, uint32_t n, uint64_t d, 
     else
         prepare_partial_kernel<false><<<grid, kThreads, 0, st>>>(in, d, chunk_log2, chunks_per_worker, partial);
     THC_CUDA(cudaGetLastError());
-    prepare_final_kernel<<<(unsigned)((sz.nblocks + 127) / 128), 128, 0, st>>>(
+    prepare_final_kernel<<<(unsigned)((sz.nblocks + 3) / 4), 128, 0, st>>>(
         partial, n, sz.nblocks, chunks_per_block, chunks_per_worker, ctx->cfg.t_p, k, scales, ctx->dev);
     THC_CUDA(cudaGetLastError());
     return THC_OK;
@@ -812,14 +817,37 @@ static size_t tile_smem_bytes(const thc_ctx *ctx, const TileGeom &g)
            (size_t)(ctx->cfg.granularity + 1) * kLutRep * 16;
 }
 
+// cudaFuncSetAttribute is needed once per kernel and dynamic shared-memory size; remember
+// what has been set per (kernel, device); a larger request raises the recorded size.  Not
+// thread-safe: concurrent first calls from several host threads may both set the attribute,
+// which is harmless.
+static int ensure_dynamic_smem(const void *kern, size_t smem)
+{
+    static const void *seen_kern[96];
+    static size_t seen_size[96];
+    static int seen_dev[96];
+    static int seen = 0;
+    int dev = 0;
+    THC_CUDA(cudaGetDevice(&dev));
+    for (int i = 0; i < seen; ++i)
+        if (seen_kern[i] == kern && seen_dev[i] == dev) {
+            if (seen_size[i] >= smem) return THC_OK;
+            THC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            seen_size[i] = smem;
+            return THC_OK;
+        }
+    THC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if (seen < 96) { seen_kern[seen] = kern; seen_size[seen] = smem; seen_dev[seen] = dev; ++seen; }
+    return THC_OK;
+}
+
 static int launch_tile(const thc_ctx *ctx, tile_kernel_t kern, const TileGeom &g, uint64_t tiles,
                        uint32_t n_local, const PtrArray &in, const MutPtrArray &out,
                        const MutPtrArray &rot, const float *scales, cudaStream_t st)
 {
     if (tiles > 0x7FFFFFFFull) return THC_EUNSUPPORTED;
     const size_t smem = tile_smem_bytes(ctx, g);
-    THC_CUDA(cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    { const int rc = ensure_dynamic_smem(reinterpret_cast<const void *>(kern), smem); if (rc != THC_OK) return rc; }
     kern<<<dim3((unsigned)tiles, n_local), kThreads, smem, st>>>(g, in, out, rot, scales, ctx->dev,
                                                                  ctx->keys);
     THC_CUDA(cudaGetLastError());
@@ -907,8 +935,7 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, const thc_siz
     const uint64_t nblk_cached = sz.nblocks < (uint64_t)kBlockConstMax ? sz.nblocks : (uint64_t)kBlockConstMax;
     const size_t smem = (size_t)2 * kPElems * 4 + kPSignWords * 4 +
                         (size_t)(ctx->cfg.granularity + 1) * kLutRep * 16 + (size_t)nblk_cached * 8;
-    THC_CUDA(cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    { const int rc = ensure_dynamic_smem(reinterpret_cast<const void *>(kern), smem); if (rc != THC_OK) return rc; }
     kern<<<pl.grid, kPCtaThreads, smem, st>>>(P, in, out, rot, ctx->keys);
     THC_CUDA(cudaGetLastError());
     return THC_OK;
