@@ -57,6 +57,12 @@ def _load():
     lib.thc_oracle_rht_forward.restype = None
     lib.thc_oracle_rht_inverse.argtypes = [f32p, u64, u32, u64, u32, f32p]
     lib.thc_oracle_rht_inverse.restype = None
+    lib.thc_oracle_rht_forward_at.argtypes = [f32p, u64, u32, u64, u32, u64, f32p]
+    lib.thc_oracle_rht_forward_at.restype = None
+    lib.thc_oracle_rht_inverse_at.argtypes = [f32p, u64, u32, u64, u32, u64, f32p]
+    lib.thc_oracle_rht_inverse_at.restype = None
+    lib.thc_oracle_quantize_at.argtypes = [f32p, u64, u32, f32p, u32, u32, u16p, u64, u32, u32, u64, u8p]
+    lib.thc_oracle_quantize_at.restype = None
     lib.thc_oracle_quantize.argtypes = [f32p, u64, u32, f32p, u32, u32, u16p, u64, u32, u32, u8p]
     lib.thc_oracle_quantize.restype = None
     lib.thc_oracle_pack.argtypes = [u8p, u64, u32, u8p]
@@ -162,34 +168,39 @@ def scales(x, cfg: Config) -> np.ndarray:
     return out
 
 
-def rht_forward(x, cfg: Config, rnd: int) -> np.ndarray:
+def rht_forward(x, cfg: Config, rnd: int, j_base: int = 0) -> np.ndarray:
+    """j_base: padded coordinate of x[0] in the whole vector (a multiple of the block), for
+    transforming a slice of a long vector."""
     x = _f32(x)
     d = x.size
+    assert j_base % cfg.block == 0
     r = np.zeros(cfg.d_pad(d), dtype=np.float32)
-    _load().thc_oracle_rht_forward(_p(x, ctypes.c_float), d, cfg.log2_block, cfg.seed, rnd,
-                                   _p(r, ctypes.c_float))
+    _load().thc_oracle_rht_forward_at(_p(x, ctypes.c_float), d, cfg.log2_block, cfg.seed, rnd,
+                                      j_base, _p(r, ctypes.c_float))
     return r
 
 
-def rht_inverse(v, d: int, cfg: Config, rnd: int) -> np.ndarray:
+def rht_inverse(v, d: int, cfg: Config, rnd: int, j_base: int = 0) -> np.ndarray:
     v = _f32(v).copy()
-    assert v.size == cfg.d_pad(d)
+    assert v.size == cfg.d_pad(d) and j_base % cfg.block == 0
     out = np.zeros(d, dtype=np.float32)
-    _load().thc_oracle_rht_inverse(_p(v, ctypes.c_float), d, cfg.log2_block, cfg.seed, rnd,
-                                   _p(out, ctypes.c_float))
+    _load().thc_oracle_rht_inverse_at(_p(v, ctypes.c_float), d, cfg.log2_block, cfg.seed, rnd,
+                                      j_base, _p(out, ctypes.c_float))
     return out
 
 
-def quantize(r, scl, cfg: Config, rnd: int, worker: int) -> np.ndarray:
-    """Rotated coordinates -> one table index per coordinate (uint8, unpacked)."""
+def quantize(r, scl, cfg: Config, rnd: int, worker: int, j_base: int = 0) -> np.ndarray:
+    """Rotated coordinates -> one table index per coordinate (uint8, unpacked).  With j_base,
+    r is a slice starting at that padded coordinate and scl[0] is the scale of its block."""
     r = _f32(r)
     scl = _f32(scl)
+    assert j_base % cfg.block == 0
     z = np.zeros(r.size, dtype=np.uint8)
     t = cfg.table_u16()
-    _load().thc_oracle_quantize(_p(r, ctypes.c_float), r.size, cfg.log2_block,
-                                _p(scl, ctypes.c_float), cfg.bits, cfg.granularity,
-                                _p(t, ctypes.c_uint16), cfg.seed, rnd, worker,
-                                _p(z, ctypes.c_uint8))
+    _load().thc_oracle_quantize_at(_p(r, ctypes.c_float), r.size, cfg.log2_block,
+                                   _p(scl, ctypes.c_float), cfg.bits, cfg.granularity,
+                                   _p(t, ctypes.c_uint16), cfg.seed, rnd, worker, j_base,
+                                   _p(z, ctypes.c_uint8))
     return z
 
 

@@ -161,8 +161,19 @@ void thc_oracle_scales(const float *x, uint32_t n, uint64_t d, uint32_t k, doubl
  * Forward RHT of one worker's vector (Section 5.1): r = c_B * H_B (D x) per block.
  * x has d entries, r has d_pad = nb * B entries.
  * ---------------------------------------------------------------------------------- */
+void thc_oracle_rht_forward_at(const float *x, uint64_t d, uint32_t k, uint64_t seed,
+                               uint32_t round, uint64_t j_base, float *r);
+
 void thc_oracle_rht_forward(const float *x, uint64_t d, uint32_t k, uint64_t seed,
                             uint32_t round, float *r)
+{
+    thc_oracle_rht_forward_at(x, d, k, seed, round, 0, r);
+}
+
+/* The same on a slice of a longer vector: element 0 of x is padded coordinate j_base (a
+ * multiple of B) of the whole vector; only the sign diagonal depends on it. */
+void thc_oracle_rht_forward_at(const float *x, uint64_t d, uint32_t k, uint64_t seed,
+                               uint32_t round, uint64_t j_base, float *r)
 {
     uint64_t B = (uint64_t)1 << k;
     uint64_t nb = (d + B - 1) / B;
@@ -173,7 +184,7 @@ void thc_oracle_rht_forward(const float *x, uint64_t d, uint32_t k, uint64_t see
         for (uint64_t t = 0; t < B; ++t) {
             uint64_t j = (uint64_t)blk * B + t;
             float a = j < d ? x[j] : 0.0f;
-            v[t] = thc_oracle_sign(seed, round, j) < 0 ? -a : a;
+            v[t] = thc_oracle_sign(seed, round, j_base + j) < 0 ? -a : a;
         }
         thc_oracle_fwht(v, B);
         for (uint64_t t = 0; t < B; ++t) v[t] = v[t] * c;
@@ -182,8 +193,17 @@ void thc_oracle_rht_forward(const float *x, uint64_t d, uint32_t k, uint64_t see
 
 /* Inverse RHT (Section 5.1): out = D (c_B * H_B v) per block; v has d_pad entries and is
  * overwritten; out receives the first d coordinates. */
+void thc_oracle_rht_inverse_at(float *v, uint64_t d, uint32_t k, uint64_t seed, uint32_t round,
+                               uint64_t j_base, float *out);
+
 void thc_oracle_rht_inverse(float *v, uint64_t d, uint32_t k, uint64_t seed, uint32_t round,
                             float *out)
+{
+    thc_oracle_rht_inverse_at(v, d, k, seed, round, 0, out);
+}
+
+void thc_oracle_rht_inverse_at(float *v, uint64_t d, uint32_t k, uint64_t seed, uint32_t round,
+                               uint64_t j_base, float *out)
 {
     uint64_t B = (uint64_t)1 << k;
     uint64_t nb = (d + B - 1) / B;
@@ -196,7 +216,7 @@ void thc_oracle_rht_inverse(float *v, uint64_t d, uint32_t k, uint64_t seed, uin
             uint64_t j = (uint64_t)blk * B + t;
             if (j >= d) break;
             float a = w[t] * c;
-            out[j] = thc_oracle_sign(seed, round, j) < 0 ? -a : a;
+            out[j] = thc_oracle_sign(seed, round, j_base + j) < 0 ? -a : a;
         }
     }
 }
@@ -209,9 +229,21 @@ void thc_oracle_rht_inverse(float *v, uint64_t d, uint32_t k, uint64_t seed, uin
  *   table   T[0..2^b-1], 0 = T[0] < ... < T[2^b-1] = g
  *   z       receives one index per coordinate (unpacked, one byte each)
  * ---------------------------------------------------------------------------------- */
+void thc_oracle_quantize_at(const float *r, uint64_t d_pad, uint32_t k, const float *scales,
+                            uint32_t b, uint32_t g, const uint16_t *table, uint64_t seed,
+                            uint32_t round, uint32_t worker, uint64_t j_base, uint8_t *z);
+
 void thc_oracle_quantize(const float *r, uint64_t d_pad, uint32_t k, const float *scales,
                          uint32_t b, uint32_t g, const uint16_t *table, uint64_t seed,
                          uint32_t round, uint32_t worker, uint8_t *z)
+{
+    thc_oracle_quantize_at(r, d_pad, k, scales, b, g, table, seed, round, worker, 0, z);
+}
+
+/* Slice form: r[0] is padded coordinate j_base (a multiple of B); scales[0] is its block. */
+void thc_oracle_quantize_at(const float *r, uint64_t d_pad, uint32_t k, const float *scales,
+                            uint32_t b, uint32_t g, const uint16_t *table, uint64_t seed,
+                            uint32_t round, uint32_t worker, uint64_t j_base, uint8_t *z)
 {
     uint64_t B = (uint64_t)1 << k;
     uint32_t levels = 1u << b;
@@ -233,7 +265,7 @@ void thc_oracle_quantize(const float *r, uint64_t d_pad, uint32_t k, const float
         float delta = fmaf(pos, (float)g, -(float)table[z0]);
         float tau = fmaf(delta, r16, 8388608.0f);                         /* RN to integer */
         uint32_t threshold = (uint32_t)(tau - 8388608.0f);
-        uint32_t u = thc_oracle_u16(seed, round, worker, j);
+        uint32_t u = thc_oracle_u16(seed, round, worker, j_base + j);
         z[j] = (uint8_t)(z0 + (u < threshold ? 1u : 0u));
     }
 }

@@ -229,3 +229,44 @@ def scaled(w: Workload, d: int, n: int | None = None, log2_block: int | None = N
     from dataclasses import replace
     return replace(w, d=d, n=w.n if n is None else n,
                    log2_block=w.log2_block if log2_block is None else log2_block)
+
+
+# --------------------------------------------------------------------------------------
+# Large workloads, generated in place on the GPU (the NumPy recipes above take minutes for
+# 10^9..10^10 samples).  Same sizes and distributions, seeded torch generators; used by the
+# full-size parity tests and by bench.py for every configuration but the default one.
+# --------------------------------------------------------------------------------------
+def fill_torch(w: Workload, grads, seed_offset: int = 0) -> None:
+    """Fill the n device tensors in `grads` (fp32 or bf16, d elements each) in place."""
+    import torch
+    dev = grads[0].device
+    chunk = 1 << 26
+    for i, g in enumerate(grads):
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(w.data_seed * 1000 + i + seed_offset)
+        for lo in range(0, w.d, chunk):
+            hi = min(w.d, lo + chunk)
+            m = hi - lo
+            if w.name.startswith("cfg3"):
+                u = torch.rand(m, generator=gen, device=dev, dtype=torch.float32) - 0.5
+                a = u.abs().clamp_(max=0.49999997)                              # keep log finite
+                x = -5e-4 * torch.sign(u) * torch.log1p(-2.0 * a)               # Laplace(0, 5e-4)
+            elif w.name.startswith("cfg4"):
+                z = torch.randn(m, generator=gen, device=dev, dtype=torch.float32)
+                chi2 = sum(torch.randn(m, generator=gen, device=dev, dtype=torch.float32) ** 2
+                           for _ in range(3))
+                x = 1e-4 * z / torch.sqrt(chi2 / 3.0)                            # Student-t(3) * 1e-4
+            elif w.name.startswith("cfg2"):
+                x = torch.randn(m, generator=gen, device=dev, dtype=torch.float32)
+                sizes, scales = resnet50_like_segments(w.d, w.data_seed)
+                per = torch.repeat_interleave(
+                    torch.as_tensor(scales, dtype=torch.float32, device=dev),
+                    torch.as_tensor(sizes, device=dev))[lo:hi]
+                x = x * per
+            elif w.name.startswith("cfg1"):
+                x = torch.randn(m, generator=gen, device=dev, dtype=torch.float32) * 1e-3
+                out_mask = torch.rand(m, generator=gen, device=dev) < 1e-3
+                x = torch.where(out_mask, torch.randn(m, generator=gen, device=dev) * 1e-1, x)
+            else:
+                x = torch.randn(m, generator=gen, device=dev, dtype=torch.float32)
+            g[lo:hi].copy_(x.to(g.dtype))

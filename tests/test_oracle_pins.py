@@ -516,3 +516,25 @@ def test_nonfinite_norm_of_any_worker_makes_the_block_degenerate():
     x = np.ones((3, 32), dtype=np.float32)
     x[1, 16:] = 0
     assert np.all(O.scales(x, c) > 0)
+
+
+def test_slice_forms_agree_with_the_whole_vector():
+    """Transforming / quantising one block of a long vector with its coordinate offset gives
+    the same result as processing the whole vector (blocks are independent; only the sign
+    diagonal and the rounding variates depend on the global coordinate)."""
+    k, d = 6, 64 * 5 - 7
+    c = cfg(k=k)
+    x = np.random.default_rng(17).standard_normal((2, d)).astype(np.float32)
+    scl = O.scales(x, c)
+    whole = O.rht_forward(x[1], c, 3)
+    zw = O.quantize(whole, scl, c, 3, worker=1)
+    vals = np.random.default_rng(18).standard_normal(c.d_pad(d)).astype(np.float32)
+    inv_whole = O.rht_inverse(vals, d, c, 3)
+    for blk in (0, 2, 4):
+        lo, hi = 64 * blk, min(d, 64 * blk + 64)
+        part = O.rht_forward(x[1, lo:hi], c, 3, j_base=lo)
+        assert np.array_equal(part.view(np.uint32), whole[lo:lo + 64].view(np.uint32))
+        zp = O.quantize(part, scl[blk:blk + 1], c, 3, worker=1, j_base=lo)
+        assert np.array_equal(zp, zw[lo:lo + 64])
+        ip = O.rht_inverse(vals[lo:lo + 64], hi - lo, c, 3, j_base=lo)
+        assert np.array_equal(ip.view(np.uint32), inv_whole[lo:hi].view(np.uint32))
