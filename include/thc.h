@@ -152,6 +152,29 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
                    const float *scales, float *out, void *workspace, uint64_t workspace_bytes,
                    void *stream);
 
+/* Preliminary stage without any allocation, for callers that may not call cudaMalloc (a
+ * plugin inside a host framework's fixed memory plan, code running under a frozen memory
+ * budget) and so can use neither thc_create (which allocates the context's device block)
+ * nor a workspace of their own.  The paper has no counterpart of this entry point: it is
+ * thc_prepare with the parameters passed as plain arguments and the fp64 partial sums kept
+ * in a fixed array inside the library's device image (THC_NOALLOC_SCRATCH_BYTES on every
+ * GPU that loads the library, until the process exits).
+ *   grads            host array of n device pointers (16-byte aligned), d elements each
+ *   log2_block, in_dtype, t_p   as in thc_config
+ *   scales           device, ceil(d / 2^log2_block) fp32, written; same values as thc_prepare
+ *   status_or_null   device word that THC_STATUS_NONFINITE / THC_STATUS_ZERO_BLOCK are OR-ed
+ *                    into, or NULL
+ * Limit: n * ceil(d_pad / 2^min(log2_block,14)) partial sums must fit the array (524,288
+ * of them), else THC_EWORKSPACE is returned and nothing is launched.  Calls cudaMalloc,
+ * cudaFree or any allocating routine never.  The first call on a device looks up the
+ * array's device address (cudaGetSymbolAddress); make that call before any stream capture.
+ * All calls share the array: calls that overlap on the GPU race; calls on one stream do
+ * not.  Nothing in the array has to be cleared between calls. */
+#define THC_NOALLOC_SCRATCH_BYTES (4u << 20)
+int thc_prepare_noalloc(const void *const *grads, uint32_t n, uint64_t d, uint32_t log2_block,
+                        uint32_t in_dtype, double t_p, float *scales, uint32_t *status_or_null,
+                        void *stream);
+
 /* Read and clear the status bits (synchronises `stream`).  flags is a host pointer. */
 int thc_status(thc_ctx *ctx, uint32_t *flags, void *stream);
 

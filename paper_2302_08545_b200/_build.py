@@ -14,7 +14,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libthc.so")
-SOURCES = ["thc.cu"]
+SOURCES = ["thc.cu", "thc_noalloc.cu"]
 HEADERS = ["thc_device.cuh", "thc_pipeline.cuh", os.path.join("..", "..", "include", "thc.h")]
 
 NVCC_FLAGS = [

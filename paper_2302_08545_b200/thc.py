@@ -20,8 +20,9 @@ THC_MAX_WORKERS = 64
 STATUS_NONFINITE, STATUS_ZERO_BLOCK, STATUS_WAIT_TIMEOUT = 1, 2, 4
 
 EXPORTS = ("thc_create", "thc_destroy", "thc_sizes", "thc_prepare", "thc_compress",
-           "thc_quantize_rotated", "thc_aggregate", "thc_decompress", "thc_status",
-           "thc_strerror", "thc_version")
+           "thc_quantize_rotated", "thc_aggregate", "thc_decompress", "thc_prepare_noalloc",
+           "thc_status", "thc_strerror", "thc_version")
+NOALLOC_SCRATCH_BYTES = 4 << 20
 
 
 class ThcError(RuntimeError):
@@ -75,6 +76,7 @@ def lib():
     L.thc_quantize_rotated.argtypes = [vp, pp, u32, u32, u64, u32, vp, pp, vp]
     L.thc_aggregate.argtypes = [vp, pp, u32, u64, vp, vp]
     L.thc_decompress.argtypes = [vp, vp, u32, u64, u32, vp, vp, vp, u64, vp]
+    L.thc_prepare_noalloc.argtypes = [pp, u32, u64, u32, u32, ctypes.c_double, vp, vp, vp]
     L.thc_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
     for name in EXPORTS[:-2]:
         getattr(L, name).restype = ctypes.c_int
@@ -120,6 +122,19 @@ def _stream(stream) -> int:
     if isinstance(stream, int):
         return stream
     return stream.cuda_stream
+
+
+def prepare_noalloc(grads, d: int, log2_block: int, in_dtype: int, t_p: float, scales,
+                    status=None, stream=None):
+    """thc_prepare_noalloc: the preliminary stage for callers that may not allocate device
+    memory.  No context and no workspace: the scratch is a fixed array inside the library
+    (NOALLOC_SCRATCH_BYTES per GPU).  `status` is an optional device uint32 tensor the status
+    bits are OR-ed into.  Raises ThcError(THC_EWORKSPACE) when the input is too large for
+    the built-in scratch."""
+    arr = _ptr_array([_dp(g) for g in grads])
+    _check(lib().thc_prepare_noalloc(arr, len(grads), d, log2_block, in_dtype, float(t_p),
+                                     _dp(scales), _dp(status), _stream(stream)),
+           "thc_prepare_noalloc")
 
 
 class Context:
