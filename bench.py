@@ -355,6 +355,60 @@ def run_gpu(args):
     return 0
 
 
+def run_sweep(args):
+    """Configuration 5: d x b x n sweep (B = 2^20).  One JSON line per point with the round's
+    algorithmic GB/s and its fraction of the measured HBM copy rate; the last line is a
+    summary.  Inputs are generated on the device (seeded) and exceed L2 from d = 2^24 up."""
+    import torch
+    from paper_2302_08545_b200 import runner, thc
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    thc.lib()
+    peak, peak_src = measured_peaks()
+    stream = torch.cuda.current_stream()
+    results = []
+    for w in W.sweep_points():
+        ctx = runner.context_for(w)
+        r = runner.Round(ctx, w.n, w.d, w.in_dtype)
+        W.fill_torch(w, r.grads)
+        r.prepare()
+        calls = [("compress", lambda: r.compress(0)), ("aggregate", r.aggregate),
+                 ("decompress", lambda: r.decompress(0))]
+        for _ in range(3):
+            for _, fn in calls:
+                fn()
+        torch.cuda.synchronize()
+        per = {}
+        for name, fn in calls:
+            evs = []
+            for _ in range(args.sweep_steps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                evs.append((a, b))
+            torch.cuda.synchronize()
+            ts = sorted(a.elapsed_time(b) for a, b in evs)
+            per[name] = ts[len(ts) // 2]
+        ab = w.algorithmic_bytes()
+        round_ms = sum(per.values())
+        line = {"workload": w.name, "d": w.d, "bits": w.bits, "n": w.n, "acc_bits": w.acc_bits,
+                "round_ms": round_ms, "per_call_ms": per,
+                "gradient_gbs": w.n * w.d * 4 / (round_ms * 1e-3) / 1e9,
+                "algorithmic_gbs": ab["round"] / (round_ms * 1e-3) / 1e9,
+                "frac_of_measured_hbm": ab["round"] / (round_ms * 1e-3) / 1e9 / peak,
+                "status_flags": ctx.status()}
+        print(json.dumps(line), flush=True)
+        results.append(line)
+        del r, ctx
+        torch.cuda.empty_cache()
+    fr = [x["frac_of_measured_hbm"] for x in results]
+    print(json.dumps({"sweep_points": len(results), "peak": peak, "peak_source": peak_src,
+                      "frac_min": min(fr), "frac_median": sorted(fr)[len(fr) // 2],
+                      "frac_max": max(fr)}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -363,9 +417,13 @@ def main():
     ap.add_argument("--impl", default="thc", choices=["thc", "reference"])
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="run the d x b x n sweep (configuration 5)")
+    ap.add_argument("--sweep-steps", type=int, default=5)
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.sweep:
+        return run_sweep(args)
     return run_gpu(args)
 
 
