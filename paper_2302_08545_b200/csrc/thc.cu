@@ -879,7 +879,7 @@ static void geom_pass_a(TileGeom &g)
 }
 
 // ---- persistent pipeline dispatch (RHT blocks of 2^15 .. 2^24 coordinates)
-typedef void (*pipe_kernel_t)(PipeParams, PtrArrayP, MutPtrArrayP, MutPtrArrayP, PhiloxKeys);
+typedef void (*pipe_kernel_t)(const TmaMaps, PipeParams, PtrArrayP, MutPtrArrayP, MutPtrArrayP, PhiloxKeys);
 
 template <int MODE, int KB>
 static pipe_kernel_t pick_pipe_kernel_kb(uint32_t bits, bool identity)
@@ -904,8 +904,44 @@ static pipe_kernel_t pick_pipe_kernel(uint32_t bits, bool identity, uint32_t k)
                    : pick_pipe_kernel_kb<MODE, 0>(bits, identity);
 }
 
-static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, const thc_sizes_t &sz, uint64_t d,
-                           uint32_t n_local, uint32_t worker_base, uint32_t round, uint32_t divisor,
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda).
+typedef CUresult (*encode_tiled_t)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static encode_tiled_t get_encode_tiled()
+{
+    static encode_tiled_t fn = nullptr;
+    if (fn == nullptr) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<encode_tiled_t>(p);
+    }
+    return fn;
+}
+
+// A 2-D map over `rows` rows of `cols` 32-bit words (row pitch in bytes), box 32 x box_rows,
+// 128-byte swizzle.  The data type is UINT32 so that bits travel unchanged.
+static int encode_map(CUtensorMap *map, const void *base, uint64_t cols, uint64_t rows,
+                      uint64_t pitch_bytes, uint32_t box_rows)
+{
+    encode_tiled_t enc = get_encode_tiled();
+    if (enc == nullptr) return THC_ECUDA;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {pitch_bytes};
+    const cuuint32_t box[2] = {32u, box_rows};
+    const cuuint32_t estr[2] = {1u, 1u};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(base), dims, strides,
+                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? THC_OK : THC_ECUDA;
+}
+
+static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress_f32,
+                           const thc_sizes_t &sz, uint64_t d, uint32_t n_local, uint32_t worker_base, uint32_t round, uint32_t divisor,
                            const float *scales, void *workspace, const PtrArrayP &in,
                            const MutPtrArrayP &out, const MutPtrArrayP &rot, cudaStream_t st)
 {
@@ -933,10 +969,26 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, const thc_siz
     P.worker_base = worker_base;
     P.c_block = (float)(1.0 / sqrt((double)(1ull << k)));
     const uint64_t nblk_cached = sz.nblocks < (uint64_t)kBlockConstMax ? sz.nblocks : (uint64_t)kBlockConstMax;
-    const size_t smem = (size_t)2 * kPElems * 4 + kPSignWords * 4 +
+    const size_t smem = (size_t)1024 + (size_t)2 * kPElems * 4 + kPSignWords * 4 +
                         (size_t)(ctx->cfg.granularity + 1) * kLutRep * 16 + (size_t)nblk_cached * 8;
     { const int rc = ensure_dynamic_smem(reinterpret_cast<const void *>(kern), smem); if (rc != THC_OK) return rc; }
-    kern<<<pl.grid, kPCtaThreads, smem, st>>>(P, in, out, rot, ctx->keys);
+    // Tensor maps: the ring (k = 20 panels are fetched by TMA) and, for fp32 compress, every
+    // worker's gradient viewed as rows of 32 floats (whole rows only; a ragged last tile is
+    // loaded by the compute warps).
+    TmaMaps maps;
+    memset(&maps, 0, sizeof maps);
+    if (k == 20) {
+        const int rc = encode_map(&maps.ring, workspace, (uint64_t)kPElems,
+                                  (uint64_t)pl.ring << (k - kPLog2), (uint64_t)kPElems * 4, 128u);
+        if (rc != THC_OK) return rc;
+    }
+    if (compress_f32 && (d >> 5) >= 256) {
+        for (uint32_t i = 0; i < n_local; ++i) {
+            const int rc = encode_map(&maps.in[i], in.p[i], 32u, d >> 5, 128u, 256u);
+            if (rc != THC_OK) return rc;
+        }
+    }
+    kern<<<pl.grid, kPCtaThreads, smem, st>>>(maps, P, in, out, rot, ctx->keys);
     THC_CUDA(cudaGetLastError());
     return THC_OK;
 }
@@ -992,8 +1044,8 @@ int thc_compress(thc_ctx *ctx, const void *const *grads, uint32_t n_local, uint3
     memcpy(&prot, &rot, sizeof prot);
     pipe_kernel_t kern = bf16 ? pick_pipe_kernel<kCompressBF16>(ctx->cfg.bits, ctx->identity, k)
                               : pick_pipe_kernel<kCompressF32>(ctx->cfg.bits, ctx->identity, k);
-    return launch_pipeline(ctx, kern, sz, d, n_local, worker_base, round, 1, scales, workspace, pin,
-                           pout, prot, st);
+    return launch_pipeline(ctx, kern, !bf16, sz, d, n_local, worker_base, round, 1, scales, workspace,
+                           pin, pout, prot, st);
 }
 
 int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, uint32_t round,
@@ -1042,7 +1094,8 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
     pipe_kernel_t kern = w == 8 ? pick_pipe_kernel<kDecompress8>(4, true, k)
                        : w == 16 ? pick_pipe_kernel<kDecompress16>(4, true, k)
                                  : pick_pipe_kernel<kDecompress32>(4, true, k);
-    return launch_pipeline(ctx, kern, sz, d, 1, 0, round, divisor, scales, workspace, pin, pout, prot, st);
+    return launch_pipeline(ctx, kern, false, sz, d, 1, 0, round, divisor, scales, workspace, pin, pout,
+                           prot, st);
 }
 
 int thc_quantize_rotated(thc_ctx *ctx, const float *const *rotated, uint32_t n_local,

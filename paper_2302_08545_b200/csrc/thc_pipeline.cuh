@@ -14,14 +14,19 @@
 // on expiry the kernel sets THC_STATUS_WAIT_TIMEOUT, raises an abort flag that ends all CTAs,
 // and returns.
 //
-// Each CTA keeps two tile buffers: while it computes task i from one, the tile of task i+1
-// (claimed one task ahead, dependency polled early) streams into the other with cp.async.
+// Each CTA is four compute warps and one control warp, a producer/consumer pair over two tile
+// buffers.  The control warp claims the next task, waits for its dependency, computes the
+// tile's sign words, starts the TMA load of its tile into the free buffer (completion on an
+// mbarrier) and hands the descriptor over through a full/empty named-barrier handshake; the
+// compute warps wait for the data, run the rounds and signal completion.  Tiles sit in shared
+// memory in TMA's 128-byte swizzle: 16-byte chunk c at c ^ ((c >> 3) & 7).
 //
 // Counters (in the context's device block, all zero between launches; the last CTA to leave
 // clears them):  head, exited, abort, a_done[R], b_done[R].  a_done[s] counts finished A tiles
 // of slot s over the whole launch (generation g of the slot is complete at (g+1)*T),
 // b_done[s] finished B panels (slot may be overwritten by generation g once it reaches g*T).
 #pragma once
+#include <cuda.h>
 #include "thc_device.cuh"
 
 namespace thc {
@@ -31,7 +36,7 @@ constexpr int kPElems = 1 << kPLog2;
 constexpr int kPChunks = kPElems / 4;
 constexpr int kPThreads = 128;                // compute threads of a CTA
 constexpr int kPCtaThreads = 160;             // plus one control warp that runs the queue
-constexpr int kPSignWords = 512;            // sign words a tile can need
+constexpr int kPSignWords = 512;            // sign words: two slots of 256 (pass A) or one of 512
 constexpr int kMaxRing = 56;
 constexpr int kBlockConstMax = 256;         // per-block constants cached in shared memory
 constexpr uint32_t kMaxPolls = 1u << 21;
@@ -77,8 +82,13 @@ struct TaskInfo {              // published by thread 0 for the whole CTA
     uint32_t r;                // RHT block
     uint32_t slot;             // ring slot
     uint32_t gen;              // generation of the slot
-    uint32_t loaded;           // dependency satisfied: its tile load may be / has been issued
-    uint32_t pad;
+    uint32_t tma;              // tile arrives by TMA on the slot's mbarrier
+    uint32_t phase;            // ... with this phase parity
+};
+
+struct TmaMaps {               // tensor maps: one per worker gradient, one for the ring
+    CUtensorMap in[THC_MAX_WORKERS];
+    CUtensorMap ring;
 };
 
 // ------------------------------------------------------------------------ small helpers
@@ -162,6 +172,62 @@ __device__ __forceinline__ void red_release_add(uint32_t *p, uint32_t v)
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
 }
 
+// ------------------------------------------------------------------ mbarrier / TMA
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(a), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(a), "r"(bytes) : "memory");
+}
+
+// Bounded wait for a phase of the mbarrier; false if it did not complete.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+{
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(a), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// One 2-D tile: box of the tensor map at element coordinates (x, y) -> shared memory.
+__device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *map, int x, int y,
+                                            uint64_t *bar, uint64_t policy)
+{
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(bar);
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+                 ".L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+                 :: "r"(d), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(b), "l"(policy)
+                 : "memory");
+}
+
+// Orders this thread's earlier generic-proxy accesses to shared memory before later
+// async-proxy (TMA) writes to it.
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ uint64_t make_evict_normal_policy()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+__device__ __forceinline__ int pswz(int c) { return c ^ ((c >> 3) & 7); }
+
 // Lane <-> unit permutation (swap bits 2 and 3): makes pairs of adjacent chunks per lane
 // conflict-free in the XOR-swizzled tile.
 __device__ __forceinline__ int swap_bits_2_3(int t)
@@ -227,7 +293,7 @@ __device__ __forceinline__ void p_round(float4 *tile, int sp, int tid)
         const int base = ((G >> sp) << (sp + E)) | low;
         float4 v[N];
 #pragma unroll
-        for (int m = 0; m < N; ++m) v[m] = tile[swz(base + (m << sp))];
+        for (int m = 0; m < N; ++m) v[m] = tile[pswz(base + (m << sp))];
 #pragma unroll
         for (int t = 0; t < E; ++t) {
 #pragma unroll
@@ -235,7 +301,7 @@ __device__ __forceinline__ void p_round(float4 *tile, int sp, int tid)
                 if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
         }
 #pragma unroll
-        for (int m = 0; m < N; ++m) tile[swz(base + (m << sp))] = v[m];
+        for (int m = 0; m < N; ++m) tile[pswz(base + (m << sp))] = v[m];
     }
 }
 
@@ -256,48 +322,58 @@ __device__ __forceinline__ void p_rounds(float4 *tile, int lo, int hi, int tid)
 }
 
 // ------------------------------------------------------------------------------- pass A
+// A tile is 256 rows of 8 chunks (32 coordinates); row r, chunk cc sits at r*8 + (cc ^ (r&7)).
+//
 // First round, in place: sign flip (compress), stages of stride 1 and 2 inside each chunk,
-// then stride 4 .. 32 across the thread's 16 consecutive chunks.  Chunk 16*tid + m lives at
-// 16*tid + (m ^ (tid & 7)).
+// then stride 4, 8, 16 across the eight chunks of a row.  Thread t owns rows t and t + 128.
 template <bool FLIP>
 __device__ __forceinline__ void pass_a_round1(float4 *tile, const uint32_t *sw, int tid)
 {
-    float4 *mine = tile + tid * 16;
     const int x = tid & 7;
     float4 v[16];
 #pragma unroll
-    for (int m = 0; m < 16; ++m) v[m] = mine[m ^ x];
-    if (FLIP) {
-        const uint2 w = *reinterpret_cast<const uint2 *>(sw + 2 * tid);
+    for (int g = 0; g < 2; ++g) {
+        float4 *row = tile + (tid + 128 * g) * 8;
 #pragma unroll
-        for (int m = 0; m < 16; ++m)
-            v[m] = flip4(v[m], (m < 8 ? w.x : w.y) >> ((m & 7) * 4));
+        for (int m = 0; m < 8; ++m) v[8 * g + m] = row[m ^ x];
+    }
+    if (FLIP) {
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            const uint32_t w = sw[tid + 128 * g];
+#pragma unroll
+            for (int m = 0; m < 8; ++m) v[8 * g + m] = flip4(v[8 * g + m], w >> (m * 4));
+        }
     }
 #pragma unroll
     for (int m = 0; m < 16; ++m) v[m] = stages01(v[m]);
 #pragma unroll
-    for (int t = 0; t < 4; ++t) {
+    for (int t = 0; t < 3; ++t) {
 #pragma unroll
         for (int m = 0; m < 16; ++m)
             if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
     }
 #pragma unroll
-    for (int m = 0; m < 16; ++m) mine[m ^ x] = v[m];
+    for (int g = 0; g < 2; ++g) {
+        float4 *row = tile + (tid + 128 * g) * 8;
+#pragma unroll
+        for (int m = 0; m < 8; ++m) row[m ^ x] = v[8 * g + m];
+    }
 }
 
-// Round on chunk bits 4..7 (also the first pass-B round when a row has 16 chunks): thread
-// tid owns chunks hi*256 + 16*m + low (low = tid & 15, hi = tid >> 4), stored with the low
-// three bits XORed by m & 7.
-__device__ __forceinline__ void round_bits_4_7(float4 *tile, int tid)
+// Round on row bits 0..3: thread (rg = tid >> 3, cc = tid & 7) owns chunk cc of rows
+// 16 rg + m.  Serves pass A (second round) and the first round of a k = 20 pass-B tile, whose
+// two 128-row halves are simply rows 0..255.
+__device__ __forceinline__ void round_rows_0_3(float4 *tile, int tid)
 {
-    float4 *mine = tile + ((tid >> 4) << 8);
-    const int low = tid & 15;
+    float4 *mine = tile + ((tid >> 3) << 7);
+    const int cc = tid & 7;
     float4 *q[8];
 #pragma unroll
-    for (int x = 0; x < 8; ++x) q[x] = mine + (low ^ x);
+    for (int x = 0; x < 8; ++x) q[x] = mine + (cc ^ x);
     float4 v[16];
 #pragma unroll
-    for (int m = 0; m < 16; ++m) v[m] = q[m & 7][16 * m];
+    for (int m = 0; m < 16; ++m) v[m] = q[m & 7][8 * m];
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
 #pragma unroll
@@ -305,29 +381,27 @@ __device__ __forceinline__ void round_bits_4_7(float4 *tile, int tid)
             if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
     }
 #pragma unroll
-    for (int m = 0; m < 16; ++m) q[m & 7][16 * m] = v[m];
+    for (int m = 0; m < 16; ++m) q[m & 7][8 * m] = v[m];
 }
 
-// Last round of a pass-A tile (chunk bits 8..10) with the result stored straight to the ring.
+// Last round of a pass-A tile (row bits 4..7): thread (rl = tid >> 3, cc = tid & 7) owns chunk
+// cc of rows rl + 16 m; the result goes straight to the ring, 512 contiguous bytes per warp.
 __device__ __forceinline__ void pass_a_round3_store(const float4 *tile, float *dst, int tid)
 {
+    const int rl = tid >> 3, cc = tid & 7;
+    const float4 *mine = tile + rl * 8 + (cc ^ (rl & 7));
+    float4 v[16];
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int low = tid + i * kPThreads;
-        const float4 *mine = tile + (low ^ ((low >> 4) & 7));
-        float4 v[8];
+    for (int m = 0; m < 16; ++m) v[m] = mine[m << 7];
 #pragma unroll
-        for (int m = 0; m < 8; ++m) v[m] = mine[m << 8];
+    for (int t = 0; t < 4; ++t) {
 #pragma unroll
-        for (int t = 0; t < 3; ++t) {
-#pragma unroll
-            for (int m = 0; m < 8; ++m)
-                if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
-        }
-        float4 *out = reinterpret_cast<float4 *>(dst) + low;
-#pragma unroll
-        for (int m = 0; m < 8; ++m) out[m << 8] = v[m];
+        for (int m = 0; m < 16; ++m)
+            if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
     }
+    float4 *out = reinterpret_cast<float4 *>(dst) + tid;
+#pragma unroll
+    for (int m = 0; m < 16; ++m) out[m << 7] = v[m];
 }
 
 // ------------------------------------------------------------------------------- pass B
@@ -400,8 +474,8 @@ __device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, in
 #pragma unroll
         for (int m = 0; m < N; ++m) {
             const int c = ((row_low + (m << rl)) << ccl) + 2 * uu;
-            a[m] = tile[swz(c)];
-            b[m] = tile[swz(c + 1)];
+            a[m] = tile[pswz(c)];
+            b[m] = tile[pswz(c + 1)];
         }
 #pragma unroll
         for (int t = 0; t < E; ++t) {
@@ -421,21 +495,24 @@ __device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, in
     }
 }
 
-// The same for the 128-row x 16-chunk tile (k = 20): rows row_low + 16 m, m = 0..7; lanes
-// 0-7 of a quarter warp cover four units of two adjacent rows, which is conflict-free.
+// The same for the k = 20 tile: two halves (columns 0-31, 32-63) of 128 rows x 8 chunks.
+// Thread (u = tid & 3, rl from bits 2..5, h = tid >> 6) owns unit 4h + u of rows rl + 16 m,
+// m = 0..7; lanes 0-7 of a quarter warp cover four units of two adjacent rows, whose XOR
+// patterns differ in bit 0, so both chunk reads are conflict-free.
 template <bool COMPRESS, int BITS, bool IDENTITY>
 __device__ __forceinline__ void pass_b_last_round_kb7(float4 *tile, int tid,
                                                       const EpilogueCtx &ep, const PhiloxKeys &keys)
 {
-    const int uu = (tid & 3) | ((tid >> 1) & 4);
-    const int row_low = ((tid >> 2) & 1) | ((tid >> 4) << 1);
-    const int x = row_low & 7;
-    float4 *pa = tile + row_low * 16 + ((2 * uu) ^ x);
-    float4 *pb = tile + row_low * 16 + ((2 * uu + 1) ^ x);
+    const int u = tid & 3;
+    const int rl = ((tid >> 2) & 1) | (((tid >> 3) & 7) << 1);
+    const int h = tid >> 6;
+    const int x = rl & 7;
+    float4 *pa = tile + (h * 128 + rl) * 8 + ((2 * u) ^ x);
+    float4 *pb = tile + (h * 128 + rl) * 8 + ((2 * u + 1) ^ x);
     {
         float4 a[8], b[8];
 #pragma unroll
-        for (int m = 0; m < 8; ++m) { a[m] = pa[m << 8]; b[m] = pb[m << 8]; }
+        for (int m = 0; m < 8; ++m) { a[m] = pa[m << 7]; b[m] = pb[m << 7]; }
 #pragma unroll
         for (int t = 0; t < 3; ++t) {
 #pragma unroll
@@ -447,25 +524,29 @@ __device__ __forceinline__ void pass_b_last_round_kb7(float4 *tile, int tid,
         }
         // back to the thread's own slots: the epilogue below is a compact loop (code size)
 #pragma unroll
-        for (int m = 0; m < 8; ++m) { pa[m << 8] = a[m]; pb[m << 8] = b[m]; }
+        for (int m = 0; m < 8; ++m) { pa[m << 7] = a[m]; pb[m << 7] = b[m]; }
     }
-    const uint64_t j0 = ep.j_tile + ((uint64_t)row_low << kPLog2) + 8 * uu;
+    const int uu = 4 * h + u;
+    const uint64_t j0 = ep.j_tile + ((uint64_t)rl << kPLog2) + 8 * uu;
 #pragma unroll 2
     for (int m = 0; m < 8; ++m)
-        epilogue_unit<COMPRESS, BITS, IDENTITY>(pa[m << 8], pb[m << 8], j0 + ((uint64_t)m << (kPLog2 + 4)),
-                                                row_low + 16 * m, uu, ep, keys);
+        epilogue_unit<COMPRESS, BITS, IDENTITY>(pa[m << 7], pb[m << 7], j0 + ((uint64_t)m << (kPLog2 + 4)),
+                                                rl + 16 * m, uu, ep, keys);
 }
 
 // ------------------------------------------------------------------------------ the kernel
 // KB = 7 specialises the k = 20 geometry at compile time; KB = 0 reads it from the params.
 template <int MODE, int BITS, bool IDENTITY, int KB>
 __global__ void __launch_bounds__(kPCtaThreads, 3)
-thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP rotated,
-                    PhiloxKeys keys)
+thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArrayP in,
+                    MutPtrArrayP outp, MutPtrArrayP rotated, PhiloxKeys keys)
 {
     constexpr bool kCompress = MODE == kCompressF32 || MODE == kCompressBF16;
-    constexpr bool kAsyncA = MODE == kCompressF32;
-    extern __shared__ __align__(1024) unsigned char pipe_smem[];
+    extern __shared__ __align__(1024) unsigned char pipe_smem_raw[];
+    // TMA's 128-byte swizzle needs the tile buffers on 1024-byte boundaries of the shared
+    // address space; the launch reserves 1 KB of slack for this round-up.
+    unsigned char *pipe_smem = pipe_smem_raw +
+        ((1024u - ((uint32_t)__cvta_generic_to_shared(pipe_smem_raw) & 1023u)) & 1023u);
     float4 *bufs[2] = {reinterpret_cast<float4 *>(pipe_smem),
                        reinterpret_cast<float4 *>(pipe_smem + kPElems * 4)};
     uint32_t *sw = reinterpret_cast<uint32_t *>(pipe_smem + 2 * kPElems * 4);
@@ -473,72 +554,131 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
     float2 *blk_const = reinterpret_cast<float2 *>(pipe_smem + 2 * kPElems * 4 + kPSignWords * 4 +
                                                    (size_t)(P.granularity + 1) * kLutRep * 16);
     __shared__ TaskInfo s_info[2];
-    __shared__ uint32_t s_published;       // tasks the control warp has handed over so far
+    __shared__ __align__(8) uint64_t s_mbar[2];
 
     const int tid = threadIdx.x;
-    if (tid == 0) s_published = 0;
     PipeCounters *pc = reinterpret_cast<PipeCounters *>(P.dev->counters);
     const int kb = KB ? KB : (int)P.kb;
     const uint32_t T = 1u << kb;                      // tiles (= panels) per worker-block
     const uint64_t B = 1ull << P.k;
     const int ccl = 11 - kb;                          // log2 chunks per pass-B row
-    const uint64_t policy = make_evict_first_policy();
+    const uint64_t d_rows32 = P.d >> 5;               // whole 32-coordinate rows of a gradient
 
+    if (tid == 0) {
+        mbar_init(&s_mbar[0], 1);
+        mbar_init(&s_mbar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     if (kCompress && !IDENTITY) {
-        for (int idx = tid; idx < (int)(P.granularity + 1) * kLutRep; idx += kPThreads)
+        for (int idx = tid; idx < (int)(P.granularity + 1) * kLutRep; idx += kPCtaThreads)
             lut[idx] = P.dev->lut[idx / kLutRep];
     }
     const uint32_t nblk_total = (uint32_t)(P.d_pad >> P.k);
     const uint32_t nblk_cached = nblk_total < (uint32_t)kBlockConstMax ? nblk_total : (uint32_t)kBlockConstMax;
-    for (uint32_t b = tid; b < nblk_cached; b += kPThreads)
+    for (uint32_t b = tid; b < nblk_cached; b += kPCtaThreads)
         blk_const[b] = block_constants<kCompress>(P.scales[b], P.granularity, P.divisor);
     __syncthreads();
 
-    // ---- issue the tile load of a task into a buffer (all threads)
-    auto issue_load = [&](const TaskInfo &ti, float4 *tile) {
-        const bool is_b = ti.is_b != 0;
-        const uint32_t wl = ti.wl;
-        const uint64_t r = ti.r;
-        const uint32_t slot = ti.slot;
-        if (is_b) {
-            // panel idx: rows 2^13 apart in the ring slot, 2^(13-kb) columns each
-            const float *src = P.ring + (size_t)slot * B + ((size_t)ti.idx << (kPLog2 - kb));
-            if (KB == 7) {
-                // chunk tid + 128 i is (row (tid >> 4) + 8 i, column chunk tid & 15)
-                const float *xs = src + ((size_t)(tid >> 4) << kPLog2) + 4 * (tid & 15);
-                float4 *dst = tile + (tid ^ ((tid >> 4) & 7));
-#pragma unroll
-                for (int i = 0; i < kPChunks / kPThreads; ++i)
-                    cp_async16(dst + i * kPThreads, xs + ((size_t)i << (kPLog2 + 3)));
-            } else
-#pragma unroll 4
-            for (int i = 0; i < kPChunks / kPThreads; ++i) {
-                const int c = tid + i * kPThreads;
-                const int row = c >> ccl, cc = c & ((1 << ccl) - 1);
-                cp_async16(&tile[swz(c)], src + ((size_t)row << kPLog2) + 4 * cc);
-            }
-        } else {
-            const uint64_t j0 = r * B + ((uint64_t)ti.idx << kPLog2);
-            if (kAsyncA) {
-                const float *x = static_cast<const float *>(in.p[wl]);
-                if (j0 + kPElems <= P.d) {
-                    const float *xs = x + j0 + 4 * tid;
-                    float4 *dst = tile + (tid ^ ((tid >> 4) & 7));
-#pragma unroll
-                    for (int i = 0; i < kPChunks / kPThreads; ++i)
-                        cp_async16_hint(dst + i * kPThreads, xs + 4 * i * kPThreads, 16u, policy);
-                } else {
-#pragma unroll 4
-                    for (int i = 0; i < kPChunks / kPThreads; ++i) {
-                        const int c = tid + i * kPThreads;
-                        const uint64_t j = j0 + 4ull * c;
-                        const uint32_t nbytes = j + 4 <= P.d ? 16u : j < P.d ? (uint32_t)(P.d - j) * 4u : 0u;
-                        cp_async16_hint(&tile[swz(c)], nbytes ? (const void *)(x + j) : (const void *)x,
-                                        nbytes, policy);
+    if (tid >= kPThreads) {
+        // ============================================================ control warp
+        const int lane = tid - kPThreads;
+        const uint64_t pol_stream = make_evict_first_policy();   // gradients: read once
+        const uint64_t pol_ring = make_evict_normal_policy();    // ring: written and read in L2
+        uint32_t uses[2] = {0u, 0u};                  // TMA loads issued per slot so far
+        for (uint32_t i = 0;; ++i) {
+            const int s = (int)(i & 1);
+            // Task i is claimed once the compute warps have picked up task i-1, i.e. have
+            // finished task i-2: buffer s and sign-word slot s are free.  One task of
+            // look-ahead only: a deeper one stretches every task's claim-to-completion time,
+            // which is what dependent tasks wait for.
+            if (i >= 1) bar_sync(3 + (s ^ 1), kPCtaThreads);
+            TaskInfo ti;
+            ti.idx = 0xFFFFFFFFu; ti.is_b = 0; ti.wl = 0; ti.r = 0; ti.slot = 0; ti.gen = 0; ti.tma = 0; ti.phase = 0;
+            if (lane == 0) {
+                const uint32_t q = atomicAdd(&pc->head, 1u);
+                const uint32_t aborted = ld_relaxed_u32(&pc->abort);
+                if ((uint64_t)q < P.total_tasks && aborted == 0) {
+                    const TaskId t = decode_task(q, P);
+                    const uint32_t *ctr = t.is_b ? &pc->a_done[t.slot] : &pc->b_done[t.slot];
+                    const uint32_t target = t.is_b ? (t.gen + 1) * T : t.gen * T;
+                    if (target == 0 || wait_at_least(ctr, target, pc, P.dev)) {
+                        ti.idx = t.idx;
+                        ti.is_b = t.is_b;
+                        ti.r = t.wb / P.n_local;
+                        ti.wl = t.wb - ti.r * P.n_local;
+                        ti.slot = t.slot;
+                        ti.gen = t.gen;
                     }
                 }
+            }
+            const uint32_t idx = __shfl_sync(0xFFFFFFFFu, ti.idx, 0);
+            const uint32_t is_b = __shfl_sync(0xFFFFFFFFu, ti.is_b, 0);
+            const uint32_t r = __shfl_sync(0xFFFFFFFFu, ti.r, 0);
+            if (idx != 0xFFFFFFFFu) {
+                const uint64_t j0 = (uint64_t)r * B + ((uint64_t)idx << kPLog2);
+                if (kCompress && !is_b) {
+                    // sign words of the tile: 64 Philox calls, two per lane
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        const int call = lane + 32 * c;
+                        const uint4 ph = sign_call(j0 + 128ull * call, P.round, keys);
+                        *reinterpret_cast<uint4 *>(sw + 256 * s + 4 * call) = ph;
+                    }
+                }
+                if (lane == 0) {
+                    if (is_b) {
+                        if (KB == 7) {
+                            // panel: 128 ring rows x 64 columns, as two boxes of 32 columns
+                            mbar_expect_tx(&s_mbar[s], kPElems * 4);
+                            const int x0 = (int)(idx << 6);
+                            const int y0 = (int)(ti.slot << 7);
+                            tma_load_2d(bufs[s], &maps.ring, x0, y0, &s_mbar[s], pol_ring);
+                            tma_load_2d(bufs[s] + 1024, &maps.ring, x0 + 32, y0, &s_mbar[s], pol_ring);
+                            ti.tma = 1;
+                        }
+                    } else if (MODE == kCompressF32 && (j0 >> 5) + 256 <= d_rows32) {
+                        mbar_expect_tx(&s_mbar[s], kPElems * 4);
+                        tma_load_2d(bufs[s], &maps.in[ti.wl], 0, (int)(j0 >> 5), &s_mbar[s], pol_stream);
+                        ti.tma = 1;
+                    }
+                    if (ti.tma) { ti.phase = uses[s] & 1u; ++uses[s]; }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) s_info[s] = ti;
+            __syncwarp();
+            bar_arrive(1 + s, kPCtaThreads);                  // slot s is full
+            if (idx == 0xFFFFFFFFu) break;
+        }
+    } else {
+        // ============================================================ compute warps
+        // Loads the control warp could not hand to the TMA unit (ragged last tile, bf16 or
+        // summed inputs, run-time geometry): done here, synchronously.
+        auto load_tile = [&](const TaskInfo &ti, float4 *tile) {
+            const uint64_t policy = make_evict_first_policy();
+            if (ti.is_b) {
+                const float *src = P.ring + (size_t)ti.slot * B + ((size_t)ti.idx << (kPLog2 - kb));
+#pragma unroll 4
+                for (int i = 0; i < kPChunks / kPThreads; ++i) {
+                    const int c = tid + i * kPThreads;
+                    const int row = c >> ccl, cc = c & ((1 << ccl) - 1);
+                    cp_async16(&tile[pswz(c)], src + ((size_t)row << kPLog2) + 4 * cc);
+                }
+                return;
+            }
+            const uint64_t j0 = (uint64_t)ti.r * B + ((uint64_t)ti.idx << kPLog2);
+            if (MODE == kCompressF32) {
+                const float *x = static_cast<const float *>(in.p[ti.wl]);
+#pragma unroll 4
+                for (int i = 0; i < kPChunks / kPThreads; ++i) {
+                    const int c = tid + i * kPThreads;
+                    const uint64_t j = j0 + 4ull * c;
+                    const uint32_t nbytes = j + 4 <= P.d ? 16u : j < P.d ? (uint32_t)(P.d - j) * 4u : 0u;
+                    cp_async16_hint(&tile[pswz(c)], nbytes ? (const void *)(x + j) : (const void *)x,
+                                    nbytes, policy);
+                }
             } else if (MODE == kCompressBF16) {
-                const uint16_t *x = static_cast<const uint16_t *>(in.p[wl]);
+                const uint16_t *x = static_cast<const uint16_t *>(in.p[ti.wl]);
 #pragma unroll 2
                 for (int i = 0; i < kPChunks / 2 / kPThreads; ++i) {
                     const int u = tid + i * kPThreads;
@@ -551,16 +691,16 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
                         for (int e = 0; e < 8; ++e)
                             if (j + e < P.d) w[e >> 1] |= (uint32_t)__ldg(x + j + e) << ((e & 1) * 16);
                     }
-                    tile[swz(2 * u)] = make_float4(__uint_as_float(w[0] << 16), __uint_as_float(w[0] & 0xFFFF0000u),
-                                                   __uint_as_float(w[1] << 16), __uint_as_float(w[1] & 0xFFFF0000u));
-                    tile[swz(2 * u + 1)] = make_float4(__uint_as_float(w[2] << 16), __uint_as_float(w[2] & 0xFFFF0000u),
-                                                       __uint_as_float(w[3] << 16), __uint_as_float(w[3] & 0xFFFF0000u));
+                    tile[pswz(2 * u)] = make_float4(__uint_as_float(w[0] << 16), __uint_as_float(w[0] & 0xFFFF0000u),
+                                                    __uint_as_float(w[1] << 16), __uint_as_float(w[1] & 0xFFFF0000u));
+                    tile[pswz(2 * u + 1)] = make_float4(__uint_as_float(w[2] << 16), __uint_as_float(w[2] & 0xFFFF0000u),
+                                                        __uint_as_float(w[3] << 16), __uint_as_float(w[3] & 0xFFFF0000u));
                 }
             } else {
                 constexpr int kPer = MODE == kDecompress8 ? 16 : MODE == kDecompress16 ? 8 : 4;
                 const unsigned char *y = static_cast<const unsigned char *>(in.p[0]);
-                const float2 bc = r < nblk_cached ? blk_const[r]
-                                                  : block_constants<false>(P.scales[r], P.granularity, P.divisor);
+                const float2 bc = ti.r < nblk_cached ? blk_const[ti.r]
+                                                     : block_constants<false>(P.scales[ti.r], P.granularity, P.divisor);
 #pragma unroll 2
                 for (int i = 0; i < kPElems / kPer / kPThreads; ++i) {
                     const int u = tid + i * kPThreads;
@@ -569,7 +709,7 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
                     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
                     for (int cc = 0; cc < kPer / 4; ++cc) {
-                        float s[4];
+                        float sv[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int ix = cc * 4 + e;
@@ -579,167 +719,112 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
                             else val = w[ix];
                             const float yf = MODE == kDecompress32 ? (float)val
                                              : __uint_as_float(0x4B000000u | val) - 8388608.0f;
-                            s[e] = fmaf(yf, bc.x, bc.y);
+                            sv[e] = fmaf(yf, bc.x, bc.y);
                         }
-                        tile[swz(u * (kPer / 4) + cc)] = make_float4(s[0], s[1], s[2], s[3]);
+                        tile[pswz(u * (kPer / 4) + cc)] = make_float4(sv[0], sv[1], sv[2], sv[3]);
                     }
                 }
-            }
-        }
-    };
-
-    // ================================================================ control warp
-    // Lane 0 claims tasks, waits (bounded) for their dependency and hands them to the compute
-    // warps through s_info[0/1]; it runs at most two tasks ahead of them.
-    if (tid >= kPThreads) {
-        const int lane = tid - kPThreads;
-        for (uint32_t i = 0;; ++i) {
-            const int s = (int)(i & 1);
-            TaskInfo ti;
-            ti.idx = 0xFFFFFFFFu; ti.is_b = 0; ti.wl = 0; ti.r = 0; ti.slot = 0; ti.gen = 0; ti.loaded = 0; ti.pad = 0;
-            // claim task i only once the compute warps have picked up task i-1: a deeper
-            // look-ahead would stretch every task's claim-to-completion time, which is what
-            // dependent tasks wait for
-            if (i >= 1) bar_sync(3 + (s ^ 1), kPCtaThreads);
-            if (lane == 0) {
-                const uint32_t q = atomicAdd(&pc->head, 1u);
-                if ((uint64_t)q < P.total_tasks) {
-                    const TaskId t = decode_task(q, P);
-                    const uint32_t *ctr = t.is_b ? &pc->a_done[t.slot] : &pc->b_done[t.slot];
-                    const uint32_t target = t.is_b ? (t.gen + 1) * T : t.gen * T;
-                    if (target == 0 || wait_at_least(ctr, target, pc, P.dev)) {
-                        ti.idx = t.idx;
-                        ti.is_b = t.is_b;
-                        ti.r = t.wb / P.n_local;
-                        ti.wl = t.wb - ti.r * P.n_local;
-                        ti.slot = t.slot;
-                        ti.gen = t.gen;
-                        ti.loaded = 1;
-                    }
-                }
-            }
-            __syncwarp();
-            if (lane == 0) {
-                s_info[s] = ti;
-                __threadfence_block();
-                *reinterpret_cast<volatile uint32_t *>(&s_published) = i + 1;
-            }
-            __syncwarp();
-            bar_arrive(1 + s, kPCtaThreads);                  // slot s is full
-            if (__shfl_sync(0xFFFFFFFFu, ti.idx, 0) == 0xFFFFFFFFu) break;
-        }
-    } else {
-    // ================================================================ compute warps
-    bar_sync(1, kPCtaThreads);
-    TaskInfo me = s_info[0];
-    bar_arrive(3, kPCtaThreads);
-    bool me_loaded = false;
-
-    for (uint32_t it = 0; me.idx != 0xFFFFFFFFu; ++it) {
-        const int cur = (int)(it & 1);
-        const int s1 = cur ^ 1;
-        if (!me_loaded) issue_load(me, bufs[cur]);
-        cp_async_commit();
-        cp_async_wait_all();
-        // Every barrier of the task doubles as a look at the hand-over flag: as soon as the
-        // control warp has published the next task, its tile starts streaming into the other
-        // buffer.  A task is never waited for before the current one is finished and
-        // signalled: it may depend on it.
-        bool have_next = false;
-        TaskInfo nxt = me;
-        auto barrier_and_prefetch = [&]() {
-            const bool pub = compute_barrier_or(
-                !have_next && *reinterpret_cast<volatile uint32_t *>(&s_published) >= it + 2);
-            if (pub) {
-                bar_sync(1 + s1, kPCtaThreads);
-                nxt = s_info[s1];
-                bar_arrive(3 + s1, kPCtaThreads);
-                if (nxt.idx != 0xFFFFFFFFu) issue_load(nxt, bufs[s1]);
-                cp_async_commit();
-                have_next = true;
             }
         };
 
-        const bool is_b = me.is_b != 0;
-        const uint32_t wl = me.wl;
-        const uint64_t r = me.r;
-        const uint32_t slot = me.slot;
-        const uint32_t idx = me.idx;
-        float4 *tile = bufs[cur];
-        const float2 bc = r < nblk_cached ? blk_const[r]
-                                          : block_constants<kCompress>(P.scales[r], P.granularity, P.divisor);
+        bar_sync(1, kPCtaThreads);
+        TaskInfo me = s_info[0];
+        fence_proxy_async();
+        bar_arrive(3, kPCtaThreads);
 
-        if (!is_b) {
-            // ================================ pass A: tile idx of worker-block wb
-            const uint64_t j0 = r * B + ((uint64_t)idx << kPLog2);
-            if (kCompress && tid < 64) {               // sign words of the tile: 64 calls
-                const uint4 ph = sign_call(j0 + 128ull * tid, P.round, keys);
-                *reinterpret_cast<uint4 *>(sw + 4 * tid) = ph;
-            }
-            barrier_and_prefetch();                   // tile and sign words visible
-            pass_a_round1<kCompress>(tile, sw, tid);
-            barrier_and_prefetch();
-            round_bits_4_7(tile, tid);
-            barrier_and_prefetch();
-            pass_a_round3_store(tile, P.ring + (size_t)slot * B + ((size_t)idx << kPLog2), tid);
-        } else {
-            // ================================ pass B: panel idx of worker-block wb
-            const uint64_t j_tile = r * B + ((uint64_t)idx << (kPLog2 - kb));
-            EpilogueCtx ep;
-            ep.j_tile = j_tile;
-            ep.kappa = bc.x; ep.half_g = bc.y; ep.gf = (float)P.granularity; ep.c_block = P.c_block;
-            ep.lut = lut + (tid & (kLutRep - 1));
-            ep.worker = P.worker_base + wl; ep.round = P.round;
-            ep.packed = kCompress ? static_cast<unsigned char *>(outp.p[wl]) : nullptr;
-            ep.rotated = kCompress ? static_cast<float *>(rotated.p[wl]) : nullptr;
-            ep.out = kCompress ? nullptr : static_cast<float *>(outp.p[0]);
-            ep.d = P.d;
-            ep.sw = sw;
-            ep.words_per_row = max(1, (1 << (kPLog2 - kb)) >> 5);
-            if (!kCompress) {
-                TileGeom g;
-                g.row_log2 = (uint32_t)kb; g.col_log2 = (uint32_t)(kPLog2 - kb);
-                g.row_stride = 1ull << kPLog2; g.round = P.round;
-                fill_sign_words(sw, g, j_tile, keys, tid, kPThreads);
-            }
-            barrier_and_prefetch();                   // tile (and sign words) visible
-            const int e1 = kb < 4 ? kb : 4;
-            if (KB == 7) {
-                round_bits_4_7(tile, tid);
-            } else {
-                switch (e1) {
-                case 4: p_round<4>(tile, ccl, tid); break;
-                case 3: p_round<3>(tile, ccl, tid); break;
-                default: p_round<2>(tile, ccl, tid); break;
+        bool aborted = false;
+        for (uint32_t it = 0; me.idx != 0xFFFFFFFFu; ++it) {
+            const int cur = (int)(it & 1);
+            float4 *tile = bufs[cur];
+            if (!aborted) {
+                bool arrived = true;
+                if (me.tma) {
+                    arrived = mbar_wait(&s_mbar[cur], me.phase);
+                } else {
+                    load_tile(me, tile);
+                    cp_async_commit();
+                    cp_async_wait_all();
+                }
+                // tile visible to all compute warps.  A TMA load that never completed ends the
+                // launch: flag it, raise the abort flag, and from here on only keep the
+                // hand-shake with the control warp going until it hands over "no task".
+                aborted = compute_barrier_or(!arrived);
+                if (aborted && tid == 0) {
+                    atomicOr(&P.dev->status, THC_STATUS_WAIT_TIMEOUT);
+                    atomicExch(&pc->abort, 1u);
                 }
             }
-            barrier_and_prefetch();
-            if (KB == 7) {
-                pass_b_last_round_kb7<kCompress, BITS, IDENTITY>(tile, tid, ep, keys);
+            if (!aborted) {
+            const bool is_b = me.is_b != 0;
+            const uint32_t wl = me.wl;
+            const uint64_t r = me.r;
+            const uint32_t slot = me.slot;
+            const uint32_t idx = me.idx;
+            const float2 bc = r < nblk_cached ? blk_const[r]
+                                              : block_constants<kCompress>(P.scales[r], P.granularity, P.divisor);
+
+            if (!is_b) {
+                // ================================ pass A: tile idx of worker-block wb
+                pass_a_round1<kCompress>(tile, sw + 256 * cur, tid);
+                compute_barrier();
+                round_rows_0_3(tile, tid);
+                compute_barrier();
+                pass_a_round3_store(tile, P.ring + (size_t)slot * B + ((size_t)idx << kPLog2), tid);
             } else {
-                const int rem = kb - e1;
-                const int e_last = rem < 3 ? rem : 3;
-                if (rem > e_last) p_rounds(tile, ccl + e1, ccl + kb - e_last, tid);
-                switch (e_last) {
-                case 3: pass_b_last_round<3, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
-                case 2: pass_b_last_round<2, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
-                case 1: pass_b_last_round<1, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
-                default: pass_b_last_round<0, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
+                // ================================ pass B: panel idx of worker-block wb
+                const uint64_t j_tile = r * B + ((uint64_t)idx << (kPLog2 - kb));
+                EpilogueCtx ep;
+                ep.j_tile = j_tile;
+                ep.kappa = bc.x; ep.half_g = bc.y; ep.gf = (float)P.granularity; ep.c_block = P.c_block;
+                ep.lut = lut + (tid & (kLutRep - 1));
+                ep.worker = P.worker_base + wl; ep.round = P.round;
+                ep.packed = kCompress ? static_cast<unsigned char *>(outp.p[wl]) : nullptr;
+                ep.rotated = kCompress ? static_cast<float *>(rotated.p[wl]) : nullptr;
+                ep.out = kCompress ? nullptr : static_cast<float *>(outp.p[0]);
+                ep.d = P.d;
+                ep.sw = sw;
+                ep.words_per_row = max(1, (1 << (kPLog2 - kb)) >> 5);
+                if (!kCompress) {
+                    TileGeom g;
+                    g.row_log2 = (uint32_t)kb; g.col_log2 = (uint32_t)(kPLog2 - kb);
+                    g.row_stride = 1ull << kPLog2; g.round = P.round;
+                    fill_sign_words(sw, g, j_tile, keys, tid, kPThreads);
+                }
+                const int e1 = kb < 4 ? kb : 4;
+                if (KB == 7) {
+                    round_rows_0_3(tile, tid);
+                } else {
+                    switch (e1) {
+                    case 4: p_round<4>(tile, ccl, tid); break;
+                    case 3: p_round<3>(tile, ccl, tid); break;
+                    default: p_round<2>(tile, ccl, tid); break;
+                    }
+                }
+                compute_barrier();
+                if (KB == 7) {
+                    pass_b_last_round_kb7<kCompress, BITS, IDENTITY>(tile, tid, ep, keys);
+                } else {
+                    const int rem = kb - e1;
+                    const int e_last = rem < 3 ? rem : 3;
+                    if (rem > e_last) p_rounds(tile, ccl + e1, ccl + kb - e_last, tid);
+                    switch (e_last) {
+                    case 3: pass_b_last_round<3, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
+                    case 2: pass_b_last_round<2, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
+                    case 1: pass_b_last_round<1, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
+                    default: pass_b_last_round<0, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
+                    }
                 }
             }
+            // every compute warp has issued its stores and is done with the tile and sign words
+            compute_barrier();
+            if (tid == 0) red_release_add(is_b ? &pc->b_done[slot] : &pc->a_done[slot], 1u);
+            }
+            // pick up the next task (only now: it may depend on the one just finished)
+            bar_sync(1 + (cur ^ 1), kPCtaThreads);
+            me = s_info[cur ^ 1];
+            fence_proxy_async();
+            bar_arrive(3 + (cur ^ 1), kPCtaThreads);
         }
-        // every compute warp has issued its stores and is done with the tile and sign words
-        compute_barrier();
-        if (tid == 0) red_release_add(is_b ? &pc->b_done[slot] : &pc->a_done[slot], 1u);
-        if (!have_next) {
-            bar_sync(1 + s1, kPCtaThreads);
-            nxt = s_info[s1];
-            bar_arrive(3 + s1, kPCtaThreads);
-        }
-        me_loaded = have_next;
-        me = nxt;
-    }
-    cp_async_wait_all();
     }
     __syncthreads();
 
@@ -748,7 +833,7 @@ thc_pipeline_kernel(PipeParams P, PtrArrayP in, MutPtrArrayP outp, MutPtrArrayP 
         __threadfence();
         const uint32_t left = atomicAdd(&pc->exited, 1u);
         if (left == gridDim.x - 1) {
-            for (int s = 0; s < kMaxRing; ++s) { pc->a_done[s] = 0; pc->b_done[s] = 0; }
+            for (int sl = 0; sl < kMaxRing; ++sl) { pc->a_done[sl] = 0; pc->b_done[sl] = 0; }
             pc->abort = 0;
             pc->head = 0;
             __threadfence();
