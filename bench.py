@@ -35,7 +35,7 @@ KERNELS_PER_STEP = {"prepare": 2, "compress": 1, "aggregate": 1, "decompress": 1
 # DRAM bytes per (worker, padded coordinate) of the compress kernel, measured with ncu on the
 # d=2^24, n=4, b=4 sweep point (profiles/thc_pipeline_kernel_sweep_d2p24_b4_n4.md); traffic
 # grows in proportion to n*d_pad, so a full launch is this times n*d_pad.
-NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.315}
+NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.261}
 
 
 def pick_workload(name: str) -> W.Workload:
