@@ -178,6 +178,13 @@ int thc_prepare_noalloc(const void *const *grads, uint32_t n, uint64_t d, uint32
 /* Read and clear the status bits (synchronises `stream`).  flags is a host pointer. */
 int thc_status(thc_ctx *ctx, uint32_t *flags, void *stream);
 
+/* Test hook for the bounded waits of the large-block pipeline (no counterpart in the paper).
+ * The next thc_compress / thc_decompress on this context starts its task queue at position
+ * `count` instead of 0, so tasks that depend on the skipped ones can never be satisfied: the
+ * kernel must notice (about two seconds), set THC_STATUS_WAIT_TIMEOUT, and return with the
+ * context still usable; the outputs of that call are undefined.  Synchronises the device. */
+int thc_debug_skip_tasks(thc_ctx *ctx, uint32_t count);
+
 const char *thc_strerror(int code);
 
 /* Library build identification, e.g. "thc-b200 sm_100a". */

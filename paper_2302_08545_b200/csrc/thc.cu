@@ -1183,6 +1183,16 @@ int thc_aggregate(thc_ctx *ctx, const void *const *packed, uint32_t n, uint64_t 
     return THC_OK;
 }
 
+int thc_debug_skip_tasks(thc_ctx *ctx, uint32_t count)
+{
+    int rc = check_launch_ctx(ctx);
+    if (rc != THC_OK) return rc;
+    THC_CUDA(cudaDeviceSynchronize());
+    PipeCounters *pc = reinterpret_cast<PipeCounters *>(ctx->dev->counters);
+    THC_CUDA(cudaMemcpy(&pc->head, &count, sizeof count, cudaMemcpyHostToDevice));
+    return THC_OK;
+}
+
 int thc_status(thc_ctx *ctx, uint32_t *flags, void *stream)
 {
     int rc = check_launch_ctx(ctx);

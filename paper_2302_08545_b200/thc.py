@@ -21,7 +21,7 @@ STATUS_NONFINITE, STATUS_ZERO_BLOCK, STATUS_WAIT_TIMEOUT = 1, 2, 4
 
 EXPORTS = ("thc_create", "thc_destroy", "thc_sizes", "thc_prepare", "thc_compress",
            "thc_quantize_rotated", "thc_aggregate", "thc_decompress", "thc_prepare_noalloc",
-           "thc_status", "thc_strerror", "thc_version")
+           "thc_debug_skip_tasks", "thc_status", "thc_strerror", "thc_version")
 NOALLOC_SCRATCH_BYTES = 4 << 20
 
 
@@ -77,6 +77,7 @@ def lib():
     L.thc_aggregate.argtypes = [vp, pp, u32, u64, vp, vp]
     L.thc_decompress.argtypes = [vp, vp, u32, u64, u32, vp, vp, vp, u64, vp]
     L.thc_prepare_noalloc.argtypes = [pp, u32, u64, u32, u32, ctypes.c_double, vp, vp, vp]
+    L.thc_debug_skip_tasks.argtypes = [vp, u32]
     L.thc_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
     for name in EXPORTS[:-2]:
         getattr(L, name).restype = ctypes.c_int
@@ -203,6 +204,10 @@ class Context:
         ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
         _check(lib().thc_decompress(self._h, _dp(total), divisor, d, rnd, _dp(scales), _dp(out),
                                     _dp(workspace), ws_bytes, _stream(stream)), "thc_decompress")
+
+    def debug_skip_tasks(self, count: int):
+        """Test hook: the next pipeline launch starts its task queue at `count`."""
+        _check(lib().thc_debug_skip_tasks(self._h, count), "thc_debug_skip_tasks")
 
     def status(self, stream=None) -> int:
         flags = ctypes.c_uint32(0)

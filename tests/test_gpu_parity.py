@@ -232,3 +232,35 @@ def test_partial_aggregation_uses_the_count_as_divisor():
     assert np.array_equal(r.sum_numpy(), sum_ref)
     out_ref = O.decompress(sum_ref, len(subset), w.d, scl, c, 0)
     assert np.array_equal(r.out.cpu().numpy().view(np.uint32), out_ref.view(np.uint32))
+
+
+def test_unsatisfiable_dependency_times_out_and_the_context_stays_usable():
+    """Host-side injection on a tiny launch: the task queue starts one task late, so the
+    pass-B panels of the first worker-block wait for a pass-A tile nobody will produce.  The
+    kernel's bounded wait must expire, set THC_STATUS_WAIT_TIMEOUT and return; afterwards
+    the same context must run a correct round."""
+    import time
+    import torch
+    from paper_2302_08545_b200 import runner, thc
+    w = _mk(1, 2 << 15, 15)
+    x, _ = _inputs(w)
+    ctx = runner.context_for(w)
+    r = runner.Round(ctx, w.n, w.d, want_rotated=False)
+    r.upload(x)
+    r.prepare()
+    torch.cuda.synchronize()
+    ctx.debug_skip_tasks(1)
+    t0 = time.time()
+    r.compress(0)
+    torch.cuda.synchronize()
+    waited = time.time() - t0
+    assert ctx.status() & thc.STATUS_WAIT_TIMEOUT
+    assert waited < 30.0
+    # the context recovers: counters were cleared by the last CTA
+    r.run(0)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    c = _ocfg(w)
+    ref = O.thc_round(x, c, 0, scl=r.scales.cpu().numpy())
+    assert np.array_equal(np.stack([p.cpu().numpy() for p in r.packed]), ref["packed"])
+    assert np.array_equal(r.out.cpu().numpy().view(np.uint32), ref["out"].view(np.uint32))
