@@ -75,6 +75,8 @@ def _load():
     lib.thc_oracle_decompress.restype = None
     lib.thc_oracle_estimate.argtypes = [vp, u32, u32, u64, u32, f32p, u32, f32p]
     lib.thc_oracle_estimate.restype = None
+    lib.thc_oracle_error_feedback.argtypes = [f32p, u8p, u64, u32, f32p, u32, u16p, u64, u32, f32p]
+    lib.thc_oracle_error_feedback.restype = None
     lib.thc_oracle_dequantize.argtypes = [u8p, u64, u32, f32p, u32, u16p, f64p]
     lib.thc_oracle_dequantize.restype = None
     _lib = lib
@@ -251,6 +253,20 @@ def estimate(total, divisor: int, scl, cfg: Config) -> np.ndarray:
                                 cfg.log2_block, _p(scl, ctypes.c_float), cfg.granularity,
                                 _p(v, ctypes.c_float))
     return v
+
+
+def error_feedback(x, z, scl, cfg: Config, rnd: int) -> np.ndarray:
+    """e = x - RHT^-1(X) for one worker (Algorithm 3): x has d entries, z d_pad indices."""
+    x = _f32(x)
+    z = np.ascontiguousarray(z, dtype=np.uint8)
+    scl = _f32(scl)
+    assert z.size == cfg.d_pad(x.size)
+    e = np.zeros(x.size, dtype=np.float32)
+    t = cfg.table_u16()
+    _load().thc_oracle_error_feedback(_p(x, ctypes.c_float), _p(z, ctypes.c_uint8), x.size,
+                                      cfg.log2_block, _p(scl, ctypes.c_float), cfg.granularity,
+                                      _p(t, ctypes.c_uint16), cfg.seed, rnd, _p(e, ctypes.c_float))
+    return e
 
 
 def dequantize(z, scl, cfg: Config) -> np.ndarray:

@@ -348,6 +348,34 @@ void thc_oracle_decompress(const void *sum, uint32_t w, uint32_t divisor, uint64
     free(v);
 }
 
+/* ------------------------------------------------------------------------------------
+ * Error feedback (Section 5.1; Algorithm 3, "Quantization error"): e = x - RHT^-1(X), where X
+ * is the worker's own quantised vector in the rotated domain, X[j] = m + T[z[j]] (M - m)/g.
+ * x has d entries, z has d_pad indices (unpacked).  X is evaluated like the estimate of a
+ * one-worker aggregate (fma(T[z], 2M/g, -M)); the subtraction is one fp32 operation.
+ * The next round compresses grad + e (Algorithm 3, "x_i = grad_i + e_i").
+ * ---------------------------------------------------------------------------------- */
+void thc_oracle_error_feedback(const float *x, const uint8_t *z, uint64_t d, uint32_t k,
+                               const float *scales, uint32_t g, const uint16_t *table,
+                               uint64_t seed, uint32_t round, float *e)
+{
+    uint64_t B = (uint64_t)1 << k;
+    uint64_t nb = (d + B - 1) / B;
+    uint64_t d_pad = nb * B;
+    float *v = (float *)malloc(sizeof(float) * d_pad);
+    float *back = (float *)malloc(sizeof(float) * d);
+    for (uint64_t j = 0; j < d_pad; ++j) {
+        float M = scales[j / B];
+        if (!(M > 0.0f) || !isfinite(M)) { v[j] = 0.0f; continue; }      /* R8 */
+        float step = (float)(2.0 * (double)M / (double)g);
+        v[j] = fmaf((float)table[z[j]], step, -M);
+    }
+    thc_oracle_rht_inverse(v, d, k, seed, round, back);
+    for (uint64_t j = 0; j < d; ++j) e[j] = x[j] - back[j];
+    free(v);
+    free(back);
+}
+
 /* Value a single worker's index stands for on the real line, before the inverse RHT
  * (Algorithm 2: the quantization value m + T[z] (M-m)/g).  Used to state the
  * homomorphic identity of Definition 3. */

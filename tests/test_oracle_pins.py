@@ -538,3 +538,51 @@ def test_slice_forms_agree_with_the_whole_vector():
         assert np.array_equal(zp, zw[lo:lo + 64])
         ip = O.rht_inverse(vals[lo:lo + 64], hi - lo, c, 3, j_base=lo)
         assert np.array_equal(ip.view(np.uint32), inv_whole[lo:hi].view(np.uint32))
+
+
+# ------------------------------------------------------------------- error feedback
+def test_error_feedback_is_the_residual_of_the_workers_own_quantised_vector():
+    """e = x - RHT^-1(X): equals x minus the decompression of a one-worker aggregate with
+    divisor 1 (Definition 3 with n = 1), so x = e + RHT^-1(X) up to one rounding."""
+    k, d = 8, 700
+    c = cfg(k=k)
+    x = np.random.default_rng(31).standard_normal((3, d)).astype(np.float32)
+    scl = O.scales(x, c)
+    for i in range(3):
+        z = O.quantize(O.rht_forward(x[i], c, 4), scl, c, 4, i)
+        e = O.error_feedback(x[i], z, scl, c, 4)
+        one = O.aggregate(O.pack(z, 4)[None, :], c.d_pad(d), c, 8)
+        back = O.decompress(one, 1, d, scl, c, 4)
+        assert np.array_equal(e, x[i] - back)
+        # the residual is small: 4-bit THC keeps a few per cent NMSE per worker
+        assert (e.astype(np.float64) ** 2).sum() < 0.1 * (x[i].astype(np.float64) ** 2).sum()
+
+
+def test_error_feedback_removes_the_truncation_bias_over_rounds():
+    """Section 5.1: truncation makes THC biased; with error feedback the running average of
+    the decompressed vectors converges to the true vector, because
+    sum_r RHT^-1(X^r) = R x - e^R and e stays bounded.  Without feedback the bias stays."""
+    k, d, R = 8, 256, 60
+    c = cfg(k=k, t_p=0.8)                      # aggressive truncation: about 42 % clamped
+    rng = np.random.default_rng(33)
+    grad = rng.standard_normal(d).astype(np.float32)
+    e = np.zeros(d, dtype=np.float32)
+    acc_ef = np.zeros(d)
+    acc_plain = np.zeros(d)
+    for r in range(R):
+        x = (grad + e).astype(np.float32)
+        scl = O.scales(x[None, :], c)
+        z = O.quantize(O.rht_forward(x, c, r), scl, c, r, 0)
+        one = O.aggregate(O.pack(z, 4)[None, :], d, c, 8)
+        acc_ef += O.decompress(one, 1, d, scl, c, r)
+        e = O.error_feedback(x, z, scl, c, r)
+        scl0 = O.scales(grad[None, :], c)
+        z0 = O.quantize(O.rht_forward(grad, c, r), scl0, c, r, 0)
+        acc_plain += O.decompress(O.aggregate(O.pack(z0, 4)[None, :], d, c, 8), 1, d, scl0, c, r)
+    g64 = grad.astype(np.float64)
+    err_ef = np.linalg.norm(acc_ef / R - g64) / np.linalg.norm(g64)
+    err_plain = np.linalg.norm(acc_plain / R - g64) / np.linalg.norm(g64)
+    assert err_ef < 0.05
+    assert err_plain > 3 * err_ef
+    # exactly: R * mean = R * grad - e^R (up to fp32 rounding of the additions)
+    assert np.allclose(acc_ef, R * g64 - e, atol=2e-4 * R)
