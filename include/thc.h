@@ -175,6 +175,24 @@ int thc_prepare_noalloc(const void *const *grads, uint32_t n, uint64_t d, uint32
                         uint32_t in_dtype, double t_p, float *scales, uint32_t *status_or_null,
                         void *stream);
 
+/* Error feedback (Section 5.1; Algorithm 3, "e_i = x_i - RHT^-1(X_i)"): for each of the n_local
+ * workers, the residual between what it compressed and what its own indices stand for,
+ *     ef[i] = x_i - RHT^-1( m + T[Z_i] (M - m)/g ),
+ * to be added to the next round's gradient (thc_accumulate_error).  fp32 contexts only
+ * (THC_EUNSUPPORTED for bf16 inputs).  Built from the library's own kernels: table values
+ * of one worker (thc_aggregate with n = 1), thc_decompress with divisor 1, one subtraction.
+ *   grads    host array of n_local device pointers: the x_i that were compressed
+ *   packed   host array of n_local device pointers: their packed indices
+ *   ef       host array of n_local device pointers, d fp32 each, written
+ *   workspace  as reported by thc_sizes (it includes room for one worker's table values)  */
+int thc_error_feedback(thc_ctx *ctx, const void *const *grads, const void *const *packed,
+                       uint32_t n_local, uint64_t d, uint32_t round, const float *scales,
+                       float *const *ef, void *workspace, uint64_t workspace_bytes, void *stream);
+
+/* Algorithm 3, "x_i = grad_i + e_i": grads[i] += ef[i] in place, fp32, d elements each. */
+int thc_accumulate_error(thc_ctx *ctx, float *const *grads, const float *const *ef,
+                         uint32_t n_local, uint64_t d, void *stream);
+
 /* Read and clear the status bits (synchronises `stream`).  flags is a host pointer. */
 int thc_status(thc_ctx *ctx, uint32_t *flags, void *stream);
 

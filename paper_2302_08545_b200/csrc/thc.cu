@@ -378,6 +378,40 @@ aggregate_b4w8_kernel(PtrArray in, uint32_t n, uint64_t units16, const DeviceBlo
     }
 }
 
+// ------------------------------------------------------------------------ error feedback
+// e <- x - e (e holds RHT^-1(X) on entry) and x <- x + e, 128-bit accesses with a scalar tail.
+__global__ void __launch_bounds__(kThreads)
+ef_subtract_kernel(const float *__restrict__ x, float *__restrict__ e, uint64_t d)
+{
+    const uint64_t n4 = d / 4;
+    for (uint64_t c = (uint64_t)blockIdx.x * kThreads + threadIdx.x; c < n4; c += (uint64_t)gridDim.x * kThreads) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(x) + c);
+        float4 b = reinterpret_cast<float4 *>(e)[c];
+        b.x = a.x - b.x; b.y = a.y - b.y; b.z = a.z - b.z; b.w = a.w - b.w;
+        reinterpret_cast<float4 *>(e)[c] = b;
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (d & 3)) {
+        const uint64_t j = n4 * 4 + threadIdx.x;
+        e[j] = x[j] - e[j];
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+accumulate_kernel(float *__restrict__ x, const float *__restrict__ e, uint64_t d)
+{
+    const uint64_t n4 = d / 4;
+    for (uint64_t c = (uint64_t)blockIdx.x * kThreads + threadIdx.x; c < n4; c += (uint64_t)gridDim.x * kThreads) {
+        float4 a = reinterpret_cast<float4 *>(x)[c];
+        const float4 b = __ldg(reinterpret_cast<const float4 *>(e) + c);
+        a.x = a.x + b.x; a.y = a.y + b.y; a.z = a.z + b.z; a.w = a.w + b.w;
+        reinterpret_cast<float4 *>(x)[c] = a;
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (d & 3)) {
+        const uint64_t j = n4 * 4 + threadIdx.x;
+        x[j] = x[j] + e[j];
+    }
+}
+
 // ------------------------------------------------------------------------------ prepare
 // Partial sums of squares in fp64: one CTA per (chunk of 2^chunk_log2 coordinates, worker).
 template <bool BF16>
@@ -740,7 +774,9 @@ int thc_sizes(const thc_ctx *ctx, uint64_t d, uint32_t n_local, thc_sizes_t *s)
         const PipePlan pl = plan_pipeline(ctx, s->nblocks * n_local);
         two_pass_ws = (uint64_t)pl.ring * B * 4;
     }
-    s->workspace_bytes = round_up((prepare_ws > two_pass_ws ? prepare_ws : two_pass_ws) + 256, 256);
+    // scratch of prepare / the pipeline's ring, then one worker's table values (error feedback)
+    s->workspace_bytes = round_up((prepare_ws > two_pass_ws ? prepare_ws : two_pass_ws) + 256, 256) +
+                         round_up(s->sum_bytes, 256);
     return THC_OK;
 }
 
@@ -1062,7 +1098,7 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
     const bool two_pass = k > (uint32_t)kTileLog2;
     if (two_pass) {
         if (workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
-        if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
+        if (workspace_bytes < sz.workspace_bytes - round_up(sz.sum_bytes, 256)) return THC_EWORKSPACE;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     PtrArray in;
@@ -1180,6 +1216,59 @@ int thc_aggregate(thc_ctx *ctx, const void *const *packed, uint32_t n, uint64_t 
 #undef THC_AGW
 #undef THC_AG
     THC_CUDA(cudaGetLastError());
+    return THC_OK;
+}
+
+int thc_error_feedback(thc_ctx *ctx, const void *const *grads, const void *const *packed,
+                       uint32_t n_local, uint64_t d, uint32_t round, const float *scales,
+                       float *const *ef, void *workspace, uint64_t workspace_bytes, void *stream)
+{
+    int rc = check_launch_ctx(ctx);
+    if (rc != THC_OK) return rc;
+    if (ctx->cfg.in_dtype != THC_F32) return THC_EUNSUPPORTED;
+    thc_sizes_t sz;
+    if ((rc = thc_sizes(ctx, d, 1, &sz)) != THC_OK) return rc;
+    if (n_local == 0 || n_local > THC_MAX_WORKERS) return THC_EINVAL;
+    if ((rc = check_ptr_array(grads, n_local)) != THC_OK) return rc;
+    if ((rc = check_ptr_array(packed, n_local)) != THC_OK) return rc;
+    if ((rc = check_ptr_array(reinterpret_cast<const void *const *>(ef), n_local)) != THC_OK) return rc;
+    if (scales == nullptr || workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
+    if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint64_t ring_bytes = sz.workspace_bytes - round_up(sz.sum_bytes, 256);
+    void *values = static_cast<unsigned char *>(workspace) + ring_bytes;
+    uint64_t blocks = (d / 4 + kThreads - 1) / kThreads;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    if (blocks == 0) blocks = 1;
+    for (uint32_t i = 0; i < n_local; ++i) {
+        if ((rc = thc_aggregate(ctx, &packed[i], 1, d, values, stream)) != THC_OK) return rc;
+        if ((rc = thc_decompress(ctx, values, 1, d, round, scales, ef[i], workspace, ring_bytes, stream)) != THC_OK)
+            return rc;
+        ef_subtract_kernel<<<(unsigned)blocks, kThreads, 0, st>>>(static_cast<const float *>(grads[i]), ef[i], d);
+        THC_CUDA(cudaGetLastError());
+    }
+    return THC_OK;
+}
+
+int thc_accumulate_error(thc_ctx *ctx, float *const *grads, const float *const *ef, uint32_t n_local,
+                         uint64_t d, void *stream)
+{
+    int rc = check_launch_ctx(ctx);
+    if (rc != THC_OK) return rc;
+    if (ctx->cfg.in_dtype != THC_F32) return THC_EUNSUPPORTED;
+    if (n_local == 0 || n_local > THC_MAX_WORKERS || d == 0) return THC_EINVAL;
+    if ((rc = check_ptr_array(reinterpret_cast<const void *const *>(grads), n_local)) != THC_OK) return rc;
+    if ((rc = check_ptr_array(reinterpret_cast<const void *const *>(ef), n_local)) != THC_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint64_t blocks = (d / 4 + kThreads - 1) / kThreads;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    if (blocks == 0) blocks = 1;
+    for (uint32_t i = 0; i < n_local; ++i) {
+        accumulate_kernel<<<(unsigned)blocks, kThreads, 0, st>>>(grads[i], ef[i], d);
+        THC_CUDA(cudaGetLastError());
+    }
     return THC_OK;
 }
 

@@ -21,7 +21,7 @@ STATUS_NONFINITE, STATUS_ZERO_BLOCK, STATUS_WAIT_TIMEOUT = 1, 2, 4
 
 EXPORTS = ("thc_create", "thc_destroy", "thc_sizes", "thc_prepare", "thc_compress",
            "thc_quantize_rotated", "thc_aggregate", "thc_decompress", "thc_prepare_noalloc",
-           "thc_debug_skip_tasks", "thc_status", "thc_strerror", "thc_version")
+           "thc_error_feedback", "thc_accumulate_error", "thc_debug_skip_tasks", "thc_status", "thc_strerror", "thc_version")
 NOALLOC_SCRATCH_BYTES = 4 << 20
 
 
@@ -77,6 +77,8 @@ def lib():
     L.thc_aggregate.argtypes = [vp, pp, u32, u64, vp, vp]
     L.thc_decompress.argtypes = [vp, vp, u32, u64, u32, vp, vp, vp, u64, vp]
     L.thc_prepare_noalloc.argtypes = [pp, u32, u64, u32, u32, ctypes.c_double, vp, vp, vp]
+    L.thc_error_feedback.argtypes = [vp, pp, pp, u32, u64, u32, vp, pp, vp, u64, vp]
+    L.thc_accumulate_error.argtypes = [vp, pp, pp, u32, u64, vp]
     L.thc_debug_skip_tasks.argtypes = [vp, u32]
     L.thc_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
     for name in EXPORTS[:-2]:
@@ -204,6 +206,20 @@ class Context:
         ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
         _check(lib().thc_decompress(self._h, _dp(total), divisor, d, rnd, _dp(scales), _dp(out),
                                     _dp(workspace), ws_bytes, _stream(stream)), "thc_decompress")
+
+    def error_feedback(self, grads, packed, d: int, rnd: int, scales, ef, workspace, stream=None):
+        ga = _ptr_array([_dp(g) for g in grads])
+        pa = _ptr_array([_dp(p) for p in packed])
+        ea = _ptr_array([_dp(e) for e in ef])
+        _check(lib().thc_error_feedback(self._h, ga, pa, len(grads), d, rnd, _dp(scales), ea,
+                                        _dp(workspace), workspace.numel() * workspace.element_size(),
+                                        _stream(stream)), "thc_error_feedback")
+
+    def accumulate_error(self, grads, ef, d: int, stream=None):
+        ga = _ptr_array([_dp(g) for g in grads])
+        ea = _ptr_array([_dp(e) for e in ef])
+        _check(lib().thc_accumulate_error(self._h, ga, ea, len(grads), d, _stream(stream)),
+               "thc_accumulate_error")
 
     def debug_skip_tasks(self, count: int):
         """Test hook: the next pipeline launch starts its task queue at `count`."""

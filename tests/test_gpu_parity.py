@@ -264,3 +264,29 @@ def test_unsatisfiable_dependency_times_out_and_the_context_stays_usable():
     ref = O.thc_round(x, c, 0, scl=r.scales.cpu().numpy())
     assert np.array_equal(np.stack([p.cpu().numpy() for p in r.packed]), ref["packed"])
     assert np.array_equal(r.out.cpu().numpy().view(np.uint32), ref["out"].view(np.uint32))
+
+
+@pytest.mark.parametrize("k,d,n", [(10, 33_001, 3), (16, 150_000, 2), (20, (1 << 21) + 99, 2)])
+def test_error_feedback_matches_oracle(k, d, n):
+    """e_i = x_i - RHT^-1(X_i) (Algorithm 3) from the worker's own packed indices: bit-exact
+    against the oracle on the same indices and scales; and x_i + e_i through
+    thc_accumulate_error is the fp32 sum."""
+    import torch
+    from paper_2302_08545_b200 import runner
+    w = _mk(n, d, k)
+    x, _ = _inputs(w)
+    ctx, r = _gpu_round(w, x, rnd=2, want_rotated=False)
+    ef = [torch.zeros(d, dtype=torch.float32, device=r.device) for _ in range(n)]
+    ctx.error_feedback(r.grads, r.packed, d, 2, r.scales, ef, r.workspace)
+    torch.cuda.synchronize()
+    c = _ocfg(w)
+    scl = r.scales.cpu().numpy()
+    for i in range(n):
+        z = O.unpack(r.packed[i].cpu().numpy(), r.sz.d_pad, w.bits)
+        ref = O.error_feedback(x[i], z, scl, c, 2)
+        got = ef[i].cpu().numpy()
+        assert np.array_equal(got.view(np.uint32), ref.view(np.uint32)), f"worker {i}"
+    ctx.accumulate_error(r.grads, ef, d)
+    torch.cuda.synchronize()
+    for i in range(n):
+        assert np.array_equal(r.grads[i].cpu().numpy(), x[i] + ef[i].cpu().numpy())
