@@ -107,13 +107,16 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p)
 }
 
 // Bounded wait (one thread): true once *ctr >= target; false if the launch was aborted or
-// the wait expired (then the timeout bit and the abort flag are set).
+// the wait expired (then the timeout bit and the abort flag are set).  on_poll() runs between
+// polls: the waiting thread keeps its other duty (signalling finished tasks) alive.
+template <class F>
 __device__ __forceinline__ bool wait_at_least(const uint32_t *ctr, uint32_t target,
-                                              PipeCounters *pc, DeviceBlock *dev)
+                                              PipeCounters *pc, DeviceBlock *dev, F on_poll)
 {
     for (uint32_t it = 0; it < kMaxPolls; ++it) {
         if (ld_acquire_u32(ctr) >= target) return true;
         if (ld_relaxed_u32(&pc->abort) != 0) return false;
+        on_poll();
         __nanosleep(it < 32 ? 20 : 200);
     }
     atomicOr(&dev->status, THC_STATUS_WAIT_TIMEOUT);
@@ -147,12 +150,16 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 __device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
 // Named barriers: 1,2 = task slot full; 3,4 = task slot consumed; 5 = compute warps only.
+// bar.sync / bar.arrive are warp-aligned instructions: the __syncwarp() makes sure the warp
+// has reconverged after any single-thread section before it.
 __device__ __forceinline__ void bar_sync(int id, int count)
 {
+    __syncwarp();
     asm volatile("bar.sync %0, %1;" :: "r"(id), "r"(count) : "memory");
 }
 __device__ __forceinline__ void bar_arrive(int id, int count)
 {
+    __syncwarp();
     asm volatile("bar.arrive %0, %1;" :: "r"(id), "r"(count) : "memory");
 }
 __device__ __forceinline__ void compute_barrier() { bar_sync(5, kPThreads); }
@@ -161,6 +168,7 @@ __device__ __forceinline__ void compute_barrier() { bar_sync(5, kPThreads); }
 __device__ __forceinline__ bool compute_barrier_or(bool pred)
 {
     uint32_t out;
+    __syncwarp();
     asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\t"
                  "barrier.cta.red.or.pred q, 5, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
                  : "=r"(out) : "r"((uint32_t)pred), "r"(kPThreads) : "memory");
@@ -185,10 +193,31 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(a), "r"(bytes) : "memory");
 }
 
-// Bounded wait for a phase of the mbarrier; false if it did not complete.
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(a) : "memory");
+}
+
+// Non-blocking: has the phase with this parity completed?
+__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity)
+{
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(a), "r"(parity) : "memory");
+    return done != 0;
+}
+
+// Bounded wait for a phase of the mbarrier; false if it did not complete within about a
+// second (2^31 SM cycles; a try_wait may itself suspend the thread for a while, so the bound
+// is on time, not on attempts).
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
 {
     const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+    long long t0 = 0;
     for (uint32_t it = 0; it < (1u << 22); ++it) {
         uint32_t done;
         asm volatile("{\n\t.reg .pred p;\n\t"
@@ -196,6 +225,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
                      "selp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(done) : "r"(a), "r"(parity) : "memory");
         if (done) return true;
+        if ((it & 63u) == 63u) {
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > (1ll << 31)) return false;
+        }
     }
     return false;
 }
@@ -217,6 +251,13 @@ __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *m
 __device__ __forceinline__ void fence_proxy_async()
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// The same for global memory: generic-proxy writes (made visible by an acquire) before this
+// thread's later TMA reads of them.
+__device__ __forceinline__ void fence_proxy_async_global()
+{
+    asm volatile("fence.proxy.async.global;" ::: "memory");
 }
 
 __device__ __forceinline__ uint64_t make_evict_normal_policy()
@@ -325,22 +366,25 @@ __device__ __forceinline__ void p_rounds(float4 *tile, int lo, int hi, int tid)
 // A tile is 256 rows of 8 chunks (32 coordinates); row r, chunk cc sits at r*8 + (cc ^ (r&7)).
 //
 // First round, in place: sign flip (compress), stages of stride 1 and 2 inside each chunk,
-// then stride 4, 8, 16 across the eight chunks of a row.  Thread t owns rows t and t + 128.
+// then stride 4, 8, 16 across the eight chunks of a row.  Thread (warp w, lane l) owns rows
+// 64 w + l and 64 w + 32 + l: a warp works on the same 64 rows here and in the next round
+// (round_rows_0_3), so only a warp barrier separates the two.
 template <bool FLIP>
 __device__ __forceinline__ void pass_a_round1(float4 *tile, const uint32_t *sw, int tid)
 {
     const int x = tid & 7;
+    const int r0 = ((tid >> 5) << 6) | (tid & 31);
     float4 v[16];
 #pragma unroll
     for (int g = 0; g < 2; ++g) {
-        float4 *row = tile + (tid + 128 * g) * 8;
+        float4 *row = tile + (r0 + 32 * g) * 8;
 #pragma unroll
         for (int m = 0; m < 8; ++m) v[8 * g + m] = row[m ^ x];
     }
     if (FLIP) {
 #pragma unroll
         for (int g = 0; g < 2; ++g) {
-            const uint32_t w = sw[tid + 128 * g];
+            const uint32_t w = sw[r0 + 32 * g];
 #pragma unroll
             for (int m = 0; m < 8; ++m) v[8 * g + m] = flip4(v[8 * g + m], w >> (m * 4));
         }
@@ -355,7 +399,7 @@ __device__ __forceinline__ void pass_a_round1(float4 *tile, const uint32_t *sw, 
     }
 #pragma unroll
     for (int g = 0; g < 2; ++g) {
-        float4 *row = tile + (tid + 128 * g) * 8;
+        float4 *row = tile + (r0 + 32 * g) * 8;
 #pragma unroll
         for (int m = 0; m < 8; ++m) row[m ^ x] = v[8 * g + m];
     }
@@ -555,6 +599,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                                                    (size_t)(P.granularity + 1) * kLutRep * 16);
     __shared__ TaskInfo s_info[2];
     __shared__ __align__(8) uint64_t s_mbar[2];
+    __shared__ __align__(8) uint64_t s_done;           // one phase per finished task (compute warps arrive)
 
     const int tid = threadIdx.x;
     PipeCounters *pc = reinterpret_cast<PipeCounters *>(P.dev->counters);
@@ -567,6 +612,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
     if (tid == 0) {
         mbar_init(&s_mbar[0], 1);
         mbar_init(&s_mbar[1], 1);
+        mbar_init(&s_done, kPThreads);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (kCompress && !IDENTITY) {
@@ -585,13 +631,24 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
         const uint64_t pol_stream = make_evict_first_policy();   // gradients: read once
         const uint64_t pol_ring = make_evict_normal_policy();    // ring: written and read in L2
         uint32_t uses[2] = {0u, 0u};                  // TMA loads issued per slot so far
+        // Completion counter of the task last handed over in each slot (lane 0; null = none).
+        // The control warp signals completions, so the release fence is off the compute
+        // warps' critical path.  It learns of a finished task either from the hand-shake
+        // (the compute warps picked up the next task) or, while it waits for a dependency,
+        // from the s_done mbarrier: a dependency wait must never hold back the signal of an
+        // earlier task, which may be the very thing waited for.
+        uint32_t *pending[2] = {nullptr, nullptr};
         for (uint32_t i = 0;; ++i) {
             const int s = (int)(i & 1);
             // Task i is claimed once the compute warps have picked up task i-1, i.e. have
             // finished task i-2: buffer s and sign-word slot s are free.  One task of
             // look-ahead only: a deeper one stretches every task's claim-to-completion time,
-            // which is what dependent tasks wait for.
-            if (i >= 1) bar_sync(3 + (s ^ 1), kPCtaThreads);
+            // which is what dependent tasks wait for.  Task i-2 is signalled first: task i
+            // may depend on it.
+            if (i >= 1) {
+                bar_sync(3 + (s ^ 1), kPCtaThreads);
+                if (lane == 0 && pending[s] != nullptr) { red_release_add(pending[s], 1u); pending[s] = nullptr; }
+            }
             TaskInfo ti;
             ti.idx = 0xFFFFFFFFu; ti.is_b = 0; ti.wl = 0; ti.r = 0; ti.slot = 0; ti.gen = 0; ti.tma = 0; ti.phase = 0;
             if (lane == 0) {
@@ -601,13 +658,22 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     const TaskId t = decode_task(q, P);
                     const uint32_t *ctr = t.is_b ? &pc->a_done[t.slot] : &pc->b_done[t.slot];
                     const uint32_t target = t.is_b ? (t.gen + 1) * T : t.gen * T;
-                    if (target == 0 || wait_at_least(ctr, target, pc, P.dev)) {
+                    auto signal_previous = [&]() {            // task i-1 is the (i-1)-th phase of s_done
+                        if (pending[s ^ 1] != nullptr && mbar_test(&s_done, (uint32_t)(s ^ 1))) {
+                            red_release_add(pending[s ^ 1], 1u);
+                            pending[s ^ 1] = nullptr;
+                        }
+                    };
+                    if (target == 0 || wait_at_least(ctr, target, pc, P.dev, signal_previous)) {
                         ti.idx = t.idx;
                         ti.is_b = t.is_b;
                         ti.r = t.wb / P.n_local;
                         ti.wl = t.wb - ti.r * P.n_local;
                         ti.slot = t.slot;
                         ti.gen = t.gen;
+                        pending[s] = t.is_b ? &pc->b_done[t.slot] : &pc->a_done[t.slot];
+                        // the ring was written through the generic proxy; the TMA unit reads it
+                        if (t.is_b) fence_proxy_async_global();
                     }
                 }
             }
@@ -648,7 +714,12 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
             if (lane == 0) s_info[s] = ti;
             __syncwarp();
             bar_arrive(1 + s, kPCtaThreads);                  // slot s is full
-            if (idx == 0xFFFFFFFFu) break;
+            if (idx == 0xFFFFFFFFu) {
+                // "no task" is picked up once task i-1 is finished: signal it, then leave.
+                bar_sync(3 + s, kPCtaThreads);
+                if (lane == 0 && pending[s ^ 1] != nullptr) red_release_add(pending[s ^ 1], 1u);
+                break;
+            }
         }
     } else {
         // ============================================================ compute warps
@@ -732,29 +803,24 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
         fence_proxy_async();
         bar_arrive(3, kPCtaThreads);
 
-        bool aborted = false;
         for (uint32_t it = 0; me.idx != 0xFFFFFFFFu; ++it) {
             const int cur = (int)(it & 1);
             float4 *tile = bufs[cur];
-            if (!aborted) {
-                bool arrived = true;
-                if (me.tma) {
-                    arrived = mbar_wait(&s_mbar[cur], me.phase);
-                } else {
-                    load_tile(me, tile);
-                    cp_async_commit();
-                    cp_async_wait_all();
-                }
-                // tile visible to all compute warps.  A TMA load that never completed ends the
-                // launch: flag it, raise the abort flag, and from here on only keep the
-                // hand-shake with the control warp going until it hands over "no task".
-                aborted = compute_barrier_or(!arrived);
-                if (aborted && tid == 0) {
+            if (me.tma) {
+                // Every thread waits for the tile itself, so no block barrier is needed here.
+                // A load that never completes ends the launch: flag it and raise the abort
+                // flag; this task then runs on whatever the buffer holds (addresses do not
+                // depend on data) and the control warp claims nothing more.
+                if (!mbar_wait(&s_mbar[cur], me.phase)) {
                     atomicOr(&P.dev->status, THC_STATUS_WAIT_TIMEOUT);
                     atomicExch(&pc->abort, 1u);
                 }
+            } else {
+                load_tile(me, tile);
+                cp_async_commit();
+                cp_async_wait_all();
+                compute_barrier();
             }
-            if (!aborted) {
             const bool is_b = me.is_b != 0;
             const uint32_t wl = me.wl;
             const uint64_t r = me.r;
@@ -766,7 +832,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
             if (!is_b) {
                 // ================================ pass A: tile idx of worker-block wb
                 pass_a_round1<kCompress>(tile, sw + 256 * cur, tid);
-                compute_barrier();
+                __syncwarp();                          // the next round stays inside the warp's rows
                 round_rows_0_3(tile, tid);
                 compute_barrier();
                 pass_a_round3_store(tile, P.ring + (size_t)slot * B + ((size_t)idx << kPLog2), tid);
@@ -815,11 +881,10 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     }
                 }
             }
-            // every compute warp has issued its stores and is done with the tile and sign words
-            compute_barrier();
-            if (tid == 0) red_release_add(is_b ? &pc->b_done[slot] : &pc->a_done[slot], 1u);
-            }
-            // pick up the next task (only now: it may depend on the one just finished)
+            // Finished: tell the control warp (it signals the completion to the other CTAs),
+            // then pick up the next task.  The block-wide barrier means every compute warp
+            // has issued its stores and is done with the tile and the sign words.
+            mbar_arrive(&s_done);
             bar_sync(1 + (cur ^ 1), kPCtaThreads);
             me = s_info[cur ^ 1];
             fence_proxy_async();
