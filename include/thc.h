@@ -95,7 +95,7 @@ typedef struct thc_sizes_t {
     uint64_t rotated_bytes;    /* per worker, 4 * d_pad                                */
     uint64_t workspace_bytes;  /* scratch any call may need for this (d, n_local)      */
     uint32_t acc_bits;         /* the resolved accumulator width                       */
-    uint32_t reserved;
+    uint32_t fused_scales;     /* 1: thc_prepare_compress is one launch for (d, n_local)  */
 } thc_sizes_t;
 
 /* Validate `cfg` (host only) and build a context.  If a CUDA device is present, the
@@ -174,6 +174,20 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
 int thc_prepare_noalloc(const void *const *grads, uint32_t n, uint64_t d, uint32_t log2_block,
                         uint32_t in_dtype, double t_p, float *scales, uint32_t *status_or_null,
                         void *stream);
+
+/* thc_prepare and thc_compress in one launch, for callers that hold all n workers' gradients
+ * (the simulated cluster): same arguments and results as the two calls in a row, `scales`
+ * (device, nblocks floats) being written here and usable by thc_decompress afterwards.
+ * Section 5.3 observes that the norm exchange can overlap the RHT: only the quantiser needs M,
+ * so where the block size is 2^20, the input fp32 and n small enough for the intermediate ring
+ * to stay in L2, the transform kernel sums the squares of the tiles it loads anyway and the
+ * gradients are read from HBM once instead of twice.  Elsewhere this runs the two calls.
+ * The fp64 sums are added in a different (fixed) order than thc_prepare's, so a scale may
+ * differ from thc_prepare's in the last bit.  */
+int thc_prepare_compress(thc_ctx *ctx, const void *const *grads, uint32_t n, uint32_t worker_base,
+                         uint64_t d, uint32_t round, float *scales, void *const *packed,
+                         float *const *rotated_or_null, void *workspace, uint64_t workspace_bytes,
+                         void *stream);
 
 /* Error feedback (Section 5.1; Algorithm 3, "e_i = x_i - RHT^-1(X_i)"): for each of the n_local
  * workers, the residual between what it compressed and what its own indices stand for,

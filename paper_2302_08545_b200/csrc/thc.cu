@@ -753,6 +753,27 @@ static PipePlan plan_pipeline(const thc_ctx *ctx, uint64_t wb_count)
     return p;
 }
 
+// The same for the fused-scales kernel: pass B of a block can start only when all n workers'
+// tiles of the block are done, so it trails by n - 1 more worker-blocks and the ring grows by
+// as many slots.  Used only where that ring still fits comfortably in L2 and the per-block
+// counters (16 residues) cannot alias; otherwise the caller runs prepare and compress apart.
+static bool plan_pipeline_fused(const thc_ctx *ctx, uint64_t nblocks, uint32_t n, PipePlan *out)
+{
+    if (ctx->cfg.log2_block != 20 || ctx->cfg.in_dtype != THC_F32) return false;
+    const uint64_t wb_count = nblocks * n;
+    PipePlan p = plan_pipeline(ctx, wb_count);
+    const uint64_t window = p.ring - p.lag;
+    const uint64_t lag = (uint64_t)p.lag + n - 1;
+    const uint64_t ring = lag + window;
+    if (ring > wb_count || ring > (uint64_t)kMaxRing) return false;
+    if (ring * ((uint64_t)4 << 20) > ((uint64_t)96 << 20)) return false;
+    if ((ring + n - 1) / n + 2 > 16) return false;
+    p.lag = (uint32_t)lag;
+    p.ring = (uint32_t)ring;
+    *out = p;
+    return true;
+}
+
 int thc_sizes(const thc_ctx *ctx, uint64_t d, uint32_t n_local, thc_sizes_t *s)
 {
     if (ctx == nullptr || s == nullptr || d == 0 || n_local == 0 || n_local > THC_MAX_WORKERS)
@@ -773,6 +794,12 @@ int thc_sizes(const thc_ctx *ctx, uint64_t d, uint32_t n_local, thc_sizes_t *s)
     if (k > (uint32_t)kTileLog2) {
         const PipePlan pl = plan_pipeline(ctx, s->nblocks * n_local);
         two_pass_ws = (uint64_t)pl.ring * B * 4;
+        PipePlan pf;
+        if (plan_pipeline_fused(ctx, s->nblocks, n_local, &pf)) {
+            const uint64_t fused_ws = (uint64_t)pf.ring * B * 4 + s->nblocks * n_local * (B >> kPLog2) * 8;
+            if (fused_ws > two_pass_ws) two_pass_ws = fused_ws;
+            s->fused_scales = 1;
+        }
     }
     // scratch of prepare / the pipeline's ring, then one worker's table values (error feedback)
     s->workspace_bytes = round_up((prepare_ws > two_pass_ws ? prepare_ws : two_pass_ws) + 256, 256) +
@@ -920,7 +947,7 @@ typedef void (*pipe_kernel_t)(const TmaMaps, PipeParams, PtrArrayP, MutPtrArrayP
 template <int MODE, int KB>
 static pipe_kernel_t pick_pipe_kernel_kb(uint32_t bits, bool identity)
 {
-    if constexpr (MODE != kCompressF32 && MODE != kCompressBF16) {
+    if constexpr (MODE != kCompressF32 && MODE != kCompressBF16 && MODE != kCompressF32Fused) {
         return thc_pipeline_kernel<MODE, 4, true, KB>;
     } else {
         switch (bits) {
@@ -979,7 +1006,8 @@ static int encode_map(CUtensorMap *map, const void *base, uint64_t cols, uint64_
 static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress_f32,
                            const thc_sizes_t &sz, uint64_t d, uint32_t n_local, uint32_t worker_base, uint32_t round, uint32_t divisor,
                            const float *scales, void *workspace, const PtrArrayP &in,
-                           const MutPtrArrayP &out, const MutPtrArrayP &rot, cudaStream_t st)
+                           const MutPtrArrayP &out, const MutPtrArrayP &rot, cudaStream_t st,
+                           float *fused_scales_out = nullptr)
 {
     const uint32_t k = ctx->cfg.log2_block;
     PipeParams P;
@@ -990,7 +1018,14 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
     const uint64_t T = 1ull << (k - kPLog2);
     P.total_tasks = P.wb_count * T * 2;
     if (P.wb_count >= 0x7FFFFFFFull || P.total_tasks >= 0x7FFFFFFFull) return THC_EUNSUPPORTED;
-    const PipePlan pl = plan_pipeline(ctx, P.wb_count);
+    PipePlan pl = plan_pipeline(ctx, P.wb_count);
+    if (fused_scales_out != nullptr) {
+        if (!plan_pipeline_fused(ctx, sz.nblocks, n_local, &pl)) return THC_EUNSUPPORTED;
+        P.tile_sq = reinterpret_cast<double *>(static_cast<unsigned char *>(workspace) +
+                                               ((uint64_t)pl.ring << k) * 4);
+        P.scales_out = fused_scales_out;
+        P.t_p = ctx->cfg.t_p;
+    }
     P.ring = static_cast<float *>(workspace);
     P.scales = scales;
     P.dev = ctx->dev;
@@ -1082,6 +1117,46 @@ int thc_compress(thc_ctx *ctx, const void *const *grads, uint32_t n_local, uint3
                               : pick_pipe_kernel<kCompressF32>(ctx->cfg.bits, ctx->identity, k);
     return launch_pipeline(ctx, kern, !bf16, sz, d, n_local, worker_base, round, 1, scales, workspace,
                            pin, pout, prot, st);
+}
+
+// Scales and compress in one launch (see thc.h).  Falls back to the two separate calls where
+// the fused kernel does not apply.
+int thc_prepare_compress(thc_ctx *ctx, const void *const *grads, uint32_t n, uint32_t worker_base,
+                         uint64_t d, uint32_t round, float *scales, void *const *packed,
+                         float *const *rotated, void *workspace, uint64_t workspace_bytes, void *stream)
+{
+    int rc = check_launch_ctx(ctx);
+    if (rc != THC_OK) return rc;
+    thc_sizes_t sz;
+    if ((rc = thc_sizes(ctx, d, n, &sz)) != THC_OK) return rc;
+    PipePlan pf;
+    if (!plan_pipeline_fused(ctx, sz.nblocks, n, &pf)) {
+        rc = thc_prepare(ctx, grads, n, d, scales, workspace, workspace_bytes, stream);
+        if (rc != THC_OK) return rc;
+        return thc_compress(ctx, grads, n, worker_base, d, round, scales, packed, rotated, workspace,
+                            workspace_bytes, stream);
+    }
+    if ((rc = check_ptr_array(grads, n)) != THC_OK) return rc;
+    if ((rc = check_ptr_array(packed, n)) != THC_OK) return rc;
+    if (scales == nullptr || workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
+    if ((uint64_t)worker_base + n > 0xFFFFFFFFull) return THC_EINVAL;
+    if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
+    PtrArrayP pin;
+    MutPtrArrayP pout, prot;
+    memset(&pin, 0, sizeof pin);
+    memset(&pout, 0, sizeof pout);
+    memset(&prot, 0, sizeof prot);
+    for (uint32_t i = 0; i < n; ++i) {
+        pin.p[i] = grads[i];
+        pout.p[i] = packed[i];
+        if (rotated != nullptr && rotated[i] != nullptr) {
+            if (!aligned16(rotated[i])) return THC_EINVAL;
+            prot.p[i] = rotated[i];
+        }
+    }
+    pipe_kernel_t kern = pick_pipe_kernel_kb<kCompressF32Fused, 7>(ctx->cfg.bits, ctx->identity);
+    return launch_pipeline(ctx, kern, true, sz, d, n, worker_base, round, 1, scales, workspace, pin, pout,
+                           prot, static_cast<cudaStream_t>(stream), scales);
 }
 
 int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, uint32_t round,

@@ -21,6 +21,16 @@
 // compute warps wait for the data, run the rounds and signal completion.  Tiles sit in shared
 // memory in TMA's 128-byte swizzle: 16-byte chunk c at c ^ ((c >> 3) & 7).
 //
+// Fused scales (kCompressF32Fused; Section 5.3 notes that the norm exchange can run beside the
+// RHT).  Pass A does not need the clamp bound M, only the epilogue of pass B does.  So every
+// pass-A task also sums the squares of its tile in fp64; the control warp stores the sum,
+// counts finished tiles per RHT block, and the CTA that finishes the last of a block's
+// n_local * T tiles computes M = t_p * max_i ||x_i|| / sqrt(B) from the stored sums in a fixed
+// order, writes it to `scales` and releases the block's pass-B tasks.  The queue trails pass B
+// behind pass A by n_local - 1 more worker-blocks so that this is normally done in time.
+// In this mode a_done[0..15] count finished tiles of block r in entry r mod 16 and
+// a_done[16..31] count finished blocks of that residue.
+//
 // Counters (in the context's device block, all zero between launches; the last CTA to leave
 // clears them):  head, exited, abort, a_done[R], b_done[R].  a_done[s] counts finished A tiles
 // of slot s over the whole launch (generation g of the slot is complete at (g+1)*T),
@@ -41,16 +51,22 @@ constexpr int kMaxRing = 56;
 constexpr int kBlockConstMax = 256;         // per-block constants cached in shared memory
 constexpr uint32_t kMaxPolls = 1u << 21;
 
-enum PipeMode { kCompressF32, kCompressBF16, kDecompress8, kDecompress16, kDecompress32 };
+enum PipeMode { kCompressF32, kCompressBF16, kDecompress8, kDecompress16, kDecompress32,
+                kCompressF32Fused };   // fp32 compress that also computes the block scales (below)
 
-struct PipeCounters {          // layout inside DeviceBlock::counters
-    uint32_t head;
-    uint32_t exited;
-    uint32_t abort;
-    uint32_t pad;
-    uint32_t a_done[kMaxRing];
-    uint32_t b_done[kMaxRing];
+// Layout inside DeviceBlock::counters.  Every CTA hits `head` and `abort` for every task and
+// the completion counters of the slots in use: each gets its own 128-byte line (head, exited,
+// abort) or 32-byte sector (per-slot counters), so that polls of one do not queue behind
+// atomics on another.
+struct alignas(32) PaddedCounter { uint32_t v; uint32_t pad[7]; };
+struct PipeCounters {
+    uint32_t head;   uint32_t pad0[31];
+    uint32_t exited; uint32_t pad1[31];
+    uint32_t abort;  uint32_t pad2[31];
+    PaddedCounter a_done[kMaxRing];
+    PaddedCounter b_done[kMaxRing];
 };
+static_assert(sizeof(PipeCounters) <= sizeof(DeviceBlock::counters), "counters do not fit the device block");
 
 struct PipeParams {
     uint64_t d;
@@ -70,6 +86,10 @@ struct PipeParams {
     uint32_t round;
     uint32_t worker_base;
     float    c_block;
+    // fused scales only
+    double  *tile_sq;          // wb_count * T sums of squares, one per pass-A tile
+    float   *scales_out;       // = scales, written by the kernel
+    double   t_p;
 };
 
 struct PtrArrayP { const void *p[THC_MAX_WORKERS]; };
@@ -84,6 +104,7 @@ struct TaskInfo {              // published by thread 0 for the whole CTA
     uint32_t gen;              // generation of the slot
     uint32_t tma;              // tile arrives by TMA on the slot's mbarrier
     uint32_t phase;            // ... with this phase parity
+    float    bcx, bcy;         // block constants (fused scales: they do not exist at launch)
 };
 
 struct TmaMaps {               // tensor maps: one per worker gradient, one for the ring
@@ -104,24 +125,6 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p)
     uint32_t v;
     asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
-}
-
-// Bounded wait (one thread): true once *ctr >= target; false if the launch was aborted or
-// the wait expired (then the timeout bit and the abort flag are set).  on_poll() runs between
-// polls: the waiting thread keeps its other duty (signalling finished tasks) alive.
-template <class F>
-__device__ __forceinline__ bool wait_at_least(const uint32_t *ctr, uint32_t target,
-                                              PipeCounters *pc, DeviceBlock *dev, F on_poll)
-{
-    for (uint32_t it = 0; it < kMaxPolls; ++it) {
-        if (ld_acquire_u32(ctr) >= target) return true;
-        if (ld_relaxed_u32(&pc->abort) != 0) return false;
-        on_poll();
-        __nanosleep(it < 32 ? 20 : 200);
-    }
-    atomicOr(&dev->status, THC_STATUS_WAIT_TIMEOUT);
-    atomicExch(&pc->abort, 1u);
-    return false;
 }
 
 __device__ __forceinline__ uint64_t make_evict_first_policy()
@@ -173,6 +176,20 @@ __device__ __forceinline__ bool compute_barrier_or(bool pred)
                  "barrier.cta.red.or.pred q, 5, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
                  : "=r"(out) : "r"((uint32_t)pred), "r"(kPThreads) : "memory");
     return out != 0;
+}
+
+__device__ __forceinline__ uint32_t atom_release_add(uint32_t *p, uint32_t v)
+{
+    uint32_t old;
+    asm volatile("atom.release.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
+
+__device__ __forceinline__ float ld_relaxed_f32(const float *p)
+{
+    float v;
+    asm volatile("ld.relaxed.gpu.global.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+    return v;
 }
 
 __device__ __forceinline__ void red_release_add(uint32_t *p, uint32_t v)
@@ -369,8 +386,10 @@ __device__ __forceinline__ void p_rounds(float4 *tile, int lo, int hi, int tid)
 // then stride 4, 8, 16 across the eight chunks of a row.  Thread (warp w, lane l) owns rows
 // 64 w + l and 64 w + 32 + l: a warp works on the same 64 rows here and in the next round
 // (round_rows_0_3), so only a warp barrier separates the two.
-template <bool FLIP>
-__device__ __forceinline__ void pass_a_round1(float4 *tile, const uint32_t *sw, int tid)
+// With SQ the thread's sum of squares of the 64 inputs (fp64, four interleaved partial
+// sums combined in a fixed order) is returned.
+template <bool FLIP, bool SQ>
+__device__ __forceinline__ double pass_a_round1(float4 *tile, const uint32_t *sw, int tid)
 {
     const int x = tid & 7;
     const int r0 = ((tid >> 5) << 6) | (tid & 31);
@@ -380,6 +399,18 @@ __device__ __forceinline__ void pass_a_round1(float4 *tile, const uint32_t *sw, 
         float4 *row = tile + (r0 + 32 * g) * 8;
 #pragma unroll
         for (int m = 0; m < 8; ++m) v[8 * g + m] = row[m ^ x];
+    }
+    double sq = 0.0;
+    if (SQ) {
+        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+#pragma unroll
+        for (int m = 0; m < 16; ++m) {
+            a0 = fma((double)v[m].x, (double)v[m].x, a0);
+            a1 = fma((double)v[m].y, (double)v[m].y, a1);
+            a2 = fma((double)v[m].z, (double)v[m].z, a2);
+            a3 = fma((double)v[m].w, (double)v[m].w, a3);
+        }
+        sq = (a0 + a1) + (a2 + a3);
     }
     if (FLIP) {
 #pragma unroll
@@ -403,6 +434,7 @@ __device__ __forceinline__ void pass_a_round1(float4 *tile, const uint32_t *sw, 
 #pragma unroll
         for (int m = 0; m < 8; ++m) row[m ^ x] = v[8 * g + m];
     }
+    return sq;
 }
 
 // Round on row bits 0..3: thread (rg = tid >> 3, cc = tid & 7) owns chunk cc of rows
@@ -585,7 +617,9 @@ __global__ void __launch_bounds__(kPCtaThreads, 3)
 thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArrayP in,
                     MutPtrArrayP outp, MutPtrArrayP rotated, PhiloxKeys keys)
 {
-    constexpr bool kCompress = MODE == kCompressF32 || MODE == kCompressBF16;
+    constexpr bool kFused = MODE == kCompressF32Fused;
+    constexpr bool kF32In = MODE == kCompressF32 || kFused;
+    constexpr bool kCompress = kF32In || MODE == kCompressBF16;
     extern __shared__ __align__(1024) unsigned char pipe_smem_raw[];
     // TMA's 128-byte swizzle needs the tile buffers on 1024-byte boundaries of the shared
     // address space; the launch reserves 1 KB of slack for this round-up.
@@ -600,6 +634,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
     __shared__ TaskInfo s_info[2];
     __shared__ __align__(8) uint64_t s_mbar[2];
     __shared__ __align__(8) uint64_t s_done;           // one phase per finished task (compute warps arrive)
+    __shared__ double s_sq[2][kPThreads / 32];          // fused scales: per-warp sums of squares of a tile
 
     const int tid = threadIdx.x;
     PipeCounters *pc = reinterpret_cast<PipeCounters *>(P.dev->counters);
@@ -621,8 +656,10 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
     }
     const uint32_t nblk_total = (uint32_t)(P.d_pad >> P.k);
     const uint32_t nblk_cached = nblk_total < (uint32_t)kBlockConstMax ? nblk_total : (uint32_t)kBlockConstMax;
-    for (uint32_t b = tid; b < nblk_cached; b += kPCtaThreads)
-        blk_const[b] = block_constants<kCompress>(P.scales[b], P.granularity, P.divisor);
+    if (!kFused) {
+        for (uint32_t b = tid; b < nblk_cached; b += kPCtaThreads)
+            blk_const[b] = block_constants<kCompress>(P.scales[b], P.granularity, P.divisor);
+    }
     __syncthreads();
 
     if (tid >= kPThreads) {
@@ -631,13 +668,70 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
         const uint64_t pol_stream = make_evict_first_policy();   // gradients: read once
         const uint64_t pol_ring = make_evict_normal_policy();    // ring: written and read in L2
         uint32_t uses[2] = {0u, 0u};                  // TMA loads issued per slot so far
-        // Completion counter of the task last handed over in each slot (lane 0; null = none).
-        // The control warp signals completions, so the release fence is off the compute
-        // warps' critical path.  It learns of a finished task either from the hand-shake
-        // (the compute warps picked up the next task) or, while it waits for a dependency,
-        // from the s_done mbarrier: a dependency wait must never hold back the signal of an
-        // earlier task, which may be the very thing waited for.
-        uint32_t *pending[2] = {nullptr, nullptr};
+        // The task last handed over in each slot whose completion is not yet signalled
+        // (warp-uniform).  The control warp signals completions, so the release fence is off
+        // the compute warps' critical path.  It learns of a finished task either from the
+        // hand-shake (the compute warps picked up the next task) or, while it waits for a
+        // dependency, from the s_done mbarrier: a dependency wait must never hold back the
+        // signal of an earlier task, which may be the very thing waited for.
+        TaskId pend[2];
+        bool pend_valid[2] = {false, false};
+        pend[0].wb = pend[0].idx = pend[0].is_b = pend[0].slot = pend[0].gen = 0;
+        pend[1] = pend[0];
+
+        // Warp-wide: publish the completion of task t (whose sums of squares sit in s_sq[sq]).
+        // Fused scales: the warp that counts the last tile of an RHT block computes the block's
+        // M from the stored sums (fixed order) and releases the block's pass-B tasks.
+        auto complete = [&](const TaskId &t, int sq) {
+            if (!kFused || t.is_b) {
+                if (lane == 0) red_release_add(t.is_b ? &pc->b_done[t.slot].v : &pc->a_done[t.slot].v, 1u);
+                return;
+            }
+            const uint32_t r = t.wb / P.n_local;
+            uint32_t old = 0;
+            if (lane == 0) {
+                const double tile_sum = (s_sq[sq][0] + s_sq[sq][1]) + (s_sq[sq][2] + s_sq[sq][3]);
+                __stcg(P.tile_sq + (((size_t)t.wb << kb) + t.idx), tile_sum);
+                old = atom_release_add(&pc->a_done[r & 15u].v, 1u);
+            }
+            old = __shfl_sync(0xFFFFFFFFu, old, 0);
+            if (old + 1u != (r / 16u + 1u) * P.n_local * T) return;
+            __threadfence();                           // the other tiles' sums, after seeing the count
+            double ell = 0.0;
+            for (uint32_t i0 = 0; i0 < P.n_local; i0 += 8u) {
+                // eight workers at a time: all loads in flight together (T = 128: four per lane)
+                double v[8][4];
+#pragma unroll
+                for (int w = 0; w < 8; ++w) {
+                    const uint32_t i = i0 + w < P.n_local ? i0 + w : P.n_local - 1u;
+                    const double *p = P.tile_sq + ((size_t)(r * P.n_local + i) << kb);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t c2 = (uint32_t)lane + 32u * j;
+                        v[w][j] = c2 < T ? __ldcg(p + c2) : 0.0;
+                    }
+                }
+#pragma unroll
+                for (int w = 0; w < 8; ++w) {
+                    double acc = 0.0;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc += v[w][j];
+                    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+                    const double norm = sqrt(acc);
+                    if (i0 + w < P.n_local && (norm > ell || norm != norm)) ell = norm;   // a NaN norm sticks
+                }
+            }
+            if (lane == 0) {
+                float M = (float)(P.t_p * ell / sqrt((double)B));
+                uint32_t flags = 0;
+                if (!isfinite(M)) { M = 0.0f; flags |= THC_STATUS_NONFINITE; }
+                if (M == 0.0f) flags |= THC_STATUS_ZERO_BLOCK;
+                __stcg(P.scales_out + r, M);
+                if (flags) atomicOr(&P.dev->status, flags);
+                red_release_add(&pc->a_done[16u + (r & 15u)].v, 1u);
+            }
+        };
+
         for (uint32_t i = 0;; ++i) {
             const int s = (int)(i & 1);
             // Task i is claimed once the compute warps have picked up task i-1, i.e. have
@@ -647,77 +741,112 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
             // may depend on it.
             if (i >= 1) {
                 bar_sync(3 + (s ^ 1), kPCtaThreads);
-                if (lane == 0 && pending[s] != nullptr) { red_release_add(pending[s], 1u); pending[s] = nullptr; }
+                if (pend_valid[s]) { complete(pend[s], s); pend_valid[s] = false; }
+            }
+            uint32_t q = 0, ab = 0;
+            if (lane == 0) {
+                q = atomicAdd(&pc->head, 1u);
+                ab = ld_relaxed_u32(&pc->abort);
+            }
+            q = __shfl_sync(0xFFFFFFFFu, q, 0);
+            ab = __shfl_sync(0xFFFFFFFFu, ab, 0);
+            bool have = (uint64_t)q < P.total_tasks && ab == 0;
+            TaskId t;
+            t.wb = t.idx = t.is_b = t.slot = t.gen = 0;
+            uint32_t r = 0, tma = 0, phase = 0;            // tma, phase: lane 0
+            if (have) {
+                t = decode_task(q, P);
+                r = t.wb / P.n_local;
+                const uint32_t wl = t.wb - r * P.n_local;
+                const uint64_t j0 = (uint64_t)r * B + ((uint64_t)t.idx << kPLog2);
+                if (!t.is_b) {
+                    // pass A reads only the caller's input: start the load before looking at
+                    // the ring slot, which only the end of the task writes to
+                    if (kCompress) {
+                        // sign words of the tile: 64 Philox calls, two per lane
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            const int call = lane + 32 * c;
+                            const uint4 ph = sign_call(j0 + 128ull * call, P.round, keys);
+                            *reinterpret_cast<uint4 *>(sw + 256 * s + 4 * call) = ph;
+                        }
+                    }
+                    if (lane == 0 && kF32In && (j0 >> 5) + 256 <= d_rows32) {
+                        mbar_expect_tx(&s_mbar[s], kPElems * 4);
+                        tma_load_2d(bufs[s], &maps.in[wl], 0, (int)(j0 >> 5), &s_mbar[s], pol_stream);
+                        tma = 1; phase = uses[s] & 1u; ++uses[s];
+                    }
+                }
+                // pass B needs its worker-block's tiles (fused scales: the block's M, which
+                // implies them); pass A needs the previous tenant of its ring slot consumed
+                const uint32_t *ctr = !t.is_b ? &pc->b_done[t.slot].v
+                                      : kFused ? &pc->a_done[16u + (r & 15u)].v : &pc->a_done[t.slot].v;
+                const uint32_t target = !t.is_b ? t.gen * T : kFused ? r / 16u + 1u : (t.gen + 1) * T;
+                if (target != 0) {
+                    have = false;
+                    bool expired = true;
+                    for (uint32_t it = 0; it < kMaxPolls; ++it) {
+                        uint32_t v = 0, a2 = 0;
+                        if (lane == 0) { v = ld_acquire_u32(ctr); a2 = ld_relaxed_u32(&pc->abort); }
+                        v = __shfl_sync(0xFFFFFFFFu, v, 0);
+                        a2 = __shfl_sync(0xFFFFFFFFu, a2, 0);
+                        if (v >= target) { have = true; expired = false; break; }
+                        if (a2 != 0) { expired = false; break; }
+                        if (pend_valid[s ^ 1]) {               // task i-1 is phase i-1 of s_done
+                            uint32_t fin = lane == 0 ? (uint32_t)mbar_test(&s_done, (uint32_t)(s ^ 1)) : 0u;
+                            fin = __shfl_sync(0xFFFFFFFFu, fin, 0);
+                            if (fin) { complete(pend[s ^ 1], s ^ 1); pend_valid[s ^ 1] = false; }
+                        }
+                        __nanosleep(it < 32 ? 20 : 200);
+                    }
+                    if (expired && lane == 0) {
+                        atomicOr(&P.dev->status, THC_STATUS_WAIT_TIMEOUT);
+                        atomicExch(&pc->abort, 1u);
+                    }
+                    // giving up with the tile's copy in flight: let it land before leaving
+                    if (!have && lane == 0 && tma) (void)mbar_wait(&s_mbar[s], phase);
+                }
             }
             TaskInfo ti;
             ti.idx = 0xFFFFFFFFu; ti.is_b = 0; ti.wl = 0; ti.r = 0; ti.slot = 0; ti.gen = 0; ti.tma = 0; ti.phase = 0;
-            if (lane == 0) {
-                const uint32_t q = atomicAdd(&pc->head, 1u);
-                const uint32_t aborted = ld_relaxed_u32(&pc->abort);
-                if ((uint64_t)q < P.total_tasks && aborted == 0) {
-                    const TaskId t = decode_task(q, P);
-                    const uint32_t *ctr = t.is_b ? &pc->a_done[t.slot] : &pc->b_done[t.slot];
-                    const uint32_t target = t.is_b ? (t.gen + 1) * T : t.gen * T;
-                    auto signal_previous = [&]() {            // task i-1 is the (i-1)-th phase of s_done
-                        if (pending[s ^ 1] != nullptr && mbar_test(&s_done, (uint32_t)(s ^ 1))) {
-                            red_release_add(pending[s ^ 1], 1u);
-                            pending[s ^ 1] = nullptr;
-                        }
-                    };
-                    if (target == 0 || wait_at_least(ctr, target, pc, P.dev, signal_previous)) {
-                        ti.idx = t.idx;
-                        ti.is_b = t.is_b;
-                        ti.r = t.wb / P.n_local;
-                        ti.wl = t.wb - ti.r * P.n_local;
-                        ti.slot = t.slot;
-                        ti.gen = t.gen;
-                        pending[s] = t.is_b ? &pc->b_done[t.slot] : &pc->a_done[t.slot];
-                        // the ring was written through the generic proxy; the TMA unit reads it
-                        if (t.is_b) fence_proxy_async_global();
+            ti.bcx = 0.f; ti.bcy = 0.f;
+            if (have) {
+                ti.idx = t.idx;
+                ti.is_b = t.is_b;
+                ti.r = r;
+                ti.wl = t.wb - r * P.n_local;
+                ti.slot = t.slot;
+                ti.gen = t.gen;
+                pend[s] = t;
+                pend_valid[s] = true;
+                if (lane == 0 && t.is_b) {
+                    if (kFused) {
+                        const float2 c = block_constants<true>(ld_relaxed_f32(P.scales + r), P.granularity, P.divisor);
+                        ti.bcx = c.x; ti.bcy = c.y;
                     }
-                }
-            }
-            const uint32_t idx = __shfl_sync(0xFFFFFFFFu, ti.idx, 0);
-            const uint32_t is_b = __shfl_sync(0xFFFFFFFFu, ti.is_b, 0);
-            const uint32_t r = __shfl_sync(0xFFFFFFFFu, ti.r, 0);
-            if (idx != 0xFFFFFFFFu) {
-                const uint64_t j0 = (uint64_t)r * B + ((uint64_t)idx << kPLog2);
-                if (kCompress && !is_b) {
-                    // sign words of the tile: 64 Philox calls, two per lane
-#pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        const int call = lane + 32 * c;
-                        const uint4 ph = sign_call(j0 + 128ull * call, P.round, keys);
-                        *reinterpret_cast<uint4 *>(sw + 256 * s + 4 * call) = ph;
-                    }
-                }
-                if (lane == 0) {
-                    if (is_b) {
-                        if (KB == 7) {
-                            // panel: 128 ring rows x 64 columns, as two boxes of 32 columns
-                            mbar_expect_tx(&s_mbar[s], kPElems * 4);
-                            const int x0 = (int)(idx << 6);
-                            const int y0 = (int)(ti.slot << 7);
-                            tma_load_2d(bufs[s], &maps.ring, x0, y0, &s_mbar[s], pol_ring);
-                            tma_load_2d(bufs[s] + 1024, &maps.ring, x0 + 32, y0, &s_mbar[s], pol_ring);
-                            ti.tma = 1;
-                        }
-                    } else if (MODE == kCompressF32 && (j0 >> 5) + 256 <= d_rows32) {
+                    // the ring was written through the generic proxy; the TMA unit reads it
+                    fence_proxy_async_global();
+                    if (KB == 7) {
+                        // panel: 128 ring rows x 64 columns, as two boxes of 32 columns
                         mbar_expect_tx(&s_mbar[s], kPElems * 4);
-                        tma_load_2d(bufs[s], &maps.in[ti.wl], 0, (int)(j0 >> 5), &s_mbar[s], pol_stream);
-                        ti.tma = 1;
+                        const int x0 = (int)(t.idx << 6);
+                        const int y0 = (int)(t.slot << 7);
+                        tma_load_2d(bufs[s], &maps.ring, x0, y0, &s_mbar[s], pol_ring);
+                        tma_load_2d(bufs[s] + 1024, &maps.ring, x0 + 32, y0, &s_mbar[s], pol_ring);
+                        tma = 1; phase = uses[s] & 1u; ++uses[s];
                     }
-                    if (ti.tma) { ti.phase = uses[s] & 1u; ++uses[s]; }
                 }
+                ti.tma = tma;
+                ti.phase = phase;
             }
             __syncwarp();
             if (lane == 0) s_info[s] = ti;
             __syncwarp();
             bar_arrive(1 + s, kPCtaThreads);                  // slot s is full
-            if (idx == 0xFFFFFFFFu) {
+            if (!have) {
                 // "no task" is picked up once task i-1 is finished: signal it, then leave.
                 bar_sync(3 + s, kPCtaThreads);
-                if (lane == 0 && pending[s ^ 1] != nullptr) red_release_add(pending[s ^ 1], 1u);
+                if (pend_valid[s ^ 1]) complete(pend[s ^ 1], s ^ 1);
                 break;
             }
         }
@@ -738,7 +867,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 return;
             }
             const uint64_t j0 = (uint64_t)ti.r * B + ((uint64_t)ti.idx << kPLog2);
-            if (MODE == kCompressF32) {
+            if (kF32In) {
                 const float *x = static_cast<const float *>(in.p[ti.wl]);
 #pragma unroll 4
                 for (int i = 0; i < kPChunks / kPThreads; ++i) {
@@ -826,12 +955,17 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
             const uint64_t r = me.r;
             const uint32_t slot = me.slot;
             const uint32_t idx = me.idx;
-            const float2 bc = r < nblk_cached ? blk_const[r]
-                                              : block_constants<kCompress>(P.scales[r], P.granularity, P.divisor);
+            const float2 bc = kFused ? make_float2(me.bcx, me.bcy)
+                              : r < nblk_cached ? blk_const[r]
+                                                : block_constants<kCompress>(P.scales[r], P.granularity, P.divisor);
 
             if (!is_b) {
                 // ================================ pass A: tile idx of worker-block wb
-                pass_a_round1<kCompress>(tile, sw + 256 * cur, tid);
+                double sq = pass_a_round1<kCompress, kFused>(tile, sw + 256 * cur, tid);
+                if (kFused) {
+                    for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, off);
+                    if ((tid & 31) == 0) s_sq[cur][tid >> 5] = sq;
+                }
                 __syncwarp();                          // the next round stays inside the warp's rows
                 round_rows_0_3(tile, tid);
                 compute_barrier();
@@ -898,7 +1032,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
         __threadfence();
         const uint32_t left = atomicAdd(&pc->exited, 1u);
         if (left == gridDim.x - 1) {
-            for (int sl = 0; sl < kMaxRing; ++sl) { pc->a_done[sl] = 0; pc->b_done[sl] = 0; }
+            for (int sl = 0; sl < kMaxRing; ++sl) { pc->a_done[sl].v = 0; pc->b_done[sl].v = 0; }
             pc->abort = 0;
             pc->head = 0;
             __threadfence();

@@ -57,6 +57,10 @@ class Round:
         self.ctx.compress(self.grads, self.d, rnd, self.scales, self.packed, self.workspace,
                           rotated=self.rotated, stream=stream)
 
+    def prepare_compress(self, rnd: int = 0, stream=None):
+        self.ctx.prepare_compress(self.grads, self.d, rnd, self.scales, self.packed, self.workspace,
+                                  rotated=self.rotated, stream=stream)
+
     def aggregate(self, stream=None):
         self.ctx.aggregate(self.packed, self.d, self.total, stream)
 
@@ -64,9 +68,12 @@ class Round:
         self.ctx.decompress(self.total, self.n, self.d, rnd, self.scales, self.out,
                             self.workspace, stream)
 
-    def run(self, rnd: int = 0, with_prepare: bool = True, stream=None):
-        if with_prepare:
-            self.prepare(stream)
-        self.compress(rnd, stream)
+    def run(self, rnd: int = 0, with_prepare: bool = True, stream=None, fused: bool = False):
+        if with_prepare and fused:
+            self.prepare_compress(rnd, stream)
+        else:
+            if with_prepare:
+                self.prepare(stream)
+            self.compress(rnd, stream)
         self.aggregate(stream)
         self.decompress(rnd, stream)

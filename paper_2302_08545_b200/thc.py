@@ -21,7 +21,7 @@ STATUS_NONFINITE, STATUS_ZERO_BLOCK, STATUS_WAIT_TIMEOUT = 1, 2, 4
 
 EXPORTS = ("thc_create", "thc_destroy", "thc_sizes", "thc_prepare", "thc_compress",
            "thc_quantize_rotated", "thc_aggregate", "thc_decompress", "thc_prepare_noalloc",
-           "thc_error_feedback", "thc_accumulate_error", "thc_debug_skip_tasks", "thc_status", "thc_strerror", "thc_version")
+           "thc_error_feedback", "thc_accumulate_error", "thc_prepare_compress", "thc_debug_skip_tasks", "thc_status", "thc_strerror", "thc_version")
 NOALLOC_SCRATCH_BYTES = 4 << 20
 
 
@@ -43,7 +43,7 @@ class _Sizes(ctypes.Structure):
     _fields_ = [("d_pad", ctypes.c_uint64), ("nblocks", ctypes.c_uint64),
                 ("packed_bytes", ctypes.c_uint64), ("sum_bytes", ctypes.c_uint64),
                 ("rotated_bytes", ctypes.c_uint64), ("workspace_bytes", ctypes.c_uint64),
-                ("acc_bits", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+                ("acc_bits", ctypes.c_uint32), ("fused_scales", ctypes.c_uint32)]
 
 
 @dataclass(frozen=True)
@@ -55,6 +55,7 @@ class Sizes:
     rotated_bytes: int
     workspace_bytes: int
     acc_bits: int
+    fused_scales: int = 0
 
 
 def lib():
@@ -77,6 +78,7 @@ def lib():
     L.thc_aggregate.argtypes = [vp, pp, u32, u64, vp, vp]
     L.thc_decompress.argtypes = [vp, vp, u32, u64, u32, vp, vp, vp, u64, vp]
     L.thc_prepare_noalloc.argtypes = [pp, u32, u64, u32, u32, ctypes.c_double, vp, vp, vp]
+    L.thc_prepare_compress.argtypes = [vp, pp, u32, u32, u64, u32, vp, pp, pp, vp, u64, vp]
     L.thc_error_feedback.argtypes = [vp, pp, pp, u32, u64, u32, vp, pp, vp, u64, vp]
     L.thc_accumulate_error.argtypes = [vp, pp, pp, u32, u64, vp]
     L.thc_debug_skip_tasks.argtypes = [vp, u32]
@@ -171,7 +173,7 @@ class Context:
         s = _Sizes()
         _check(lib().thc_sizes(self._h, d, n_local, ctypes.byref(s)), "thc_sizes")
         return Sizes(s.d_pad, s.nblocks, s.packed_bytes, s.sum_bytes, s.rotated_bytes,
-                     s.workspace_bytes, s.acc_bits)
+                     s.workspace_bytes, s.acc_bits, s.fused_scales)
 
     def prepare(self, grads, d: int, scales, workspace, stream=None):
         arr = _ptr_array([_dp(g) for g in grads])
@@ -188,6 +190,16 @@ class Context:
         ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
         _check(lib().thc_compress(self._h, ga, n, worker_base, d, rnd, _dp(scales), pa, ra,
                                   _dp(workspace), ws_bytes, _stream(stream)), "thc_compress")
+
+    def prepare_compress(self, grads, d: int, rnd: int, scales, packed, workspace, rotated=None,
+                         worker_base: int = 0, stream=None):
+        n = len(grads)
+        ga = _ptr_array([_dp(g) for g in grads])
+        pa = _ptr_array([_dp(p) for p in packed])
+        ra = _ptr_array([_dp(r) for r in rotated]) if rotated is not None else None
+        _check(lib().thc_prepare_compress(self._h, ga, n, worker_base, d, rnd, _dp(scales), pa, ra,
+                                          _dp(workspace), workspace.numel() * workspace.element_size(),
+                                          _stream(stream)), "thc_prepare_compress")
 
     def quantize_rotated(self, rotated, d: int, rnd: int, scales, packed, worker_base: int = 0,
                          stream=None):

@@ -290,3 +290,77 @@ def test_error_feedback_matches_oracle(k, d, n):
     torch.cuda.synchronize()
     for i in range(n):
         assert np.array_equal(r.grads[i].cpu().numpy(), x[i] + ef[i].cpu().numpy())
+
+
+@pytest.mark.parametrize("n,nblk,tail", [(2, 14, 12_345), (3, 9, 0), (8, 6, 77)])
+def test_prepare_compress_fused_equals_the_two_calls(n, nblk, tail):
+    """thc_prepare_compress (block norms summed inside the transform kernel, Section 5.3's
+    overlap of the norm exchange with the RHT): its scales agree with thc_prepare's (fp64 sums
+    in another order: equal, or one ulp apart in rare cases) and with the oracle's; the packed
+    indices are bit-identical to thc_compress run on those same scales and to the oracle's."""
+    import torch
+    from paper_2302_08545_b200 import runner
+    k = 20
+    d = (nblk - 1) * (1 << k) + (tail if tail else (1 << k))
+    w = _mk(n, d, k)
+    x, _ = _inputs(w)
+    ctx = runner.context_for(w)
+    r = runner.Round(ctx, n, d)
+    assert r.sz.fused_scales == 1
+    r.upload(x)
+    r.prepare()
+    torch.cuda.synchronize()
+    s_two = r.scales.cpu().numpy().copy()
+    r.scales.zero_()
+    r.prepare_compress(rnd=1)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    s_fused = r.scales.cpu().numpy().copy()
+    p_fused = [p.cpu().numpy().copy() for p in r.packed]
+    ulp = np.abs(s_fused.view(np.int32).astype(np.int64) - s_two.view(np.int32).astype(np.int64))
+    assert ulp.max() <= 1 and (ulp > 0).mean() <= 0.1, ulp
+    c = _ocfg(w)
+    s_or = O.scales(x, c)
+    ulp_o = np.abs(s_fused.view(np.int32).astype(np.int64) - s_or.view(np.int32).astype(np.int64))
+    assert ulp_o.max() <= 1
+    for p in r.packed:
+        p.zero_()
+    r.compress(rnd=1)                      # same scales, separate call
+    torch.cuda.synchronize()
+    for i in range(n):
+        assert np.array_equal(r.packed[i].cpu().numpy(), p_fused[i]), f"worker {i}"
+    # and the oracle on the first and last blocks of two workers
+    for i in (0, n - 1):
+        for blk in (0, nblk - 1):
+            lo, hi = blk << k, min(d, (blk + 1) << k)
+            xb = np.zeros(1 << k, np.float32)
+            xb[: hi - lo] = x[i, lo:hi]
+            rot = O.rht_forward(xb, c, 1, j_base=lo)
+            z = O.quantize(rot, s_fused[blk:blk + 1], c, worker=i, rnd=1, j_base=lo)
+            got = O.unpack(p_fused[i][(lo * w.bits) // 8:((lo + (1 << k)) * w.bits) // 8], 1 << k, w.bits)
+            assert np.array_equal(got, z), (i, blk)
+
+
+def test_prepare_compress_falls_back_where_the_fused_kernel_does_not_apply():
+    """Other block sizes (and problems too small for the longer pipeline) take the two calls
+    inside the same entry point: results identical to calling them."""
+    import torch
+    from paper_2302_08545_b200 import runner
+    for k, d, n in [(16, 300_000, 3), (20, (1 << 20) + 5, 2)]:
+        w = _mk(n, d, k)
+        x, _ = _inputs(w)
+        ctx = runner.context_for(w)
+        r = runner.Round(ctx, n, d)
+        assert r.sz.fused_scales == 0
+        r.upload(x)
+        r.prepare(); r.compress(rnd=3)
+        torch.cuda.synchronize()
+        s0 = r.scales.cpu().numpy().copy(); p0 = [p.cpu().numpy().copy() for p in r.packed]
+        r.scales.zero_()
+        for p in r.packed:
+            p.zero_()
+        r.prepare_compress(rnd=3)
+        torch.cuda.synchronize()
+        assert np.array_equal(r.scales.cpu().numpy(), s0)
+        for i in range(n):
+            assert np.array_equal(r.packed[i].cpu().numpy(), p0[i])
