@@ -3,8 +3,11 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg2]
 
-A step is one pass of the whole path over one batch of synthetic gradients:
-thc_prepare + thc_compress (all n simulated workers) + thc_aggregate + one thc_decompress.
+A step is one pass of the whole path over one batch of synthetic gradients: scales and
+compress of all n simulated workers (thc_prepare_compress, one launch where the fused kernel
+applies, else thc_prepare + thc_compress), thc_aggregate and one thc_decompress.  After the
+timed region the two halves are also timed as separate calls (`split_calls_ms`), which gives
+the compress + aggregate + decompress round with the scales given.
 `value` is fp32-gradient GB/s (n * d * 4 bytes per step) with inputs resident in HBM;
 `e2e` is the same metric with the gradients coming from pinned host memory and the result
 copied back, every step.  With N > 1 every rank runs an independent replica of the workload
@@ -31,11 +34,13 @@ from paper_2302_08545_b200 import workloads as W  # noqa: E402
 
 METRIC = "gradient GB/s per compress+aggregate+decompress round; % of HBM roofline"
 UNIT = "GB/s"
-KERNELS_PER_STEP = {"prepare": 2, "compress": 1, "aggregate": 1, "decompress": 1}
-# DRAM bytes per (worker, padded coordinate) of the compress kernel, measured with ncu on the
-# d=2^24, n=4, b=4 sweep point (profiles/thc_pipeline_kernel_sweep_d2p24_b4_n4.md); traffic
-# grows in proportion to n*d_pad, so a full launch is this times n*d_pad.
-NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.261}
+KERNELS_PER_STEP = {"prepare": 2, "compress": 1, "prepare_compress": 1, "aggregate": 1, "decompress": 1}
+# DRAM bytes per (worker, padded coordinate) of the compress kernel and of its fused-scales
+# variant, measured with ncu on the d=2^24, n=4, b=4 sweep point
+# (profiles/thc_pipeline_kernel_sweep_d2p24_b4_n4.md); traffic grows in proportion to n*d_pad,
+# so a full launch is this times n*d_pad.
+NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.293}
+NCU_FUSED_DRAM_BYTES_PER_COORD = {("f32", 4): 6.213}
 
 
 def pick_workload(name: str) -> W.Workload:
@@ -237,8 +242,10 @@ def run_gpu(args):
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream()
 
-    calls = [("prepare", r.prepare), ("compress", lambda: r.compress(0)),
-             ("aggregate", r.aggregate), ("decompress", lambda: r.decompress(0))]
+    fused = bool(r.sz.fused_scales)
+    head = [("prepare_compress", lambda: r.prepare_compress(0))] if fused else \
+        [("prepare", r.prepare), ("compress", lambda: r.compress(0))]
+    calls = head + [("aggregate", r.aggregate), ("decompress", lambda: r.decompress(0))]
 
     def step(events=None):
         for name, fn in calls:
@@ -282,6 +289,25 @@ def run_gpu(args):
     per_call_ms = {k: float(np.mean(v)) for k, v in per_call.items()}
     status = ctx.status()
 
+    # ---- the two halves as separate calls (not part of `value`): scales, then compress
+    split_ms = dict(per_call_ms)
+    if fused:
+        split_events = []
+        for it in range(3 + min(args.steps, 20)):
+            for name, fn in [("prepare", r.prepare), ("compress", lambda: r.compress(0))]:
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                if it >= 3:
+                    split_events.append((name, a, b))
+        torch.cuda.synchronize()
+        acc = {}
+        for name, a, b in split_events:
+            acc.setdefault(name, []).append(a.elapsed_time(b))
+        split_ms.update({k: float(np.mean(v)) for k, v in acc.items()})
+
     # ---- end to end: gradients from pinned host memory, result copied back, every step
     e2e_steps = max(1, min(args.steps, 5))
     x_host = torch.from_numpy(x).pin_memory() if w.in_dtype == "f32" else \
@@ -316,11 +342,13 @@ def run_gpu(args):
     ab = w.algorithmic_bytes()
     peak, peak_src = measured_peaks()
     value = world * grad_bytes / (ms * 1e-3) / 1e9
-    round_ms = per_call_ms["compress"] + per_call_ms["aggregate"] + per_call_ms["decompress"]
-    comp_ms = per_call_ms["compress"]
+    round_ms = split_ms["compress"] + per_call_ms["aggregate"] + per_call_ms["decompress"]
+    top = "prepare_compress" if fused else "compress"
+    comp_ms = per_call_ms[top]
     achieved = ab["compress"] / (comp_ms * 1e-3) / 1e9
     in_bytes = w.n * w.d * (4 if w.in_dtype == "f32" else 2)
-    per_coord = NCU_COMPRESS_DRAM_BYTES_PER_COORD.get((w.in_dtype, w.bits))
+    per_coord = (NCU_FUSED_DRAM_BYTES_PER_COORD if fused else NCU_COMPRESS_DRAM_BYTES_PER_COORD).get(
+        (w.in_dtype, w.bits))
     traffic = None if per_coord is None or w.log2_block < 15 else per_coord * w.n * w.d_pad
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -331,8 +359,10 @@ def run_gpu(args):
         "e2e": {"value": world * grad_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": w.d * 4,
                 "ms_per_step": e2e_ms, "steps": e2e_steps},
-        "gpu_launches": args.steps * sum(KERNELS_PER_STEP.values()),
-        "roofline": {"kernel": "thc_compress: one persistent RHT + quantise + pack kernel per call",
+        "gpu_launches": args.steps * sum(KERNELS_PER_STEP[name] for name, _ in calls),
+        "roofline": {"kernel": ("thc_prepare_compress: one persistent norms + RHT + quantise + pack kernel per call"
+                                if fused else
+                                "thc_compress: one persistent RHT + quantise + pack kernel per call"),
                      "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": ab["compress"], "ms_per_launch": comp_ms,
@@ -340,6 +370,7 @@ def run_gpu(args):
                      "traffic_source": "ncu dram bytes on the d=2^24 n=4 b=4 sweep point, scaled by n*d_pad"
                                        if traffic is not None else None},
         "per_call_ms": per_call_ms,
+        "split_calls_ms": {k: split_ms[k] for k in ("prepare", "compress") if k in split_ms},
         "round_excl_prepare": {
             "ms": round_ms, "gradient_gbs": grad_bytes / (round_ms * 1e-3) / 1e9,
             "algorithmic_gbs": ab["round"] / (round_ms * 1e-3) / 1e9,
