@@ -947,7 +947,14 @@ typedef void (*pipe_kernel_t)(const TmaMaps, PipeParams, PtrArrayP, MutPtrArrayP
 template <int MODE, int KB>
 static pipe_kernel_t pick_pipe_kernel_kb(uint32_t bits, bool identity)
 {
-    if constexpr (MODE != kCompressF32 && MODE != kCompressBF16 && MODE != kCompressF32Fused) {
+    if constexpr (MODE == kErrorFeedback) {
+        switch (bits) {
+        case 1: return thc_pipeline_kernel<MODE, 1, true, KB>;
+        case 2: return thc_pipeline_kernel<MODE, 2, true, KB>;
+        case 4: return thc_pipeline_kernel<MODE, 4, true, KB>;
+        default: return thc_pipeline_kernel<MODE, 8, true, KB>;
+        }
+    } else if constexpr (MODE != kCompressF32 && MODE != kCompressBF16 && MODE != kCompressF32Fused) {
         return thc_pipeline_kernel<MODE, 4, true, KB>;
     } else {
         switch (bits) {
@@ -1310,6 +1317,24 @@ int thc_error_feedback(thc_ctx *ctx, const void *const *grads, const void *const
     if (scales == nullptr || workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
     if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ctx->cfg.log2_block > (uint32_t)kTileLog2) {
+        // one launch of the pipeline for all workers: indices in, x_i - RHT^-1(X_i) out
+        thc_sizes_t szn;
+        if ((rc = thc_sizes(ctx, d, n_local, &szn)) != THC_OK) return rc;
+        if (workspace_bytes < szn.workspace_bytes) return THC_EWORKSPACE;
+        PtrArrayP pin;
+        MutPtrArrayP pout, px;
+        memset(&pin, 0, sizeof pin);
+        memset(&pout, 0, sizeof pout);
+        memset(&px, 0, sizeof px);
+        for (uint32_t i = 0; i < n_local; ++i) {
+            pin.p[i] = packed[i];
+            pout.p[i] = ef[i];
+            px.p[i] = const_cast<void *>(grads[i]);
+        }
+        pipe_kernel_t kern = pick_pipe_kernel<kErrorFeedback>(ctx->cfg.bits, true, ctx->cfg.log2_block);
+        return launch_pipeline(ctx, kern, false, szn, d, n_local, 0, round, 1, scales, workspace, pin, pout, px, st);
+    }
     const uint64_t ring_bytes = sz.workspace_bytes - round_up(sz.sum_bytes, 256);
     void *values = static_cast<unsigned char *>(workspace) + ring_bytes;
     uint64_t blocks = (d / 4 + kThreads - 1) / kThreads;

@@ -52,7 +52,8 @@ constexpr int kBlockConstMax = 256;         // per-block constants cached in sha
 constexpr uint32_t kMaxPolls = 1u << 21;
 
 enum PipeMode { kCompressF32, kCompressBF16, kDecompress8, kDecompress16, kDecompress32,
-                kCompressF32Fused };   // fp32 compress that also computes the block scales (below)
+                kCompressF32Fused,     // fp32 compress that also computes the block scales (below)
+                kErrorFeedback };      // e_i = x_i - RHT^-1(X_i) from worker i's own packed indices
 
 // Layout inside DeviceBlock::counters.  Every CTA hits `head` and `abort` for every task and
 // the completion counters of the slots in use: each gets its own 128-byte line (head, exited,
@@ -277,6 +278,11 @@ __device__ __forceinline__ void fence_proxy_async_global()
     asm volatile("fence.proxy.async.global;" ::: "memory");
 }
 
+__device__ __forceinline__ void prefetch_l2(const void *p)
+{
+    asm volatile("prefetch.global.L2 [%0];" :: "l"(p));
+}
+
 __device__ __forceinline__ uint64_t make_evict_normal_policy()
 {
     uint64_t pol;
@@ -489,6 +495,7 @@ struct EpilogueCtx {
     unsigned char *packed;
     float *rotated;
     float *out;
+    const float *xsub;      // error feedback: the output is xsub - (inverse transform)
     uint64_t d;
     const uint32_t *sw;
     int words_per_row;
@@ -519,15 +526,21 @@ __device__ __forceinline__ void epilogue_unit(const float4 &va, const float4 &vb
     } else {
         if (j >= ep.d) return;
         const uint32_t bits = ep.sw[row * ep.words_per_row + (uu >> 2)] >> (uint32_t)(j & 31);
-        const float4 oa = flip4(ra, bits);
-        const float4 ob = flip4(rb, bits >> 4);
+        float4 oa = flip4(ra, bits);
+        float4 ob = flip4(rb, bits >> 4);
         if (j + 8 <= ep.d) {
+            if (ep.xsub != nullptr) {
+                const float4 xa = __ldcs(reinterpret_cast<const float4 *>(ep.xsub + j));
+                const float4 xb = __ldcs(reinterpret_cast<const float4 *>(ep.xsub + j + 4));
+                oa = make_float4(xa.x - oa.x, xa.y - oa.y, xa.z - oa.z, xa.w - oa.w);
+                ob = make_float4(xb.x - ob.x, xb.y - ob.y, xb.z - ob.z, xb.w - ob.w);
+            }
             *reinterpret_cast<float4 *>(ep.out + j) = oa;
             *reinterpret_cast<float4 *>(ep.out + j + 4) = ob;
         } else {
             const float o[8] = {oa.x, oa.y, oa.z, oa.w, ob.x, ob.y, ob.z, ob.w};
             for (int e = 0; e < 8; ++e)
-                if (j + e < ep.d) ep.out[j + e] = o[e];
+                if (j + e < ep.d) ep.out[j + e] = ep.xsub != nullptr ? ep.xsub[j + e] - o[e] : o[e];
         }
     }
 }
@@ -618,6 +631,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     MutPtrArrayP outp, MutPtrArrayP rotated, PhiloxKeys keys)
 {
     constexpr bool kFused = MODE == kCompressF32Fused;
+    constexpr bool kEF = MODE == kErrorFeedback;
     constexpr bool kF32In = MODE == kCompressF32 || kFused;
     constexpr bool kCompress = kF32In || MODE == kCompressBF16;
     extern __shared__ __align__(1024) unsigned char pipe_smem_raw[];
@@ -653,6 +667,13 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
     if (kCompress && !IDENTITY) {
         for (int idx = tid; idx < (int)(P.granularity + 1) * kLutRep; idx += kPCtaThreads)
             lut[idx] = P.dev->lut[idx / kLutRep];
+    }
+    // error feedback: table values as floats, one copy per lane (8 copies for 8-bit indices)
+    constexpr int kFRep = BITS <= 4 ? 32 : 8;
+    float *ftab = reinterpret_cast<float *>(lut);
+    if (kEF) {
+        for (int idx = tid; idx < (1 << BITS) * kFRep; idx += kPCtaThreads)
+            ftab[idx] = (float)P.dev->table[idx / kFRep];
     }
     const uint32_t nblk_total = (uint32_t)(P.d_pad >> P.k);
     const uint32_t nblk_cached = nblk_total < (uint32_t)kBlockConstMax ? nblk_total : (uint32_t)kBlockConstMax;
@@ -776,6 +797,18 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                         tma_load_2d(bufs[s], &maps.in[wl], 0, (int)(j0 >> 5), &s_mbar[s], pol_stream);
                         tma = 1; phase = uses[s] & 1u; ++uses[s];
                     }
+                    if (!kF32In) {
+                        // tiles the compute warps load themselves: pull the lines into L2 now
+                        const uint32_t in_bits = MODE == kCompressBF16 ? 16u : MODE == kDecompress8 ? 8u
+                                                 : MODE == kDecompress16 ? 16u : MODE == kDecompress32 ? 32u
+                                                 : (uint32_t)BITS;
+                        const unsigned char *src = static_cast<const unsigned char *>(in.p[kEF || kCompress ? wl : 0]);
+                        const uint64_t first = j0 * in_bits / 8;
+                        const uint64_t limit = (MODE == kCompressBF16 ? P.d : P.d_pad) * in_bits / 8;
+                        const uint32_t lines = (uint32_t)kPElems * in_bits / 8 / 128;
+                        for (uint32_t l = (uint32_t)lane; l < lines; l += 32u)
+                            if (first + 128ull * l < limit) prefetch_l2(src + first + 128ull * l);
+                    }
                 }
                 // pass B needs its worker-block's tiles (fused scales: the block's M, which
                 // implies them); pass A needs the previous tenant of its ring slot consumed
@@ -819,6 +852,25 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 ti.gen = t.gen;
                 pend[s] = t;
                 pend_valid[s] = true;
+                if (t.is_b && !kCompress && KB == 7) {
+                    // inverse transform: sign words of the panel's 128 rows x 64 columns (two
+                    // words per row), and for error feedback the x values the epilogue will read
+                    const uint64_t j_panel = (uint64_t)r * B + ((uint64_t)t.idx << 6);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int row = lane + 32 * c;
+                        const uint64_t jr = j_panel + ((uint64_t)row << kPLog2);
+                        const uint4 ph = sign_call(jr, P.round, keys);
+                        const bool hi = ((jr >> 5) & 3u) != 0;         // words 2,3 of the call
+                        sw[256 * s + 2 * row] = hi ? ph.z : ph.x;
+                        sw[256 * s + 2 * row + 1] = hi ? ph.w : ph.y;
+                        if (kEF) {
+                            const float *xr = static_cast<const float *>(rotated.p[t.wb - r * P.n_local]) + jr;
+                            if (jr < P.d) prefetch_l2(xr);
+                            if (jr + 32 < P.d) prefetch_l2(xr + 32);
+                        }
+                    }
+                }
                 if (lane == 0 && t.is_b) {
                     if (kFused) {
                         const float2 c = block_constants<true>(ld_relaxed_f32(P.scales + r), P.granularity, P.divisor);
@@ -895,6 +947,30 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                                                     __uint_as_float(w[1] << 16), __uint_as_float(w[1] & 0xFFFF0000u));
                     tile[pswz(2 * u + 1)] = make_float4(__uint_as_float(w[2] << 16), __uint_as_float(w[2] & 0xFFFF0000u),
                                                         __uint_as_float(w[3] << 16), __uint_as_float(w[3] & 0xFFFF0000u));
+                }
+            } else if (kEF) {
+                // worker wl's own indices -> table values -> m + T[z] (M - m)/g
+                constexpr int kPer = 128 / BITS;           // coordinates per 16-byte load
+                const unsigned char *z = static_cast<const unsigned char *>(in.p[ti.wl]);
+                const float2 bc = ti.r < nblk_cached ? blk_const[ti.r]
+                                                     : block_constants<false>(P.scales[ti.r], P.granularity, P.divisor);
+                const float *ft = ftab + (tid & (kFRep - 1));
+#pragma unroll 1
+                for (int u = tid; u < kPElems / kPer; u += kPThreads) {
+                    const uint64_t j = j0 + (uint64_t)u * kPer;
+                    const uint4 q = __ldg(reinterpret_cast<const uint4 *>(z + j * BITS / 8));
+                    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                    for (int cc = 0; cc < kPer / 4; ++cc) {
+                        float sv[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int bit = (cc * 4 + e) * BITS;
+                            const uint32_t zz = (w[bit >> 5] >> (bit & 31)) & ((1u << BITS) - 1u);
+                            sv[e] = fmaf(ft[zz * kFRep], bc.x, bc.y);
+                        }
+                        tile[pswz(u * (kPer / 4) + cc)] = make_float4(sv[0], sv[1], sv[2], sv[3]);
+                    }
                 }
             } else {
                 constexpr int kPer = MODE == kDecompress8 ? 16 : MODE == kDecompress16 ? 8 : 4;
@@ -980,11 +1056,12 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 ep.worker = P.worker_base + wl; ep.round = P.round;
                 ep.packed = kCompress ? static_cast<unsigned char *>(outp.p[wl]) : nullptr;
                 ep.rotated = kCompress ? static_cast<float *>(rotated.p[wl]) : nullptr;
-                ep.out = kCompress ? nullptr : static_cast<float *>(outp.p[0]);
+                ep.out = kCompress ? nullptr : static_cast<float *>(outp.p[wl]);
+                ep.xsub = kEF ? static_cast<const float *>(rotated.p[wl]) : nullptr;
                 ep.d = P.d;
-                ep.sw = sw;
+                ep.sw = (!kCompress && KB == 7) ? sw + 256 * cur : sw;
                 ep.words_per_row = max(1, (1 << (kPLog2 - kb)) >> 5);
-                if (!kCompress) {
+                if (!kCompress && KB != 7) {
                     TileGeom g;
                     g.row_log2 = (uint32_t)kb; g.col_log2 = (uint32_t)(kPLog2 - kb);
                     g.row_stride = 1ull << kPLog2; g.round = P.round;

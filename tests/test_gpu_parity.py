@@ -364,3 +364,22 @@ def test_prepare_compress_falls_back_where_the_fused_kernel_does_not_apply():
         assert np.array_equal(r.scales.cpu().numpy(), s0)
         for i in range(n):
             assert np.array_equal(r.packed[i].cpu().numpy(), p0[i])
+
+
+@pytest.mark.parametrize("bits,g", [(1, 1), (2, 3), (8, 255)])
+def test_error_feedback_other_index_widths(bits, g):
+    """The one-launch error-feedback path unpacks 1-, 2- and 8-bit indices as well."""
+    import torch
+    k, d, n = 16, 200_003, 2
+    w = _mk(n, d, k, bits=bits, g=g, table=tuple(range(g + 1)) if bits > 1 else (0, 1))
+    x, _ = _inputs(w)
+    ctx, r = _gpu_round(w, x, rnd=5, want_rotated=False)
+    ef = [torch.zeros(d, dtype=torch.float32, device=r.device) for _ in range(n)]
+    ctx.error_feedback(r.grads, r.packed, d, 5, r.scales, ef, r.workspace)
+    torch.cuda.synchronize()
+    c = _ocfg(w)
+    scl = r.scales.cpu().numpy()
+    for i in range(n):
+        z = O.unpack(r.packed[i].cpu().numpy(), r.sz.d_pad, w.bits)
+        ref = O.error_feedback(x[i], z, scl, c, 5)
+        assert np.array_equal(ef[i].cpu().numpy().view(np.uint32), ref.view(np.uint32)), f"worker {i}"
