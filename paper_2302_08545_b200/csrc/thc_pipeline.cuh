@@ -443,6 +443,69 @@ __device__ __forceinline__ double pass_a_round1(float4 *tile, const uint32_t *sw
     return sq;
 }
 
+// First round of a pass-A tile of the inverse transform (decompress, error feedback): the same
+// stages as pass_a_round1, but the thread fetches its two rows straight from global memory
+// (the control warp has pulled the lines into L2) and de-quantises them in registers:
+// sums Y -> m + Y (M - m)/(g n), or own indices z -> m + T[z] (M - m)/g  (Algorithm 2).
+// A row of 32 coordinates is IN_BITS 32-bit words; a warp's rows are contiguous in memory.
+template <int MODE, int BITS, int FREP>
+__device__ __forceinline__ void pass_a_round1_inverse(float4 *tile, const unsigned char *src, float2 bc,
+                                                      const float *ft, int tid)
+{
+    constexpr int IN_BITS = MODE == kDecompress8 ? 8 : MODE == kDecompress16 ? 16
+                            : MODE == kDecompress32 ? 32 : BITS;
+    const int x = tid & 7;
+    const int r0 = ((tid >> 5) << 6) | (tid & 31);
+    float4 v[16];
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+        const unsigned char *p = src + (size_t)(r0 + 32 * g) * (IN_BITS * 4);
+        uint32_t w[IN_BITS];
+        if constexpr (IN_BITS >= 4) {
+#pragma unroll
+            for (int q = 0; q < IN_BITS / 4; ++q) {
+                const uint4 t4 = __ldg(reinterpret_cast<const uint4 *>(p) + q);
+                w[4 * q] = t4.x; w[4 * q + 1] = t4.y; w[4 * q + 2] = t4.z; w[4 * q + 3] = t4.w;
+            }
+        } else if constexpr (IN_BITS == 2) {
+            const uint2 t2 = __ldg(reinterpret_cast<const uint2 *>(p));
+            w[0] = t2.x; w[1] = t2.y;
+        } else {
+            w[0] = __ldg(reinterpret_cast<const uint32_t *>(p));
+        }
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+            float sv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int bit = (m * 4 + e) * IN_BITS;
+                const uint32_t val = IN_BITS == 32 ? w[bit >> 5]
+                                                   : (w[bit >> 5] >> (bit & 31)) & ((1u << (IN_BITS & 31)) - 1u);
+                float yf;
+                if (MODE == kErrorFeedback) yf = ft[val * FREP];
+                else if (MODE == kDecompress32) yf = (float)val;
+                else yf = __uint_as_float(0x4B000000u | val) - 8388608.0f;
+                sv[e] = fmaf(yf, bc.x, bc.y);
+            }
+            v[8 * g + m] = make_float4(sv[0], sv[1], sv[2], sv[3]);
+        }
+    }
+#pragma unroll
+    for (int m = 0; m < 16; ++m) v[m] = stages01(v[m]);
+#pragma unroll
+    for (int t = 0; t < 3; ++t) {
+#pragma unroll
+        for (int m = 0; m < 16; ++m)
+            if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
+    }
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+        float4 *row = tile + (r0 + 32 * g) * 8;
+#pragma unroll
+        for (int m = 0; m < 8; ++m) row[m ^ x] = v[8 * g + m];
+    }
+}
+
 // Round on row bits 0..3: thread (rg = tid >> 3, cc = tid & 7) owns chunk cc of rows
 // 16 rg + m.  Serves pass A (second round) and the first round of a k = 20 pass-B tile, whose
 // two 128-row halves are simply rows 0..255.
@@ -948,58 +1011,6 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     tile[pswz(2 * u + 1)] = make_float4(__uint_as_float(w[2] << 16), __uint_as_float(w[2] & 0xFFFF0000u),
                                                         __uint_as_float(w[3] << 16), __uint_as_float(w[3] & 0xFFFF0000u));
                 }
-            } else if (kEF) {
-                // worker wl's own indices -> table values -> m + T[z] (M - m)/g
-                constexpr int kPer = 128 / BITS;           // coordinates per 16-byte load
-                const unsigned char *z = static_cast<const unsigned char *>(in.p[ti.wl]);
-                const float2 bc = ti.r < nblk_cached ? blk_const[ti.r]
-                                                     : block_constants<false>(P.scales[ti.r], P.granularity, P.divisor);
-                const float *ft = ftab + (tid & (kFRep - 1));
-#pragma unroll 1
-                for (int u = tid; u < kPElems / kPer; u += kPThreads) {
-                    const uint64_t j = j0 + (uint64_t)u * kPer;
-                    const uint4 q = __ldg(reinterpret_cast<const uint4 *>(z + j * BITS / 8));
-                    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                    for (int cc = 0; cc < kPer / 4; ++cc) {
-                        float sv[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int bit = (cc * 4 + e) * BITS;
-                            const uint32_t zz = (w[bit >> 5] >> (bit & 31)) & ((1u << BITS) - 1u);
-                            sv[e] = fmaf(ft[zz * kFRep], bc.x, bc.y);
-                        }
-                        tile[pswz(u * (kPer / 4) + cc)] = make_float4(sv[0], sv[1], sv[2], sv[3]);
-                    }
-                }
-            } else {
-                constexpr int kPer = MODE == kDecompress8 ? 16 : MODE == kDecompress16 ? 8 : 4;
-                const unsigned char *y = static_cast<const unsigned char *>(in.p[0]);
-                const float2 bc = ti.r < nblk_cached ? blk_const[ti.r]
-                                                     : block_constants<false>(P.scales[ti.r], P.granularity, P.divisor);
-#pragma unroll 2
-                for (int i = 0; i < kPElems / kPer / kPThreads; ++i) {
-                    const int u = tid + i * kPThreads;
-                    const uint64_t j = j0 + (uint64_t)u * kPer;
-                    const uint4 q = __ldg(reinterpret_cast<const uint4 *>(y + j * (16 / kPer)));
-                    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                    for (int cc = 0; cc < kPer / 4; ++cc) {
-                        float sv[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int ix = cc * 4 + e;
-                            uint32_t val;
-                            if (MODE == kDecompress8) val = (w[ix >> 2] >> ((ix & 3) * 8)) & 0xFFu;
-                            else if (MODE == kDecompress16) val = (w[ix >> 1] >> ((ix & 1) * 16)) & 0xFFFFu;
-                            else val = w[ix];
-                            const float yf = MODE == kDecompress32 ? (float)val
-                                             : __uint_as_float(0x4B000000u | val) - 8388608.0f;
-                            sv[e] = fmaf(yf, bc.x, bc.y);
-                        }
-                        tile[pswz(u * (kPer / 4) + cc)] = make_float4(sv[0], sv[1], sv[2], sv[3]);
-                    }
-                }
             }
         };
 
@@ -1020,12 +1031,12 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     atomicOr(&P.dev->status, THC_STATUS_WAIT_TIMEOUT);
                     atomicExch(&pc->abort, 1u);
                 }
-            } else {
+            } else if (kCompress || me.is_b) {
                 load_tile(me, tile);
                 cp_async_commit();
                 cp_async_wait_all();
                 compute_barrier();
-            }
+            }                                          // inverse pass A: round 1 fetches its own rows
             const bool is_b = me.is_b != 0;
             const uint32_t wl = me.wl;
             const uint64_t r = me.r;
@@ -1037,7 +1048,16 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
 
             if (!is_b) {
                 // ================================ pass A: tile idx of worker-block wb
-                double sq = pass_a_round1<kCompress, kFused>(tile, sw + 256 * cur, tid);
+                double sq = 0.0;
+                if constexpr (kCompress) {
+                    sq = pass_a_round1<true, kFused>(tile, sw + 256 * cur, tid);
+                } else {
+                    constexpr int kInBits = MODE == kDecompress8 ? 8 : MODE == kDecompress16 ? 16
+                                            : MODE == kDecompress32 ? 32 : BITS;
+                    const unsigned char *src = static_cast<const unsigned char *>(in.p[kEF ? wl : 0]) +
+                        (r * B + ((uint64_t)idx << kPLog2)) * kInBits / 8;
+                    pass_a_round1_inverse<MODE, BITS, kFRep>(tile, src, bc, ftab + (tid & (kFRep - 1)), tid);
+                }
                 if (kFused) {
                     for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, off);
                     if ((tid & 31) == 0) s_sq[cur][tid >> 5] = sq;
