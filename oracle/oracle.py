@@ -79,6 +79,16 @@ def _load():
     lib.thc_oracle_error_feedback.restype = None
     lib.thc_oracle_dequantize.argtypes = [u8p, u64, u32, f32p, u32, u16p, f64p]
     lib.thc_oracle_dequantize.restype = None
+    lib.thc_oracle_quantize_range_at.argtypes = [f32p, u64, u32, f32p, f32p, u32, u32, u16p, u64, u32, u32, u64, u8p]
+    lib.thc_oracle_quantize_range_at.restype = None
+    lib.thc_oracle_estimate_range.argtypes = [vp, u32, u32, u64, u32, f32p, f32p, u32, f32p]
+    lib.thc_oracle_estimate_range.restype = None
+    lib.thc_oracle_decompress_range.argtypes = [vp, u32, u32, u64, u32, f32p, f32p, u32, u64, u32, f32p]
+    lib.thc_oracle_decompress_range.restype = None
+    lib.thc_oracle_error_feedback_range.argtypes = [f32p, u8p, u64, u32, f32p, f32p, u32, u16p, u64, u32, f32p]
+    lib.thc_oracle_error_feedback_range.restype = None
+    lib.thc_oracle_ranges.argtypes = [f32p, u32, u64, u32, u64, u32, f32p, f32p]
+    lib.thc_oracle_ranges.restype = None
     _lib = lib
     return lib
 
@@ -170,6 +180,19 @@ def scales(x, cfg: Config) -> np.ndarray:
     return out
 
 
+def ranges(x, cfg: Config, rnd: int):
+    """Exact (lo, hi) per RHT block of the rotated coordinates over all workers (Algorithm 1's
+    preliminary stage applied after the rotation).  x is [n, d]."""
+    x = _f32(x)
+    n, d = x.shape
+    nb = cfg.d_pad(d) // cfg.block
+    lo = np.zeros(nb, dtype=np.float32)
+    hi = np.zeros(nb, dtype=np.float32)
+    _load().thc_oracle_ranges(_p(x, ctypes.c_float), n, d, cfg.log2_block, cfg.seed, rnd,
+                              _p(lo, ctypes.c_float), _p(hi, ctypes.c_float))
+    return lo, hi
+
+
 def rht_forward(x, cfg: Config, rnd: int, j_base: int = 0) -> np.ndarray:
     """j_base: padded coordinate of x[0] in the whole vector (a multiple of the block), for
     transforming a slice of a long vector."""
@@ -191,14 +214,23 @@ def rht_inverse(v, d: int, cfg: Config, rnd: int, j_base: int = 0) -> np.ndarray
     return out
 
 
-def quantize(r, scl, cfg: Config, rnd: int, worker: int, j_base: int = 0) -> np.ndarray:
+def quantize(r, scl, cfg: Config, rnd: int, worker: int, j_base: int = 0, lo=None) -> np.ndarray:
     """Rotated coordinates -> one table index per coordinate (uint8, unpacked).  With j_base,
-    r is a slice starting at that padded coordinate and scl[0] is the scale of its block."""
+    r is a slice starting at that padded coordinate and scl[0] is the scale of its block.
+    With lo, the range of a block is [lo, scl] (Algorithm 1's exact range) instead of
+    [-scl, scl]."""
     r = _f32(r)
     scl = _f32(scl)
     assert j_base % cfg.block == 0
     z = np.zeros(r.size, dtype=np.uint8)
     t = cfg.table_u16()
+    if lo is not None:
+        lo = _f32(lo)
+        _load().thc_oracle_quantize_range_at(_p(r, ctypes.c_float), r.size, cfg.log2_block,
+                                             _p(lo, ctypes.c_float), _p(scl, ctypes.c_float),
+                                             cfg.bits, cfg.granularity, _p(t, ctypes.c_uint16),
+                                             cfg.seed, rnd, worker, j_base, _p(z, ctypes.c_uint8))
+        return z
     _load().thc_oracle_quantize_at(_p(r, ctypes.c_float), r.size, cfg.log2_block,
                                    _p(scl, ctypes.c_float), cfg.bits, cfg.granularity,
                                    _p(t, ctypes.c_uint16), cfg.seed, rnd, worker, j_base,
@@ -232,30 +264,44 @@ def aggregate(packed, d_pad: int, cfg: Config, w: int) -> np.ndarray:
     return out
 
 
-def decompress(total, divisor: int, d: int, scl, cfg: Config, rnd: int) -> np.ndarray:
+def decompress(total, divisor: int, d: int, scl, cfg: Config, rnd: int, lo=None) -> np.ndarray:
     total = np.ascontiguousarray(total)
     w = total.dtype.itemsize * 8
     scl = _f32(scl)
     out = np.zeros(d, dtype=np.float32)
+    if lo is not None:
+        lo = _f32(lo)
+        _load().thc_oracle_decompress_range(total.ctypes.data_as(ctypes.c_void_p), w, divisor, d,
+                                            cfg.log2_block, _p(lo, ctypes.c_float),
+                                            _p(scl, ctypes.c_float), cfg.granularity, cfg.seed, rnd,
+                                            _p(out, ctypes.c_float))
+        return out
     _load().thc_oracle_decompress(total.ctypes.data_as(ctypes.c_void_p), w, divisor, d,
                                   cfg.log2_block, _p(scl, ctypes.c_float), cfg.granularity,
                                   cfg.seed, rnd, _p(out, ctypes.c_float))
     return out
 
 
-def estimate(total, divisor: int, scl, cfg: Config) -> np.ndarray:
+def estimate(total, divisor: int, scl, cfg: Config, lo=None) -> np.ndarray:
     """Algorithm 2's 'Estimate' line: the averaged vector, still in the rotated domain."""
     total = np.ascontiguousarray(total)
     w = total.dtype.itemsize * 8
     scl = _f32(scl)
     v = np.zeros(total.size, dtype=np.float32)
+    if lo is not None:
+        lo = _f32(lo)
+        _load().thc_oracle_estimate_range(total.ctypes.data_as(ctypes.c_void_p), w, divisor,
+                                          total.size, cfg.log2_block, _p(lo, ctypes.c_float),
+                                          _p(scl, ctypes.c_float), cfg.granularity,
+                                          _p(v, ctypes.c_float))
+        return v
     _load().thc_oracle_estimate(total.ctypes.data_as(ctypes.c_void_p), w, divisor, total.size,
                                 cfg.log2_block, _p(scl, ctypes.c_float), cfg.granularity,
                                 _p(v, ctypes.c_float))
     return v
 
 
-def error_feedback(x, z, scl, cfg: Config, rnd: int) -> np.ndarray:
+def error_feedback(x, z, scl, cfg: Config, rnd: int, lo=None) -> np.ndarray:
     """e = x - RHT^-1(X) for one worker (Algorithm 3): x has d entries, z d_pad indices."""
     x = _f32(x)
     z = np.ascontiguousarray(z, dtype=np.uint8)
@@ -263,6 +309,14 @@ def error_feedback(x, z, scl, cfg: Config, rnd: int) -> np.ndarray:
     assert z.size == cfg.d_pad(x.size)
     e = np.zeros(x.size, dtype=np.float32)
     t = cfg.table_u16()
+    if lo is not None:
+        lo = _f32(lo)
+        _load().thc_oracle_error_feedback_range(_p(x, ctypes.c_float), _p(z, ctypes.c_uint8), x.size,
+                                                cfg.log2_block, _p(lo, ctypes.c_float),
+                                                _p(scl, ctypes.c_float), cfg.granularity,
+                                                _p(t, ctypes.c_uint16), cfg.seed, rnd,
+                                                _p(e, ctypes.c_float))
+        return e
     _load().thc_oracle_error_feedback(_p(x, ctypes.c_float), _p(z, ctypes.c_uint8), x.size,
                                       cfg.log2_block, _p(scl, ctypes.c_float), cfg.granularity,
                                       _p(t, ctypes.c_uint16), cfg.seed, rnd, _p(e, ctypes.c_float))
@@ -282,7 +336,7 @@ def dequantize(z, scl, cfg: Config) -> np.ndarray:
 
 
 # ---------------------------------------------------------------------------------------
-def compress(x, scl, cfg: Config, rnd: int, worker_base: int = 0):
+def compress(x, scl, cfg: Config, rnd: int, worker_base: int = 0, lo=None):
     """All of a worker's compress step for each row of x: returns (packed [n, bytes],
     rotated [n, d_pad])."""
     x = _f32(x)
@@ -292,19 +346,24 @@ def compress(x, scl, cfg: Config, rnd: int, worker_base: int = 0):
     packed = np.zeros((n, d_pad * cfg.bits // 8), dtype=np.uint8)
     for i in range(n):
         rotated[i] = rht_forward(x[i], cfg, rnd)
-        packed[i] = pack(quantize(rotated[i], scl, cfg, rnd, worker_base + i), cfg.bits)
+        packed[i] = pack(quantize(rotated[i], scl, cfg, rnd, worker_base + i, lo=lo), cfg.bits)
     return packed, rotated
 
 
-def thc_round(x, cfg: Config, rnd: int = 0, scl=None):
-    """One whole round (Algorithm 3, THC lines): returns a dict with every stage."""
+def thc_round(x, cfg: Config, rnd: int = 0, scl=None, exact_range: bool = False):
+    """One whole round (Algorithm 3, THC lines): returns a dict with every stage.  With
+    exact_range the clamp range is the exact min/max of the rotated coordinates (Algorithm 1's
+    preliminary stage) instead of the norm-based [-M, M] of Section 5.3."""
     x = _f32(x)
     n, d = x.shape
-    if scl is None:
+    lo = None
+    if exact_range:
+        lo, scl = ranges(x, cfg, rnd)
+    elif scl is None:
         scl = scales(x, cfg)
-    packed, rotated = compress(x, scl, cfg, rnd)
+    packed, rotated = compress(x, scl, cfg, rnd, lo=lo)
     w = acc_bits(n, cfg.granularity)
     total = aggregate(packed, cfg.d_pad(d), cfg, w)
-    out = decompress(total, n, d, scl, cfg, rnd)
-    return {"scales": scl, "rotated": rotated, "packed": packed, "sum": total, "out": out,
+    out = decompress(total, n, d, scl, cfg, rnd, lo=lo)
+    return {"lo": lo, "scales": scl, "rotated": rotated, "packed": packed, "sum": total, "out": out,
             "acc_bits": w}

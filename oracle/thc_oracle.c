@@ -240,20 +240,26 @@ void thc_oracle_quantize(const float *r, uint64_t d_pad, uint32_t k, const float
     thc_oracle_quantize_at(r, d_pad, k, scales, b, g, table, seed, round, worker, 0, z);
 }
 
-/* Slice form: r[0] is padded coordinate j_base (a multiple of B); scales[0] is its block. */
-void thc_oracle_quantize_at(const float *r, uint64_t d_pad, uint32_t k, const float *scales,
-                            uint32_t b, uint32_t g, const uint16_t *table, uint64_t seed,
-                            uint32_t round, uint32_t worker, uint64_t j_base, uint8_t *z)
+/* General range [lo, hi] per block (Algorithm 2 worker lines with m = lo, M = hi; Algorithm 1's
+ * preliminary stage supplies an exact range, Section 5.3 the symmetric one lo = -M, hi = M):
+ *   u = clamp(fma(r, kappa, off), 0, 1),  kappa = (float)(1/(hi - lo)),  off = (float)(-lo/(hi - lo)),
+ * which for lo = -hi is kappa = 1/(2M), off = 1/2 exactly.  Slice form as below. */
+void thc_oracle_quantize_range_at(const float *r, uint64_t d_pad, uint32_t k, const float *lo,
+                                  const float *hi, uint32_t b, uint32_t g, const uint16_t *table,
+                                  uint64_t seed, uint32_t round, uint32_t worker, uint64_t j_base,
+                                  uint8_t *z)
 {
     uint64_t B = (uint64_t)1 << k;
     uint32_t levels = 1u << b;
 #pragma omp parallel for schedule(static)
     for (int64_t jj = 0; jj < (int64_t)d_pad; ++jj) {
         uint64_t j = (uint64_t)jj;
-        float M = scales[j / B];
-        if (!(M > 0.0f) || !isfinite(M)) { z[j] = 0; continue; }          /* R8 */
-        float kappa = (float)(1.0 / (2.0 * (double)M));
-        float pos = fmaf(r[j], kappa, 0.5f);                              /* R5 */
+        float m = lo[j / B], M = hi[j / B];
+        if (!(M > m) || !isfinite(M) || !isfinite(m)) { z[j] = 0; continue; }   /* R8 */
+        double width = (double)M - (double)m;
+        float kappa = (float)(1.0 / width);
+        float off = (float)(-(double)m / width);
+        float pos = fmaf(r[j], kappa, off);                               /* R5 */
         if (!(pos >= 0.0f)) pos = 0.0f;                                   /* NaN -> 0 */
         if (pos > 1.0f) pos = 1.0f;
         int f = (int)floor((double)pos * (double)g);                      /* exact product */
@@ -268,6 +274,25 @@ void thc_oracle_quantize_at(const float *r, uint64_t d_pad, uint32_t k, const fl
         uint32_t u = thc_oracle_u16(seed, round, worker, j_base + j);
         z[j] = (uint8_t)(z0 + (u < threshold ? 1u : 0u));
     }
+}
+
+static float *negated(const float *scales, uint64_t count)
+{
+    float *lo = (float *)malloc(sizeof(float) * (count ? count : 1));
+    for (uint64_t i = 0; i < count; ++i) lo[i] = -scales[i];
+    return lo;
+}
+
+/* Slice form: r[0] is padded coordinate j_base (a multiple of B); scales[0] is its block.
+ * The symmetric range of Section 5.3: m = -M. */
+void thc_oracle_quantize_at(const float *r, uint64_t d_pad, uint32_t k, const float *scales,
+                            uint32_t b, uint32_t g, const uint16_t *table, uint64_t seed,
+                            uint32_t round, uint32_t worker, uint64_t j_base, uint8_t *z)
+{
+    uint64_t nb = (d_pad + ((uint64_t)1 << k) - 1) >> k;
+    float *lo = negated(scales, nb);
+    thc_oracle_quantize_range_at(r, d_pad, k, lo, scales, b, g, table, seed, round, worker, j_base, z);
+    free(lo);
 }
 
 /* Bit-packing (Section 3; reading R7). packed has d_pad*b/8 bytes. */
@@ -320,19 +345,40 @@ void thc_oracle_aggregate(const uint8_t *packed, uint32_t n, uint64_t d_pad, uin
  * `divisor` is n (or the number of workers actually summed).  thc_oracle_estimate is the
  * "Estimate" line alone (d_pad values, still in the rotated domain).
  * ---------------------------------------------------------------------------------- */
-void thc_oracle_estimate(const void *sum, uint32_t w, uint32_t divisor, uint64_t d_pad,
-                         uint32_t k, const float *scales, uint32_t g, float *v)
+void thc_oracle_estimate_range(const void *sum, uint32_t w, uint32_t divisor, uint64_t d_pad,
+                               uint32_t k, const float *lo, const float *hi, uint32_t g, float *v)
 {
     uint64_t B = (uint64_t)1 << k;
     for (uint64_t j = 0; j < d_pad; ++j) {
-        float M = scales[j / B];
-        if (!(M > 0.0f) || !isfinite(M)) { v[j] = 0.0f; continue; }      /* R8 */
+        float m = lo[j / B], M = hi[j / B];
+        if (!(M > m) || !isfinite(M) || !isfinite(m)) { v[j] = 0.0f; continue; }   /* R8 */
         uint32_t y = w == 8 ? ((const uint8_t *)sum)[j]
                    : w == 16 ? ((const uint16_t *)sum)[j]
                              : ((const uint32_t *)sum)[j];
-        float step = (float)(2.0 * (double)M / ((double)g * (double)divisor));
-        v[j] = fmaf((float)y, step, -M);
+        float step = (float)(((double)M - (double)m) / ((double)g * (double)divisor));
+        v[j] = fmaf((float)y, step, m);
     }
+}
+
+void thc_oracle_estimate(const void *sum, uint32_t w, uint32_t divisor, uint64_t d_pad,
+                         uint32_t k, const float *scales, uint32_t g, float *v)
+{
+    float *lo = negated(scales, d_pad >> k);
+    thc_oracle_estimate_range(sum, w, divisor, d_pad, k, lo, scales, g, v);
+    free(lo);
+}
+
+void thc_oracle_decompress_range(const void *sum, uint32_t w, uint32_t divisor, uint64_t d,
+                                 uint32_t k, const float *lo, const float *hi, uint32_t g,
+                                 uint64_t seed, uint32_t round, float *out)
+{
+    uint64_t B = (uint64_t)1 << k;
+    uint64_t nb = (d + B - 1) / B;
+    uint64_t d_pad = nb * B;
+    float *v = (float *)malloc(sizeof(float) * d_pad);
+    thc_oracle_estimate_range(sum, w, divisor, d_pad, k, lo, hi, g, v);
+    thc_oracle_rht_inverse(v, d, k, seed, round, out);
+    free(v);
 }
 
 void thc_oracle_decompress(const void *sum, uint32_t w, uint32_t divisor, uint64_t d,
@@ -340,24 +386,21 @@ void thc_oracle_decompress(const void *sum, uint32_t w, uint32_t divisor, uint64
                            uint32_t round, float *out)
 {
     uint64_t B = (uint64_t)1 << k;
-    uint64_t nb = (d + B - 1) / B;
-    uint64_t d_pad = nb * B;
-    float *v = (float *)malloc(sizeof(float) * d_pad);
-    thc_oracle_estimate(sum, w, divisor, d_pad, k, scales, g, v);
-    thc_oracle_rht_inverse(v, d, k, seed, round, out);
-    free(v);
+    float *lo = negated(scales, (d + B - 1) / B);
+    thc_oracle_decompress_range(sum, w, divisor, d, k, lo, scales, g, seed, round, out);
+    free(lo);
 }
 
 /* ------------------------------------------------------------------------------------
  * Error feedback (Section 5.1; Algorithm 3, "Quantization error"): e = x - RHT^-1(X), where X
  * is the worker's own quantised vector in the rotated domain, X[j] = m + T[z[j]] (M - m)/g.
  * x has d entries, z has d_pad indices (unpacked).  X is evaluated like the estimate of a
- * one-worker aggregate (fma(T[z], 2M/g, -M)); the subtraction is one fp32 operation.
+ * one-worker aggregate (fma(T[z], (M-m)/g, m)); the subtraction is one fp32 operation.
  * The next round compresses grad + e (Algorithm 3, "x_i = grad_i + e_i").
  * ---------------------------------------------------------------------------------- */
-void thc_oracle_error_feedback(const float *x, const uint8_t *z, uint64_t d, uint32_t k,
-                               const float *scales, uint32_t g, const uint16_t *table,
-                               uint64_t seed, uint32_t round, float *e)
+void thc_oracle_error_feedback_range(const float *x, const uint8_t *z, uint64_t d, uint32_t k,
+                                     const float *lo, const float *hi, uint32_t g,
+                                     const uint16_t *table, uint64_t seed, uint32_t round, float *e)
 {
     uint64_t B = (uint64_t)1 << k;
     uint64_t nb = (d + B - 1) / B;
@@ -365,15 +408,25 @@ void thc_oracle_error_feedback(const float *x, const uint8_t *z, uint64_t d, uin
     float *v = (float *)malloc(sizeof(float) * d_pad);
     float *back = (float *)malloc(sizeof(float) * d);
     for (uint64_t j = 0; j < d_pad; ++j) {
-        float M = scales[j / B];
-        if (!(M > 0.0f) || !isfinite(M)) { v[j] = 0.0f; continue; }      /* R8 */
-        float step = (float)(2.0 * (double)M / (double)g);
-        v[j] = fmaf((float)table[z[j]], step, -M);
+        float m = lo[j / B], M = hi[j / B];
+        if (!(M > m) || !isfinite(M) || !isfinite(m)) { v[j] = 0.0f; continue; }   /* R8 */
+        float step = (float)(((double)M - (double)m) / (double)g);
+        v[j] = fmaf((float)table[z[j]], step, m);
     }
     thc_oracle_rht_inverse(v, d, k, seed, round, back);
     for (uint64_t j = 0; j < d; ++j) e[j] = x[j] - back[j];
     free(v);
     free(back);
+}
+
+void thc_oracle_error_feedback(const float *x, const uint8_t *z, uint64_t d, uint32_t k,
+                               const float *scales, uint32_t g, const uint16_t *table,
+                               uint64_t seed, uint32_t round, float *e)
+{
+    uint64_t B = (uint64_t)1 << k;
+    float *lo = negated(scales, (d + B - 1) / B);
+    thc_oracle_error_feedback_range(x, z, d, k, lo, scales, g, table, seed, round, e);
+    free(lo);
 }
 
 /* Value a single worker's index stands for on the real line, before the inverse RHT
@@ -387,4 +440,33 @@ void thc_oracle_dequantize(const uint8_t *z, uint64_t d_pad, uint32_t k, const f
         double M = (double)scales[j / B];
         value[j] = -M + (double)table[z[j]] * (2.0 * M / (double)g);
     }
+}
+
+/* ------------------------------------------------------------------------------------
+ * Exact range of the rotated coordinates (Algorithm 1's preliminary stage, "m = min_i m_i,
+ * M = max_i M_i", applied per RHT block after the rotation): lo[k], hi[k] = min and max over
+ * all n workers and all B coordinates of block k of RHT(x_i).  No coordinate is clamped with
+ * this range.  A block with a non-finite rotated coordinate gets the degenerate range (0, 0).
+ * x is [n][d].
+ * ---------------------------------------------------------------------------------- */
+void thc_oracle_ranges(const float *x, uint32_t n, uint64_t d, uint32_t k, uint64_t seed,
+                       uint32_t round, float *lo, float *hi)
+{
+    uint64_t B = (uint64_t)1 << k;
+    uint64_t nb = (d + B - 1) / B;
+    uint64_t d_pad = nb * B;
+    float *r = (float *)malloc(sizeof(float) * d_pad);
+    for (uint64_t blk = 0; blk < nb; ++blk) { lo[blk] = INFINITY; hi[blk] = -INFINITY; }
+    for (uint32_t i = 0; i < n; ++i) {
+        thc_oracle_rht_forward(x + (uint64_t)i * d, d, k, seed, round, r);
+        for (uint64_t j = 0; j < d_pad; ++j) {
+            uint64_t blk = j / B;
+            if (!isfinite(r[j])) { lo[blk] = NAN; hi[blk] = NAN; continue; }
+            if (r[j] < lo[blk]) lo[blk] = r[j];                           /* false once NaN */
+            if (r[j] > hi[blk]) hi[blk] = r[j];
+        }
+    }
+    for (uint64_t blk = 0; blk < nb; ++blk)
+        if (!isfinite(lo[blk]) || !isfinite(hi[blk])) { lo[blk] = 0.0f; hi[blk] = 0.0f; }
+    free(r);
 }

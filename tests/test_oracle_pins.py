@@ -586,3 +586,112 @@ def test_error_feedback_removes_the_truncation_bias_over_rounds():
     assert err_plain > 3 * err_ef
     # exactly: R * mean = R * grad - e^R (up to fp32 rounding of the additions)
     assert np.allclose(acc_ef, R * g64 - e, atol=2e-4 * R)
+
+
+# ------------------------------------------------- exact range (Algorithm 1's preliminary stage)
+def test_ranges_are_min_and_max_of_the_dense_rotation():
+    """(lo, hi) per block = min and max over workers and coordinates of (1/sqrt B) H D x,
+    written out with SciPy's dense Sylvester matrix in float64."""
+    k, n, d = 4, 3, 37                                     # three blocks of 16, the last ragged
+    c = cfg(k=k)
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((n, d)).astype(np.float32)
+    lo, hi = O.ranges(x, c, 5)
+    B = 1 << k
+    H = hadamard(B).astype(np.float64)
+    for blk in range(3):
+        vals = []
+        for i in range(n):
+            xp = np.zeros(3 * B)
+            xp[:d] = x[i]
+            s = O.signs(c.seed, 5, blk * B, B).astype(np.float64)
+            vals.append(H @ (s * xp[blk * B:(blk + 1) * B]) / np.sqrt(B))
+        vals = np.concatenate(vals)
+        assert abs(lo[blk] - vals.min()) <= 1e-6 and abs(hi[blk] - vals.max()) <= 1e-6
+        assert lo[blk] < 0.0 < hi[blk]
+
+
+def test_symmetric_range_is_the_special_case_lo_equals_minus_hi():
+    """The general [lo, hi] quantiser and decoder with lo = -M reproduce the Section 5.3 path
+    bit for bit (kappa = 1/(2M), offset = 1/2 exactly)."""
+    c = cfg(k=8)
+    rng = np.random.default_rng(3)
+    r = rng.standard_normal(4 * 256).astype(np.float32)
+    scl = np.array([0.7, 2.0, 1e-3, 3.3], np.float32)
+    z0 = O.quantize(r, scl, c, rnd=2, worker=1)
+    z1 = O.quantize(r, scl, c, rnd=2, worker=1, lo=-scl)
+    assert np.array_equal(z0, z1)
+    tot = O.aggregate(O.pack(z0, 4)[None, :], r.size, c, 8)
+    assert np.array_equal(O.estimate(tot, 1, scl, c).view(np.uint32),
+                          O.estimate(tot, 1, scl, c, lo=-scl).view(np.uint32))
+
+
+def test_exact_range_clamps_nothing_and_decodes_without_bias():
+    """With Algorithm 1's exact range no coordinate is truncated: the block's minimum gets
+    index 0 and decodes to lo, its maximum gets the last index and decodes to hi, and the
+    mean of the decoded value over independent rounding draws (different worker ids, same
+    rotation) approaches r at every coordinate, extremes included."""
+    k = 6
+    c = cfg(k=k)
+    rng = np.random.default_rng(19)
+    x = (rng.standard_normal((1, 64)) * np.exp(rng.standard_normal((1, 64)))).astype(np.float32)
+    lo, hi = O.ranges(x, c, 0)
+    r = O.rht_forward(x[0], c, 0)
+    assert r.min() == lo[0] and r.max() == hi[0]
+    draws = 4000
+    acc = np.zeros(64)
+    acc2 = np.zeros(64)
+    for wkr in range(draws):
+        z = O.quantize(r, hi, c, rnd=0, worker=wkr, lo=lo)
+        if wkr == 0:
+            assert z[np.argmin(r)] == 0 and z[np.argmax(r)] == 15
+        tot = O.aggregate(O.pack(z, 4)[None, :], 64, c, 8)
+        v = O.estimate(tot, 1, hi, c, lo=lo).astype(np.float64)
+        acc += v
+        acc2 += v * v
+    mean = acc / draws
+    sd = np.sqrt(np.maximum(acc2 / draws - mean ** 2, 0.0) / draws)
+    width = float(hi[0]) - float(lo[0])
+    assert np.all(np.abs(mean - r) <= 4.5 * sd + 3e-5 * width)
+    assert abs(mean[np.argmin(r)] - lo[0]) <= 1e-6 * width and abs(mean[np.argmax(r)] - hi[0]) <= 1e-6 * width
+
+
+def test_uniform_thc_is_textbook_usq_on_the_exact_range():
+    """Algorithm 1: identity table with g = 2^b - 1 on [m, M]: the index is floor((r-m)/(M-m) g)
+    or one more, and the estimate line is m + (X/n) (M-m)/(2^b-1)."""
+    b, g, k = 2, 3, 5
+    c = cfg(bits=b, g=g, table=(0, 1, 2, 3), k=k)
+    rng = np.random.default_rng(23)
+    x = rng.standard_normal((2, 32)).astype(np.float32)
+    lo, hi = O.ranges(x, c, 1)
+    width = float(hi[0]) - float(lo[0])
+    zs = []
+    for i in range(2):
+        r = O.rht_forward(x[i], c, 1)
+        z = O.quantize(r, hi, c, rnd=1, worker=i, lo=lo)
+        pos = (r.astype(np.float64) - float(lo[0])) / width * g
+        fl = np.minimum(np.floor(pos + 1e-9), g - 1)
+        assert np.all((z == fl) | (z == fl + 1) | (np.abs(pos - np.round(pos)) < 1e-5))
+        zs.append(z)
+    X = zs[0].astype(np.int64) + zs[1]
+    tot = O.aggregate(np.stack([O.pack(z, b) for z in zs]), 32, c, 8)
+    assert np.array_equal(tot.astype(np.int64), X)
+    v = O.estimate(tot, 2, hi, c, lo=lo)
+    expect = float(lo[0]) + X / 2.0 * width / (2 ** b - 1)
+    assert np.allclose(v, expect, rtol=0, atol=2e-6 * width)
+
+
+def test_exact_range_round_has_no_truncation_error_on_heavy_tails():
+    """Whole rounds on heavy-tailed input with a tight clamp (p = 1/2): the norm-based range
+    truncates and the error of the average stays large however many workers there are; the
+    exact range only has quantisation noise, which the average over workers shrinks."""
+    k, n, d = 8, 32, 512
+    tight = cfg(k=k, t_p=0.6744897501960817)               # p = 1/2
+    rng = np.random.default_rng(29)
+    base = (rng.standard_normal(d) * np.exp(1.5 * rng.standard_normal(d))).astype(np.float32)
+    x = np.tile(base, (n, 1))
+    out_norm = O.thc_round(x, tight, 3)["out"].astype(np.float64)
+    out_exact = O.thc_round(x, tight, 3, exact_range=True)["out"].astype(np.float64)
+    e_norm = ((out_norm - base) ** 2).sum() / (base.astype(np.float64) ** 2).sum()
+    e_exact = ((out_exact - base) ** 2).sum() / (base.astype(np.float64) ** 2).sum()
+    assert e_exact < 0.05 and e_norm > 5 * e_exact
