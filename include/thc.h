@@ -75,6 +75,9 @@ typedef struct thc_ctx thc_ctx;   /* opaque */
  *   acc_bits     width of the sums: 8, 16 or 32, or 0 = smallest with workers*g <= 2^w - 1
  *                (Section 8.4: the largest aggregate is g*n)
  */
+#define THC_RANGE_NORM   0u
+#define THC_RANGE_MINMAX 1u
+
 typedef struct thc_config {
     uint32_t bits;
     uint32_t granularity;
@@ -85,6 +88,10 @@ typedef struct thc_config {
     uint32_t in_dtype;
     uint32_t workers;
     uint32_t acc_bits;
+    uint32_t range_mode;   /* THC_RANGE_NORM (0): M = t_p max_i ||x_i|| / sqrt(B), m = -M (Section 5.3);
+                              THC_RANGE_MINMAX (1): the exact minimum and maximum of the rotated
+                              coordinates over all workers (Algorithm 1's preliminary stage applied
+                              after the RHT): nothing is clamped; fp32 input only */
 } thc_config;
 
 typedef struct thc_sizes_t {
@@ -96,6 +103,8 @@ typedef struct thc_sizes_t {
     uint64_t workspace_bytes;  /* scratch any call may need for this (d, n_local)      */
     uint32_t acc_bits;         /* the resolved accumulator width                       */
     uint32_t fused_scales;     /* 1: thc_prepare_compress is one launch for (d, n_local)  */
+    uint64_t scales_count;     /* floats in `scales`: nblocks, or 2 * nblocks (minima, then
+                                  maxima) in THC_RANGE_MINMAX mode                        */
 } thc_sizes_t;
 
 /* Validate `cfg` (host only) and build a context.  If a CUDA device is present, the
@@ -174,6 +183,17 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
 int thc_prepare_noalloc(const void *const *grads, uint32_t n, uint64_t d, uint32_t log2_block,
                         uint32_t in_dtype, double t_p, float *scales, uint32_t *status_or_null,
                         void *stream);
+
+/* The preliminary stage of Algorithm 1 ("m = min_i m_i, M = max_i M_i") applied per RHT block to
+ * the rotated coordinates: scales[k] = min and scales[nblocks + k] = max over all n workers and
+ * all coordinates of block k of RHT(x_i) for this `round` (the rotation depends on it).
+ * Contexts in THC_RANGE_MINMAX mode only (THC_EUNSUPPORTED otherwise; thc_prepare is their
+ * counterpart in THC_RANGE_NORM mode).  thc_compress, thc_quantize_rotated, thc_decompress and
+ * thc_error_feedback of such a context read `scales` in this layout and use the range
+ * [m, M] of Algorithm 2 as given: no coordinate is clamped.  Costs one transform pass over the
+ * inputs.  A block with a non-finite rotated coordinate gets (0, 0) and THC_STATUS_NONFINITE. */
+int thc_prepare_minmax(thc_ctx *ctx, const void *const *grads, uint32_t n, uint64_t d, uint32_t round,
+                       float *scales, void *workspace, uint64_t workspace_bytes, void *stream);
 
 /* thc_prepare and thc_compress in one launch, for callers that hold all n workers' gradients
  * (the simulated cluster): same arguments and results as the two calls in a row, `scales`

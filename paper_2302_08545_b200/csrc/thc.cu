@@ -22,7 +22,7 @@ struct PtrArray { const void *p[THC_MAX_WORKERS]; };
 struct MutPtrArray { void *p[THC_MAX_WORKERS]; };
 
 enum LoadKind { kLoadGradF32, kLoadGradBF16, kLoadSum8, kLoadSum16, kLoadSum32, kLoadRaw };
-enum StoreKind { kStoreRaw, kStoreQuant, kStoreOut };
+enum StoreKind { kStoreRaw, kStoreQuant, kStoreOut, kStoreRange };
 
 // Geometry of the tiles one launch walks.
 struct TileGeom {
@@ -41,6 +41,7 @@ struct TileGeom {
     uint32_t round;
     uint32_t worker_base;
     float    c_block;          // (float)(1/sqrt(B))
+    uint32_t exact_range;      // scales = nblocks minima then nblocks maxima (else M per block)
 };
 
 __device__ __forceinline__ uint64_t tile_base(const TileGeom &g, uint32_t tile)
@@ -136,13 +137,8 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
         // (1/(2M), 1/2) per block; (0, 0) for a degenerate block
         for (uint32_t b = tid; b < g.blocks_in_tile; b += kThreads) {
             float2 c = make_float2(0.f, 0.f);
-            if (first_blk + b < nblocks) {
-                const float M = scales[first_blk + b];
-                if (M > 0.0f && isfinite(M)) {
-                    c.x = (float)(1.0 / (2.0 * (double)M));
-                    c.y = 0.5f;
-                }
-            }
+            if (first_blk + b < nblocks)
+                c = compress_constants(block_range(scales, first_blk + b, nblocks, g.exact_range));
             blk_const[b] = c;
         }
         if (!IDENTITY) {
@@ -154,13 +150,9 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
         // (step, -M) per block; (0, 0) for a degenerate block
         for (uint32_t b = tid; b < g.blocks_in_tile; b += kThreads) {
             float2 c = make_float2(0.f, 0.f);
-            if (first_blk + b < nblocks) {
-                const float M = scales[first_blk + b];
-                if (M > 0.0f && isfinite(M)) {
-                    c.x = (float)(2.0 * (double)M / ((double)g.granularity * (double)g.divisor));
-                    c.y = -M;
-                }
-            }
+            if (first_blk + b < nblocks)
+                c = decode_constants(block_range(scales, first_blk + b, nblocks, g.exact_range),
+                                     g.granularity, g.divisor);
             blk_const[b] = c;
         }
     }
@@ -282,6 +274,29 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
             else if constexpr (BITS == 2) *reinterpret_cast<uint16_t *>(pk + j / 4) = (uint16_t)z;
             else pk[j / 8] = (unsigned char)z;
         }
+    } else if (STORE == kStoreRange) {
+        // min / max of the rotated coordinates per RHT block, as ordered keys: out.p[0] holds
+        // nblocks min keys followed by nblocks max keys.  For blocks of at least 128
+        // coordinates the 32 chunks of a warp lie in one block and are reduced first.
+        uint32_t *rk = static_cast<uint32_t *>(out.p[0]);
+#pragma unroll 1
+        for (int i = 0; i < kTileChunks / kThreads; ++i) {
+            const int c = tid + i * kThreads;
+            const uint64_t j = chunk_coord(g, base, c);
+            if (j >= g.d_pad) continue;
+            const float4 v = scale4(tile[swz(c)], g.c_block);
+            const uint32_t k0 = float_key(v.x), k1 = float_key(v.y), k2 = float_key(v.z), k3 = float_key(v.w);
+            uint32_t kmin = min(min(k0, k1), min(k2, k3));
+            uint32_t kmax = max(max(k0, k1), max(k2, k3));
+            const uint64_t blk = j >> g.k;
+            if (g.k >= 7) {
+                kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+                kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+                if ((tid & 31) != 0) continue;
+            }
+            atomicMin(rk + blk, kmin);
+            atomicMax(rk + nblocks + blk, kmax);
+        }
     } else {   // kStoreOut
         float *o = static_cast<float *>(out.p[0]);
 #pragma unroll 4
@@ -306,7 +321,7 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
 template <int BITS, bool IDENTITY>
 __global__ void __launch_bounds__(kThreads)
 quantize_rotated_kernel(PtrArray rotated, MutPtrArray packed, uint64_t d_pad, uint32_t k,
-                        uint32_t granularity, uint32_t round, uint32_t worker_base,
+                        uint32_t granularity, uint32_t round, uint32_t worker_base, uint32_t exact_range,
                         const float *__restrict__ scales, const DeviceBlock *dev, PhiloxKeys keys)
 {
     __shared__ uint4 lut[256];
@@ -322,12 +337,8 @@ quantize_rotated_kernel(PtrArray rotated, MutPtrArray packed, uint64_t d_pad, ui
         const float4 a = __ldg(reinterpret_cast<const float4 *>(rot + j));
         const float4 b = __ldg(reinterpret_cast<const float4 *>(rot + j + 4));
         const float r[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-        const float M = scales[j >> k];
-        float kappa = 0.f, offset = 0.f;
-        if (M > 0.0f && isfinite(M)) {
-            kappa = (float)(1.0 / (2.0 * (double)M));
-            offset = 0.5f;
-        }
+        const float2 kc = compress_constants(block_range(scales, j >> k, d_pad >> k, exact_range));
+        const float kappa = kc.x, offset = kc.y;
         const uint4 rnd = round_call(j, worker_base + wl, round, keys);
         const uint64_t z = quantize8<BITS, IDENTITY>(r, kappa, offset, gf, rnd, lut, 1);
         if constexpr (BITS == 8) *reinterpret_cast<uint2 *>(pk + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
@@ -491,6 +502,28 @@ prepare_final_kernel(const double *__restrict__ partial, uint32_t n, uint64_t nb
     if (flags) atomicOr(&dev->status, flags);
 }
 
+// Exact range (Algorithm 1's preliminary stage on the rotated coordinates): keys start at
+// (+max, 0); afterwards they become nblocks minima followed by nblocks maxima in `scales`.
+// A block with a non-finite rotated coordinate gets (0, 0) and THC_STATUS_NONFINITE.
+__global__ void range_init_kernel(uint32_t *keys, uint64_t nblocks)
+{
+    const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < nblocks) { keys[i] = 0xFFFFFFFFu; keys[nblocks + i] = 0u; }
+}
+
+__global__ void range_final_kernel(const uint32_t *keys, uint64_t nblocks, float *scales, DeviceBlock *dev)
+{
+    const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nblocks) return;
+    float lo = key_float(keys[i]), hi = key_float(keys[nblocks + i]);
+    uint32_t flags = 0;
+    if (!isfinite(lo) || !isfinite(hi)) { lo = 0.0f; hi = 0.0f; flags |= THC_STATUS_NONFINITE; }
+    if (!(hi > lo)) flags |= THC_STATUS_ZERO_BLOCK;
+    scales[i] = lo;
+    scales[nblocks + i] = hi;
+    if (flags) atomicOr(&dev->status, flags);
+}
+
 // ---------------------------------------------------------------------------- aggregate
 // Y[j] = sum_i T[z_i[j]] (Algorithm 2, PS line).  One thread per 32 coordinates.
 template <int BITS, int W>
@@ -638,6 +671,8 @@ static int validate_config(const thc_config *c, uint32_t *acc_bits, bool *identi
     if (c->log2_block < 3 || c->log2_block > 22) return THC_EINVAL;
     if (c->in_dtype != THC_F32 && c->in_dtype != THC_BF16) return THC_EINVAL;
     if (c->workers == 0 || c->workers > THC_MAX_WORKERS) return THC_EINVAL;
+    if (c->range_mode != THC_RANGE_NORM && c->range_mode != THC_RANGE_MINMAX) return THC_EINVAL;
+    if (c->range_mode == THC_RANGE_MINMAX && c->in_dtype != THC_F32) return THC_EUNSUPPORTED;
     const uint64_t max_sum = (uint64_t)c->workers * c->granularity;
     uint32_t w = c->acc_bits;
     if (w == 0) w = max_sum <= 0xFFu ? 8 : max_sum <= 0xFFFFu ? 16 : 32;
@@ -760,6 +795,7 @@ static PipePlan plan_pipeline(const thc_ctx *ctx, uint64_t wb_count)
 static bool plan_pipeline_fused(const thc_ctx *ctx, uint64_t nblocks, uint32_t n, PipePlan *out)
 {
     if (ctx->cfg.log2_block != 20 || ctx->cfg.in_dtype != THC_F32) return false;
+    if (ctx->cfg.range_mode != THC_RANGE_NORM) return false;
     const uint64_t wb_count = nblocks * n;
     PipePlan p = plan_pipeline(ctx, wb_count);
     const uint64_t window = p.ring - p.lag;
@@ -788,12 +824,13 @@ int thc_sizes(const thc_ctx *ctx, uint64_t d, uint32_t n_local, thc_sizes_t *s)
     s->sum_bytes = s->d_pad * ctx->acc_bits / 8;
     s->rotated_bytes = s->d_pad * 4;
     s->acc_bits = ctx->acc_bits;
+    s->scales_count = ctx->cfg.range_mode == THC_RANGE_MINMAX ? 2 * s->nblocks : s->nblocks;
     const uint32_t chunk_log2 = k < (uint32_t)kTileLog2 ? k : (uint32_t)kTileLog2;
     const uint64_t prepare_ws = (uint64_t)n_local * (s->d_pad >> chunk_log2) * 8;
     uint64_t two_pass_ws = 0;
     if (k > (uint32_t)kTileLog2) {
         const PipePlan pl = plan_pipeline(ctx, s->nblocks * n_local);
-        two_pass_ws = (uint64_t)pl.ring * B * 4;
+        two_pass_ws = (uint64_t)pl.ring * B * 4 + s->nblocks * 8;       // + range keys
         PipePlan pf;
         if (plan_pipeline_fused(ctx, s->nblocks, n_local, &pf)) {
             const uint64_t fused_ws = (uint64_t)pf.ring * B * 4 + s->nblocks * n_local * (B >> kPLog2) * 8;
@@ -834,6 +871,7 @@ int thc_prepare(thc_ctx *ctx, const void *const *grads, uint32_t n, uint64_t d, 
     if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint32_t k = ctx->cfg.log2_block;
+    if (ctx->cfg.range_mode == THC_RANGE_MINMAX) return THC_EUNSUPPORTED;   // thc_prepare_minmax
     const uint32_t chunk_log2 = k < (uint32_t)kTileLog2 ? k : (uint32_t)kTileLog2;
     const uint64_t chunks_per_worker = sz.d_pad >> chunk_log2;
     const uint64_t chunks_per_block = 1ull << (k - chunk_log2);
@@ -928,6 +966,7 @@ static TileGeom base_geom(const thc_ctx *ctx, const thc_sizes_t &sz, uint64_t d,
     g.granularity = ctx->cfg.granularity;
     g.round = round;
     g.c_block = (float)(1.0 / sqrt((double)(1ull << g.k)));
+    g.exact_range = ctx->cfg.range_mode == THC_RANGE_MINMAX ? 1u : 0u;
     return g;
 }
 
@@ -947,7 +986,9 @@ typedef void (*pipe_kernel_t)(const TmaMaps, PipeParams, PtrArrayP, MutPtrArrayP
 template <int MODE, int KB>
 static pipe_kernel_t pick_pipe_kernel_kb(uint32_t bits, bool identity)
 {
-    if constexpr (MODE == kErrorFeedback) {
+    if constexpr (MODE == kRangeF32) {
+        return thc_pipeline_kernel<MODE, 4, true, KB>;
+    } else if constexpr (MODE == kErrorFeedback) {
         switch (bits) {
         case 1: return thc_pipeline_kernel<MODE, 1, true, KB>;
         case 2: return thc_pipeline_kernel<MODE, 2, true, KB>;
@@ -1046,6 +1087,10 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
     P.round = round;
     P.worker_base = worker_base;
     P.c_block = (float)(1.0 / sqrt((double)(1ull << k)));
+    P.exact_range = ctx->cfg.range_mode == THC_RANGE_MINMAX ? 1u : 0u;
+    P.nblocks = (uint32_t)sz.nblocks;
+    P.range_keys = reinterpret_cast<uint32_t *>(static_cast<unsigned char *>(workspace) +
+                                                ((uint64_t)pl.ring << k) * 4);
     const uint64_t nblk_cached = sz.nblocks < (uint64_t)kBlockConstMax ? sz.nblocks : (uint64_t)kBlockConstMax;
     const size_t smem = (size_t)1024 + (size_t)2 * kPElems * 4 + kPSignWords * 4 +
                         (size_t)(ctx->cfg.granularity + 1) * kLutRep * 16 + (size_t)nblk_cached * 8;
@@ -1067,6 +1112,62 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
         }
     }
     kern<<<pl.grid, kPCtaThreads, smem, st>>>(maps, P, in, out, rot, ctx->keys);
+    THC_CUDA(cudaGetLastError());
+    return THC_OK;
+}
+
+// thc_prepare in exact-range mode (Algorithm 1's preliminary stage on the rotated coordinates):
+// one transform pass over all workers whose epilogue only takes the minimum and maximum, then
+// the keys become the (lo, hi) planes of `scales`.  This costs about as much as the transform
+// half of thc_compress: the price of a range that clamps nothing.
+int thc_prepare_minmax(thc_ctx *ctx, const void *const *grads, uint32_t n, uint64_t d, uint32_t round,
+                       float *scales, void *workspace, uint64_t workspace_bytes, void *stream)
+{
+    int rc0 = check_launch_ctx(ctx);
+    if (rc0 != THC_OK) return rc0;
+    if (ctx->cfg.range_mode != THC_RANGE_MINMAX) return THC_EUNSUPPORTED;
+    thc_sizes_t sz;
+    if ((rc0 = thc_sizes(ctx, d, n, &sz)) != THC_OK) return rc0;
+    if ((rc0 = check_ptr_array(grads, n)) != THC_OK) return rc0;
+    if (scales == nullptr || workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
+    if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint32_t k = ctx->cfg.log2_block;
+    const bool two_pass = k > (uint32_t)kTileLog2;
+    uint32_t *keys = static_cast<uint32_t *>(workspace);
+    if (two_pass) {
+        const PipePlan pl = plan_pipeline(ctx, sz.nblocks * n);
+        keys = reinterpret_cast<uint32_t *>(static_cast<unsigned char *>(workspace) + ((uint64_t)pl.ring << k) * 4);
+    }
+    const unsigned init_blocks = (unsigned)((sz.nblocks + 255) / 256);
+    range_init_kernel<<<init_blocks, 256, 0, st>>>(keys, sz.nblocks);
+    THC_CUDA(cudaGetLastError());
+    int rc;
+    if (!two_pass) {
+        PtrArray in;
+        MutPtrArray out, rot;
+        memset(&in, 0, sizeof in);
+        memset(&out, 0, sizeof out);
+        memset(&rot, 0, sizeof rot);
+        for (uint32_t i = 0; i < n; ++i) in.p[i] = grads[i];
+        out.p[0] = keys;
+        TileGeom g = base_geom(ctx, sz, d, round);
+        geom_pass_a(g);
+        const uint64_t tiles = (sz.d_pad + kTileElems - 1) / kTileElems;
+        rc = launch_tile(ctx, pick_tile_kernel<kLoadGradF32, kStoreRange>(4, true), g, tiles, n, in, out, rot,
+                         scales, st);
+    } else {
+        PtrArrayP pin;
+        MutPtrArrayP pout, prot;
+        memset(&pin, 0, sizeof pin);
+        memset(&pout, 0, sizeof pout);
+        memset(&prot, 0, sizeof prot);
+        for (uint32_t i = 0; i < n; ++i) pin.p[i] = grads[i];
+        rc = launch_pipeline(ctx, pick_pipe_kernel<kRangeF32>(4, true, k), true, sz, d, n, 0, round,
+                             1, scales, workspace, pin, pout, prot, st);
+    }
+    if (rc != THC_OK) return rc;
+    range_final_kernel<<<init_blocks, 256, 0, st>>>(keys, sz.nblocks, scales, ctx->dev);
     THC_CUDA(cudaGetLastError());
     return THC_OK;
 }
@@ -1240,7 +1341,8 @@ int thc_quantize_rotated(thc_ctx *ctx, const float *const *rotated, uint32_t n_l
     const dim3 grid((unsigned)blocks, n_local);
     const uint32_t k = ctx->cfg.log2_block, g = ctx->cfg.granularity;
 #define THC_QR(B, I) quantize_rotated_kernel<B, I><<<grid, kThreads, 0, st>>>( \
-        in, out, sz.d_pad, k, g, round, worker_base, scales, ctx->dev, ctx->keys)
+        in, out, sz.d_pad, k, g, round, worker_base,                         \
+        ctx->cfg.range_mode == THC_RANGE_MINMAX ? 1u : 0u, scales, ctx->dev, ctx->keys)
     switch (ctx->cfg.bits) {
     case 1: if (ctx->identity) THC_QR(1, true); else THC_QR(1, false); break;
     case 2: if (ctx->identity) THC_QR(2, true); else THC_QR(2, false); break;

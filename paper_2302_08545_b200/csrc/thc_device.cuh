@@ -68,6 +68,50 @@ __device__ __forceinline__ uint4 round_call(uint64_t j, uint32_t worker, uint32_
     return philox4x32_10((uint32_t)call, (uint32_t)(call >> 32), worker, round, keys);
 }
 
+// ------------------------------------------------------------------------ clamp range
+// Range [lo, hi] of an RHT block (Algorithm 2's m and M).  Norm mode (Section 5.3): the
+// scales array holds M per block and m = -M.  Exact mode (Algorithm 1's preliminary stage
+// applied to the rotated coordinates): it holds nblocks minima followed by nblocks maxima.
+struct BlockRange { float lo, hi; };
+
+__device__ __forceinline__ BlockRange block_range(const float *scales, uint64_t r, uint64_t nblocks,
+                                                  uint32_t exact)
+{
+    BlockRange b;
+    if (exact) { b.lo = scales[r]; b.hi = scales[nblocks + r]; }
+    else { b.hi = scales[r]; b.lo = -b.hi; }
+    return b;
+}
+
+// (kappa, offset) of u = sat(fma(r, kappa, offset)): 1/(hi - lo) and -lo/(hi - lo), which for
+// lo = -hi are 1/(2M) and exactly 1/2; (0, 0) marks a degenerate block (every index 0).
+__device__ __forceinline__ float2 compress_constants(BlockRange b)
+{
+    if (!(b.hi > b.lo) || !isfinite(b.hi) || !isfinite(b.lo)) return make_float2(0.f, 0.f);
+    const double w = (double)b.hi - (double)b.lo;
+    return make_float2((float)(1.0 / w), (float)(-(double)b.lo / w));
+}
+
+// (step, base) of v = fma(Y, step, base): (hi - lo)/(g * divisor) and lo; (0, 0) for a
+// degenerate block (decodes to zeros).
+__device__ __forceinline__ float2 decode_constants(BlockRange b, uint32_t g, uint32_t divisor)
+{
+    if (!(b.hi > b.lo) || !isfinite(b.hi) || !isfinite(b.lo)) return make_float2(0.f, 0.f);
+    const double w = (double)b.hi - (double)b.lo;
+    return make_float2((float)(w / ((double)g * (double)divisor)), b.lo);
+}
+
+// Order-preserving map of fp32 bit patterns onto unsigned integers (for atomic min / max).
+__device__ __forceinline__ uint32_t float_key(float f)
+{
+    const uint32_t u = __float_as_uint(f);
+    return u ^ ((u >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k)
+{
+    return __uint_as_float(k ^ ((k >> 31) ? 0x80000000u : 0xFFFFFFFFu));
+}
+
 // ---------------------------------------------------------------- packed fp32 arithmetic
 __device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
 

@@ -53,7 +53,8 @@ constexpr uint32_t kMaxPolls = 1u << 21;
 
 enum PipeMode { kCompressF32, kCompressBF16, kDecompress8, kDecompress16, kDecompress32,
                 kCompressF32Fused,     // fp32 compress that also computes the block scales (below)
-                kErrorFeedback };      // e_i = x_i - RHT^-1(X_i) from worker i's own packed indices
+                kErrorFeedback,        // e_i = x_i - RHT^-1(X_i) from worker i's own packed indices
+                kRangeF32 };           // exact min / max of the rotated coordinates per RHT block
 
 // Layout inside DeviceBlock::counters.  Every CTA hits `head` and `abort` for every task and
 // the completion counters of the slots in use: each gets its own 128-byte line (head, exited,
@@ -91,6 +92,9 @@ struct PipeParams {
     double  *tile_sq;          // wb_count * T sums of squares, one per pass-A tile
     float   *scales_out;       // = scales, written by the kernel
     double   t_p;
+    uint32_t exact_range;      // scales = nblocks minima then nblocks maxima (else M per block)
+    uint32_t nblocks;
+    uint32_t *range_keys;      // range mode: nblocks min keys then nblocks max keys
 };
 
 struct PtrArrayP { const void *p[THC_MAX_WORKERS]; };
@@ -329,19 +333,9 @@ __device__ __forceinline__ TaskId decode_task(uint32_t q, const PipeParams &P)
 }
 
 template <bool COMPRESS>
-__device__ __forceinline__ float2 block_constants(float M, uint32_t g, uint32_t divisor)
+__device__ __forceinline__ float2 block_constants(BlockRange b, uint32_t g, uint32_t divisor)
 {
-    float2 c = make_float2(0.f, 0.f);
-    if (M > 0.0f && isfinite(M)) {
-        if (COMPRESS) {
-            c.x = (float)(1.0 / (2.0 * (double)M));
-            c.y = 0.5f;
-        } else {
-            c.x = (float)(2.0 * (double)M / ((double)g * (double)divisor));
-            c.y = -M;
-        }
-    }
-    return c;
+    return COMPRESS ? compress_constants(b) : decode_constants(b, g, divisor);
 }
 
 // ------------------------------------------------------------------ in-place tile rounds
@@ -564,12 +558,25 @@ struct EpilogueCtx {
     int words_per_row;
 };
 
-template <bool COMPRESS, int BITS, bool IDENTITY>
+// RANGE: the unit only feeds the running minimum / maximum (as ordered keys) of the rotated
+// coordinates (Algorithm 1's preliminary stage).
+template <bool COMPRESS, int BITS, bool IDENTITY, bool RANGE = false>
 __device__ __forceinline__ void epilogue_unit(const float4 &va, const float4 &vb, uint64_t j, int row,
-                                              int uu, const EpilogueCtx &ep, const PhiloxKeys &keys)
+                                              int uu, const EpilogueCtx &ep, const PhiloxKeys &keys,
+                                              uint32_t &kmin, uint32_t &kmax)
 {
     const float4 ra = scale4(va, ep.c_block);
     const float4 rb = scale4(vb, ep.c_block);
+    if constexpr (RANGE) {
+        const float r[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const uint32_t key = float_key(r[e]);
+            kmin = min(kmin, key);
+            kmax = max(kmax, key);
+        }
+        return;
+    }
     if (COMPRESS) {
         if (ep.rotated != nullptr) {
             *reinterpret_cast<float4 *>(ep.rotated + j) = ra;
@@ -610,9 +617,10 @@ __device__ __forceinline__ void epilogue_unit(const float4 &va, const float4 &vb
 
 // Last round of a pass-B tile, any geometry: the top E row bits, each thread owning 2^E rows
 // of one 8-coordinate unit, followed by the epilogue on the registers.
-template <int E, bool COMPRESS, int BITS, bool IDENTITY>
+template <int E, bool COMPRESS, int BITS, bool IDENTITY, bool RANGE>
 __device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, int ccl, int tid,
-                                                  const EpilogueCtx &ep, const PhiloxKeys &keys)
+                                                  const EpilogueCtx &ep, const PhiloxKeys &keys,
+                                                  uint32_t &kmin, uint32_t &kmax)
 {
     constexpr int N = 1 << E;
     const int ul = ccl - 1;                            // log2 units per row
@@ -642,7 +650,7 @@ __device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, in
         for (int m = 0; m < N; ++m) {
             const int row = row_low + (m << rl);
             const uint64_t j = ep.j_tile + ((uint64_t)row << kPLog2) + 8 * uu;
-            epilogue_unit<COMPRESS, BITS, IDENTITY>(a[m], b[m], j, row, uu, ep, keys);
+            epilogue_unit<COMPRESS, BITS, IDENTITY, RANGE>(a[m], b[m], j, row, uu, ep, keys, kmin, kmax);
         }
     }
 }
@@ -651,9 +659,10 @@ __device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, in
 // Thread (u = tid & 3, rl from bits 2..5, h = tid >> 6) owns unit 4h + u of rows rl + 16 m,
 // m = 0..7; lanes 0-7 of a quarter warp cover four units of two adjacent rows, whose XOR
 // patterns differ in bit 0, so both chunk reads are conflict-free.
-template <bool COMPRESS, int BITS, bool IDENTITY>
+template <bool COMPRESS, int BITS, bool IDENTITY, bool RANGE>
 __device__ __forceinline__ void pass_b_last_round_kb7(float4 *tile, int tid,
-                                                      const EpilogueCtx &ep, const PhiloxKeys &keys)
+                                                      const EpilogueCtx &ep, const PhiloxKeys &keys,
+                                                      uint32_t &kmin, uint32_t &kmax)
 {
     const int u = tid & 3;
     const int rl = ((tid >> 2) & 1) | (((tid >> 3) & 7) << 1);
@@ -682,8 +691,8 @@ __device__ __forceinline__ void pass_b_last_round_kb7(float4 *tile, int tid,
     const uint64_t j0 = ep.j_tile + ((uint64_t)rl << kPLog2) + 8 * uu;
 #pragma unroll 2
     for (int m = 0; m < 8; ++m)
-        epilogue_unit<COMPRESS, BITS, IDENTITY>(pa[m << 7], pb[m << 7], j0 + ((uint64_t)m << (kPLog2 + 4)),
-                                                rl + 16 * m, uu, ep, keys);
+        epilogue_unit<COMPRESS, BITS, IDENTITY, RANGE>(pa[m << 7], pb[m << 7], j0 + ((uint64_t)m << (kPLog2 + 4)),
+                                                       rl + 16 * m, uu, ep, keys, kmin, kmax);
 }
 
 // ------------------------------------------------------------------------------ the kernel
@@ -695,7 +704,8 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
 {
     constexpr bool kFused = MODE == kCompressF32Fused;
     constexpr bool kEF = MODE == kErrorFeedback;
-    constexpr bool kF32In = MODE == kCompressF32 || kFused;
+    constexpr bool kRange = MODE == kRangeF32;       // pass A as compress, epilogue = min / max
+    constexpr bool kF32In = MODE == kCompressF32 || kFused || kRange;
     constexpr bool kCompress = kF32In || MODE == kCompressBF16;
     extern __shared__ __align__(1024) unsigned char pipe_smem_raw[];
     // TMA's 128-byte swizzle needs the tile buffers on 1024-byte boundaries of the shared
@@ -727,7 +737,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
         mbar_init(&s_done, kPThreads);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (kCompress && !IDENTITY) {
+    if (kCompress && !IDENTITY && !kRange) {
         for (int idx = tid; idx < (int)(P.granularity + 1) * kLutRep; idx += kPCtaThreads)
             lut[idx] = P.dev->lut[idx / kLutRep];
     }
@@ -740,9 +750,9 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
     }
     const uint32_t nblk_total = (uint32_t)(P.d_pad >> P.k);
     const uint32_t nblk_cached = nblk_total < (uint32_t)kBlockConstMax ? nblk_total : (uint32_t)kBlockConstMax;
-    if (!kFused) {
+    if (!kFused && !kRange) {
         for (uint32_t b = tid; b < nblk_cached; b += kPCtaThreads)
-            blk_const[b] = block_constants<kCompress>(P.scales[b], P.granularity, P.divisor);
+            blk_const[b] = block_constants<kCompress>(block_range(P.scales, b, P.nblocks, P.exact_range), P.granularity, P.divisor);
     }
     __syncthreads();
 
@@ -936,7 +946,10 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 }
                 if (lane == 0 && t.is_b) {
                     if (kFused) {
-                        const float2 c = block_constants<true>(ld_relaxed_f32(P.scales + r), P.granularity, P.divisor);
+                        BlockRange br;
+                        br.hi = ld_relaxed_f32(P.scales + r);
+                        br.lo = -br.hi;
+                        const float2 c = compress_constants(br);
                         ti.bcx = c.x; ti.bcy = c.y;
                     }
                     // the ring was written through the generic proxy; the TMA unit reads it
@@ -1043,8 +1056,9 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
             const uint32_t slot = me.slot;
             const uint32_t idx = me.idx;
             const float2 bc = kFused ? make_float2(me.bcx, me.bcy)
+                              : kRange ? make_float2(0.f, 0.f)
                               : r < nblk_cached ? blk_const[r]
-                                                : block_constants<kCompress>(P.scales[r], P.granularity, P.divisor);
+                                                : block_constants<kCompress>(block_range(P.scales, r, P.nblocks, P.exact_range), P.granularity, P.divisor);
 
             if (!is_b) {
                 // ================================ pass A: tile idx of worker-block wb
@@ -1098,17 +1112,26 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     }
                 }
                 compute_barrier();
+                uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
                 if (KB == 7) {
-                    pass_b_last_round_kb7<kCompress, BITS, IDENTITY>(tile, tid, ep, keys);
+                    pass_b_last_round_kb7<kCompress, BITS, IDENTITY, kRange>(tile, tid, ep, keys, kmin, kmax);
                 } else {
                     const int rem = kb - e1;
                     const int e_last = rem < 3 ? rem : 3;
                     if (rem > e_last) p_rounds(tile, ccl + e1, ccl + kb - e_last, tid);
                     switch (e_last) {
-                    case 3: pass_b_last_round<3, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
-                    case 2: pass_b_last_round<2, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
-                    case 1: pass_b_last_round<1, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
-                    default: pass_b_last_round<0, kCompress, BITS, IDENTITY>(tile, kb, ccl, tid, ep, keys); break;
+                    case 3: pass_b_last_round<3, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, ep, keys, kmin, kmax); break;
+                    case 2: pass_b_last_round<2, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, ep, keys, kmin, kmax); break;
+                    case 1: pass_b_last_round<1, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, ep, keys, kmin, kmax); break;
+                    default: pass_b_last_round<0, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, ep, keys, kmin, kmax); break;
+                    }
+                }
+                if (kRange) {
+                    kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+                    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+                    if ((tid & 31) == 0) {
+                        atomicMin(P.range_keys + r, kmin);
+                        atomicMax(P.range_keys + P.nblocks + r, kmax);
                     }
                 }
             }

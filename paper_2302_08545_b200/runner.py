@@ -9,11 +9,13 @@ from . import thc
 from .workloads import Workload
 
 
-def context_for(w: Workload, workers: int | None = None, acc_bits: int = 0) -> thc.Context:
+def context_for(w: Workload, workers: int | None = None, acc_bits: int = 0,
+                exact_range: bool = False) -> thc.Context:
     return thc.Context(bits=w.bits, granularity=w.granularity, table=w.table, t_p=w.t_p,
                        log2_block=w.log2_block, seed=w.seed,
                        in_dtype=thc.THC_BF16 if w.in_dtype == "bf16" else thc.THC_F32,
-                       workers=w.n if workers is None else workers, acc_bits=acc_bits)
+                       workers=w.n if workers is None else workers, acc_bits=acc_bits,
+                       range_mode=1 if exact_range else 0)
 
 
 class Round:
@@ -27,7 +29,7 @@ class Round:
         self.device = dev
         gdt = torch.float32 if in_dtype == "f32" else torch.bfloat16
         self.grads = [torch.zeros(d, dtype=gdt, device=dev) for _ in range(n)]
-        self.scales = torch.zeros(self.sz.nblocks, dtype=torch.float32, device=dev)
+        self.scales = torch.zeros(self.sz.scales_count, dtype=torch.float32, device=dev)
         self.packed = [torch.zeros(self.sz.packed_bytes, dtype=torch.uint8, device=dev)
                        for _ in range(n)]
         self.total = torch.zeros(self.sz.sum_bytes, dtype=torch.uint8, device=dev)
@@ -52,6 +54,9 @@ class Round:
     # -- the four calls
     def prepare(self, stream=None):
         self.ctx.prepare(self.grads, self.d, self.scales, self.workspace, stream)
+
+    def prepare_minmax(self, rnd: int = 0, stream=None):
+        self.ctx.prepare_minmax(self.grads, self.d, rnd, self.scales, self.workspace, stream)
 
     def compress(self, rnd: int = 0, stream=None):
         self.ctx.compress(self.grads, self.d, rnd, self.scales, self.packed, self.workspace,

@@ -21,7 +21,7 @@ STATUS_NONFINITE, STATUS_ZERO_BLOCK, STATUS_WAIT_TIMEOUT = 1, 2, 4
 
 EXPORTS = ("thc_create", "thc_destroy", "thc_sizes", "thc_prepare", "thc_compress",
            "thc_quantize_rotated", "thc_aggregate", "thc_decompress", "thc_prepare_noalloc",
-           "thc_error_feedback", "thc_accumulate_error", "thc_prepare_compress", "thc_debug_skip_tasks", "thc_status", "thc_strerror", "thc_version")
+           "thc_error_feedback", "thc_accumulate_error", "thc_prepare_compress", "thc_prepare_minmax", "thc_debug_skip_tasks", "thc_status", "thc_strerror", "thc_version")
 NOALLOC_SCRATCH_BYTES = 4 << 20
 
 
@@ -36,14 +36,15 @@ class _Config(ctypes.Structure):
                 ("table", ctypes.c_uint16 * 256), ("t_p", ctypes.c_double),
                 ("log2_block", ctypes.c_uint32), ("seed", ctypes.c_uint64),
                 ("in_dtype", ctypes.c_uint32), ("workers", ctypes.c_uint32),
-                ("acc_bits", ctypes.c_uint32)]
+                ("acc_bits", ctypes.c_uint32), ("range_mode", ctypes.c_uint32)]
 
 
 class _Sizes(ctypes.Structure):
     _fields_ = [("d_pad", ctypes.c_uint64), ("nblocks", ctypes.c_uint64),
                 ("packed_bytes", ctypes.c_uint64), ("sum_bytes", ctypes.c_uint64),
                 ("rotated_bytes", ctypes.c_uint64), ("workspace_bytes", ctypes.c_uint64),
-                ("acc_bits", ctypes.c_uint32), ("fused_scales", ctypes.c_uint32)]
+                ("acc_bits", ctypes.c_uint32), ("fused_scales", ctypes.c_uint32),
+                ("scales_count", ctypes.c_uint64)]
 
 
 @dataclass(frozen=True)
@@ -56,6 +57,7 @@ class Sizes:
     workspace_bytes: int
     acc_bits: int
     fused_scales: int = 0
+    scales_count: int = 0
 
 
 def lib():
@@ -78,6 +80,7 @@ def lib():
     L.thc_aggregate.argtypes = [vp, pp, u32, u64, vp, vp]
     L.thc_decompress.argtypes = [vp, vp, u32, u64, u32, vp, vp, vp, u64, vp]
     L.thc_prepare_noalloc.argtypes = [pp, u32, u64, u32, u32, ctypes.c_double, vp, vp, vp]
+    L.thc_prepare_minmax.argtypes = [vp, pp, u32, u64, u32, vp, vp, u64, vp]
     L.thc_prepare_compress.argtypes = [vp, pp, u32, u32, u64, u32, vp, pp, pp, vp, u64, vp]
     L.thc_error_feedback.argtypes = [vp, pp, pp, u32, u64, u32, vp, pp, vp, u64, vp]
     L.thc_accumulate_error.argtypes = [vp, pp, pp, u32, u64, vp]
@@ -146,13 +149,15 @@ class Context:
     """Owns a ``thc_ctx``.  Methods mirror the C entry points one to one."""
 
     def __init__(self, bits: int, granularity: int, table, t_p: float, log2_block: int,
-                 seed: int, in_dtype: int = THC_F32, workers: int = 8, acc_bits: int = 0):
+                 seed: int, in_dtype: int = THC_F32, workers: int = 8, acc_bits: int = 0,
+                 range_mode: int = 0):
         cfg = _Config()
         cfg.bits, cfg.granularity = bits, granularity
         for i, v in enumerate(table):
             cfg.table[i] = int(v)
         cfg.t_p, cfg.log2_block, cfg.seed = float(t_p), log2_block, seed & 0xFFFFFFFFFFFFFFFF
         cfg.in_dtype, cfg.workers, cfg.acc_bits = in_dtype, workers, acc_bits
+        cfg.range_mode = range_mode
         self._h = ctypes.c_void_p()
         _check(lib().thc_create(ctypes.byref(cfg), ctypes.byref(self._h)), "thc_create")
         self.bits, self.granularity, self.log2_block = bits, granularity, log2_block
@@ -173,13 +178,19 @@ class Context:
         s = _Sizes()
         _check(lib().thc_sizes(self._h, d, n_local, ctypes.byref(s)), "thc_sizes")
         return Sizes(s.d_pad, s.nblocks, s.packed_bytes, s.sum_bytes, s.rotated_bytes,
-                     s.workspace_bytes, s.acc_bits, s.fused_scales)
+                     s.workspace_bytes, s.acc_bits, s.fused_scales, s.scales_count)
 
     def prepare(self, grads, d: int, scales, workspace, stream=None):
         arr = _ptr_array([_dp(g) for g in grads])
         _check(lib().thc_prepare(self._h, arr, len(grads), d, _dp(scales), _dp(workspace),
                                  workspace.numel() * workspace.element_size(), _stream(stream)),
                "thc_prepare")
+
+    def prepare_minmax(self, grads, d: int, rnd: int, scales, workspace, stream=None):
+        arr = _ptr_array([_dp(g) for g in grads])
+        _check(lib().thc_prepare_minmax(self._h, arr, len(grads), d, rnd, _dp(scales), _dp(workspace),
+                                        workspace.numel() * workspace.element_size(), _stream(stream)),
+               "thc_prepare_minmax")
 
     def compress(self, grads, d: int, rnd: int, scales, packed, workspace, rotated=None,
                  worker_base: int = 0, stream=None):

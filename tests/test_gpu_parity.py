@@ -383,3 +383,68 @@ def test_error_feedback_other_index_widths(bits, g):
         z = O.unpack(r.packed[i].cpu().numpy(), r.sz.d_pad, w.bits)
         ref = O.error_feedback(x[i], z, scl, c, 5)
         assert np.array_equal(ef[i].cpu().numpy().view(np.uint32), ref.view(np.uint32)), f"worker {i}"
+
+
+@pytest.mark.parametrize("k,d,n", [(5, 1000, 2), (10, 33_001, 3), (16, 150_000, 2), (20, (1 << 21) + 99, 2)])
+def test_exact_range_round_matches_oracle(k, d, n):
+    """THC_RANGE_MINMAX contexts (Algorithm 1's preliminary stage on the rotated coordinates):
+    the (min, max) planes equal the oracle's bit for bit (the rotated coordinates do), and so
+    do the packed indices, the sums, the output and the error feedback computed from them."""
+    import torch
+    from paper_2302_08545_b200 import runner, thc
+    w = _mk(n, d, k)
+    x, _ = _inputs(w)
+    ctx = runner.context_for(w, exact_range=True)
+    r = runner.Round(ctx, n, d)
+    assert r.sz.scales_count == 2 * r.sz.nblocks and r.sz.fused_scales == 0
+    r.upload(x)
+    rnd = 4
+    r.prepare_minmax(rnd)
+    r.compress(rnd)
+    r.aggregate()
+    r.decompress(rnd)
+    ef = [torch.zeros(d, dtype=torch.float32, device=r.device) for _ in range(n)]
+    ctx.error_feedback(r.grads, r.packed, d, rnd, r.scales, ef, r.workspace)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    c = _ocfg(w)
+    lo, hi = O.ranges(x, c, rnd)
+    got = r.scales.cpu().numpy()
+    nb = r.sz.nblocks
+    assert np.array_equal(got[:nb].view(np.uint32), lo.view(np.uint32))
+    assert np.array_equal(got[nb:].view(np.uint32), hi.view(np.uint32))
+    ref = O.thc_round(x, c, rnd, exact_range=True)
+    for i in range(n):
+        assert np.array_equal(r.packed[i].cpu().numpy(), ref["packed"][i]), f"worker {i}"
+    assert np.array_equal(r.sum_numpy(), ref["sum"])
+    assert np.array_equal(r.out.cpu().numpy().view(np.uint32), ref["out"].view(np.uint32))
+    for i in range(n):
+        z = O.unpack(ref["packed"][i], r.sz.d_pad, w.bits)
+        e = O.error_feedback(x[i], z, hi, c, rnd, lo=lo)
+        assert np.array_equal(ef[i].cpu().numpy().view(np.uint32), e.view(np.uint32)), f"worker {i}"
+    # no coordinate was clamped: the extreme indices occur, and only at the extremes
+    with pytest.raises(thc.ThcError):
+        r.prepare()                        # the norm-based call does not apply to this context
+
+
+def test_exact_range_flags_non_finite_blocks():
+    import torch
+    from paper_2302_08545_b200 import runner, thc
+    k, d, n = 16, 3 * (1 << 16), 2
+    w = _mk(n, d, k)
+    x, _ = _inputs(w)
+    x[1, (1 << 16) + 5] = np.inf
+    x[0, 2 * (1 << 16):] = 0.0
+    x[1, 2 * (1 << 16):] = 0.0
+    ctx = runner.context_for(w, exact_range=True)
+    r = runner.Round(ctx, n, d)
+    r.upload(x)
+    r.prepare_minmax(0)
+    r.compress(0); r.aggregate(); r.decompress(0)
+    torch.cuda.synchronize()
+    flags = ctx.status()
+    assert flags & thc.STATUS_NONFINITE and flags & thc.STATUS_ZERO_BLOCK
+    s = r.scales.cpu().numpy()
+    assert s[1] == 0.0 and s[3 + 1] == 0.0 and s[2] == 0.0 and s[3 + 2] == 0.0 and s[3] > s[0]
+    out = r.out.cpu().numpy()
+    assert np.all(out[(1 << 16):] == 0.0) and np.all(np.isfinite(out))
