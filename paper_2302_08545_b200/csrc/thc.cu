@@ -1,13 +1,11 @@
 // libthc: kernels and C ABI.  See include/thc.h for the contract of every entry point.
 //
-// Structure of the transform.  An RHT block of B = 2^k coordinates is handled as one or two
-// passes over 2^14-coordinate tiles held in shared memory:
-//   pass A  a tile is 2^14 consecutive coordinates: load (+ sign flip or de-quantisation),
-//           stages of stride 1 .. 2^13 (or 2^(k-1) if k < 14)
-//   pass B  (only if k > 14) a tile is 2^(k-14) rows, 2^14 coordinates apart, by 2^(28-k)
-//           consecutive columns: the remaining stages of stride 2^14 .. 2^(k-1)
-// The last pass of a block ends in the fused epilogue: scale by 1/sqrt(B), then either
-// truncate + quantise + pack (compress) or sign flip + store (decompress).
+// Structure of the transform.  An RHT block of B = 2^k coordinates with k <= 14 is handled by
+// rht_tile_kernel below: a CTA holds a tile of 2^14 consecutive coordinates (one block or
+// several small ones) in shared memory: load (+ sign flip or de-quantisation), stages of
+// stride 1 .. 2^(k-1), then the fused epilogue: scale by 1/sqrt(B) and either truncate +
+// quantise + pack (compress), sign flip + store (decompress) or min / max (exact range).
+// Larger blocks go through the persistent two-pass pipeline of thc_pipeline.cuh.
 #include "../../include/thc.h"
 #include "thc_device.cuh"
 
@@ -21,8 +19,8 @@ namespace thc {
 struct PtrArray { const void *p[THC_MAX_WORKERS]; };
 struct MutPtrArray { void *p[THC_MAX_WORKERS]; };
 
-enum LoadKind { kLoadGradF32, kLoadGradBF16, kLoadSum8, kLoadSum16, kLoadSum32, kLoadRaw };
-enum StoreKind { kStoreRaw, kStoreQuant, kStoreOut, kStoreRange };
+enum LoadKind { kLoadGradF32, kLoadGradBF16, kLoadSum8, kLoadSum16, kLoadSum32 };
+enum StoreKind { kStoreQuant, kStoreOut, kStoreRange };
 
 // Geometry of the tiles one launch walks.
 struct TileGeom {
@@ -225,14 +223,6 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
                 tile[swz(u * (kPer / 4) + cc)] = stages01(make_float4(s[0], s[1], s[2], s[3]));
             }
         }
-    } else {   // kLoadRaw: second pass, rows 2^14 apart
-        const float *x = static_cast<const float *>(in.p[0]) + (uint64_t)wl * g.d_pad;
-#pragma unroll 4
-        for (int i = 0; i < kTileChunks / kThreads; ++i) {
-            const int c = tid + i * kThreads;
-            const uint64_t j = chunk_coord(g, base, c);
-            tile[swz(c)] = *reinterpret_cast<const float4 *>(x + j);
-        }
     }
     __syncthreads();
 
@@ -240,15 +230,7 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
     fwht_rounds(tile, (int)g.lo_cbit, (int)g.hi_cbit, tid);
 
     // ---- store phase
-    if (STORE == kStoreRaw) {
-        float *ws = static_cast<float *>(out.p[0]) + (uint64_t)wl * g.d_pad;
-#pragma unroll 4
-        for (int i = 0; i < kTileChunks / kThreads; ++i) {
-            const int c = tid + i * kThreads;
-            const uint64_t j = chunk_coord(g, base, c);
-            if (j < g.d_pad) *reinterpret_cast<float4 *>(ws + j) = tile[swz(c)];
-        }
-    } else if (STORE == kStoreQuant) {
+    if (STORE == kStoreQuant) {
         unsigned char *pk = static_cast<unsigned char *>(out.p[wl]);
         float *rot = static_cast<float *>(rotated.p[wl]);
         const float gf = (float)g.granularity;
@@ -1192,11 +1174,10 @@ int thc_compress(thc_ctx *ctx, const void *const *grads, uint32_t n_local, uint3
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     PtrArray in;
-    MutPtrArray out, rot, ws;
+    MutPtrArray out, rot;
     memset(&in, 0, sizeof in);
     memset(&out, 0, sizeof out);
     memset(&rot, 0, sizeof rot);
-    memset(&ws, 0, sizeof ws);
     for (uint32_t i = 0; i < n_local; ++i) {
         in.p[i] = grads[i];
         out.p[i] = packed[i];
@@ -1205,7 +1186,6 @@ int thc_compress(thc_ctx *ctx, const void *const *grads, uint32_t n_local, uint3
             rot.p[i] = rotated[i];
         }
     }
-    ws.p[0] = workspace;
     TileGeom g = base_geom(ctx, sz, d, round);
     g.worker_base = worker_base;
     const bool bf16 = ctx->cfg.in_dtype == THC_BF16;
@@ -1285,14 +1265,12 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     PtrArray in;
-    MutPtrArray out, rot, ws;
+    MutPtrArray out, rot;
     memset(&in, 0, sizeof in);
     memset(&out, 0, sizeof out);
     memset(&rot, 0, sizeof rot);
-    memset(&ws, 0, sizeof ws);
     in.p[0] = sum;
     out.p[0] = outp;
-    ws.p[0] = workspace;
     TileGeom g = base_geom(ctx, sz, d, round);
     g.divisor = divisor;
     const uint64_t tiles = (sz.d_pad + kTileElems - 1) / kTileElems;
