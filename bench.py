@@ -440,12 +440,41 @@ def run_sweep(args):
     return 0
 
 
+def sweep_table(path: str) -> int:
+    """Markdown tables (one per index width) from the JSON lines `--sweep` printed."""
+    rows = [json.loads(l) for l in open(path) if l.startswith("{")]
+    pts = [r for r in rows if "workload" in r]
+    summ = [r for r in rows if "sweep_points" in r]
+    for bits in sorted({r["bits"] for r in pts}):
+        sel = [r for r in pts if r["bits"] == bits]
+        ns = sorted({r["n"] for r in sel})
+        print(f"## b = {bits}\n")
+        print("| d \\ n | " + " | ".join(str(n) for n in ns) + " |")
+        print("|---|" + "---|" * len(ns))
+        for d in sorted({r["d"] for r in sel}):
+            cells = []
+            for n in ns:
+                m = [r for r in sel if r["d"] == d and r["n"] == n]
+                cells.append(f"{m[0]['round_ms']:.3f} / {100 * m[0]['frac_of_measured_hbm']:.1f} %" if m else "")
+            print(f"| 2^{d.bit_length() - 1} | " + " | ".join(cells) + " |")
+        print()
+    if summ:
+        s0 = summ[-1]
+        print(f"Over the {s0['sweep_points']} points: fraction min {100 * s0['frac_min']:.1f} %, "
+              f"median {100 * s0['frac_median']:.1f} %, max {100 * s0['frac_max']:.1f} %.")
+    flagged = [r["workload"] for r in pts if r.get("status_flags")]
+    print("Status flags set at: " + (", ".join(flagged) if flagged else "no point") + ".")
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="thc", choices=["thc", "reference"])
+    ap.add_argument("--sweep-table", default=None, metavar="JSONL",
+                    help="print markdown tables from the output of an earlier --sweep run (no GPU)")
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="run the d x b x n sweep (configuration 5)")
@@ -453,6 +482,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.sweep_table:
+        return sweep_table(args.sweep_table)
     if args.sweep:
         return run_sweep(args)
     return run_gpu(args)
