@@ -41,6 +41,11 @@ KERNELS_PER_STEP = {"prepare": 2, "compress": 1, "prepare_compress": 1, "aggrega
 # so a full launch is this times n*d_pad.
 NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.293}
 NCU_FUSED_DRAM_BYTES_PER_COORD = {("f32", 4): 6.213}
+# Executed thread-instructions per (worker, padded coordinate) from the same captures
+# (smsp__inst_executed x 32 / coordinates): the kernel is bound by instruction issue and the
+# shared-memory pipe rather than by HBM, so the issue rate is reported beside the HBM fraction.
+NCU_COMPRESS_THREAD_INST_PER_COORD = {("f32", 4): 47.7}
+NCU_FUSED_THREAD_INST_PER_COORD = {("f32", 4): 50.9}
 
 
 def pick_workload(name: str) -> W.Workload:
@@ -350,12 +355,23 @@ def run_gpu(args):
     per_coord = (NCU_FUSED_DRAM_BYTES_PER_COORD if fused else NCU_COMPRESS_DRAM_BYTES_PER_COORD).get(
         (w.in_dtype, w.bits))
     traffic = None if per_coord is None or w.log2_block < 15 else per_coord * w.n * w.d_pad
+    clk = clocks.summary()
+    inst = (NCU_FUSED_THREAD_INST_PER_COORD if fused else NCU_COMPRESS_THREAD_INST_PER_COORD).get(
+        (w.in_dtype, w.bits))
+    issue = None
+    if inst is not None and w.log2_block >= 15 and clk.get("sm_mhz"):
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        lane_peak = sms * 128 * clk["sm_mhz"] * 1e6
+        lane_rate = inst * w.n * w.d_pad / (comp_ms * 1e-3)
+        issue = {"thread_inst_per_coord": inst, "achieved_lane_inst_per_s": lane_rate,
+                 "peak_lane_inst_per_s": lane_peak, "frac": lane_rate / lane_peak,
+                 "source": "ncu smsp__inst_executed on the d=2^24 n=4 b=4 sweep point; peak = SMs x 128 lanes x sampled SM clock"}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": workload_config(w),
-        "clocks": clocks.summary(),
+        "clocks": clk,
         "e2e": {"value": world * grad_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": w.d * 4,
                 "ms_per_step": e2e_ms, "steps": e2e_steps},
@@ -366,7 +382,7 @@ def run_gpu(args):
                      "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": ab["compress"], "ms_per_launch": comp_ms,
-                     "traffic": traffic,
+                     "traffic": traffic, "issue": issue,
                      "traffic_source": "ncu dram bytes on the d=2^24 n=4 b=4 sweep point, scaled by n*d_pad"
                                        if traffic is not None else None},
         "per_call_ms": per_call_ms,
