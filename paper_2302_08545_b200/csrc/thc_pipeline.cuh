@@ -774,20 +774,26 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
         pend[1] = pend[0];
 
         // Warp-wide: publish the completion of task t (whose sums of squares sit in s_sq[sq]).
-        // Fused scales: the warp that counts the last tile of an RHT block computes the block's
-        // M from the stored sums (fixed order) and releases the block's pass-B tasks.
-        auto complete = [&](const TaskId &t, int sq) {
+        // Fused scales: a pass-A tile is counted with a returning atomic; complete_issue only
+        // issues it (lane 0 keeps the result, which nothing needs yet, so the claim of the next
+        // task can be in flight at the same time) and complete_finish looks at it: the warp
+        // that counted the last tile of an RHT block computes the block's M from the stored
+        // sums (fixed order) and releases the block's pass-B tasks.
+        auto complete_issue = [&](const TaskId &t, int sq, uint32_t &old, uint32_t &r) -> bool {
             if (!kFused || t.is_b) {
                 if (lane == 0) red_release_add(t.is_b ? &pc->b_done[t.slot].v : &pc->a_done[t.slot].v, 1u);
-                return;
+                return false;
             }
-            const uint32_t r = t.wb / P.n_local;
-            uint32_t old = 0;
+            r = t.wb / P.n_local;
+            old = 0;
             if (lane == 0) {
                 const double tile_sum = (s_sq[sq][0] + s_sq[sq][1]) + (s_sq[sq][2] + s_sq[sq][3]);
                 __stcg(P.tile_sq + (((size_t)t.wb << kb) + t.idx), tile_sum);
                 old = atom_release_add(&pc->a_done[r & 15u].v, 1u);
             }
+            return true;
+        };
+        auto complete_finish = [&](uint32_t old, uint32_t r) {
             old = __shfl_sync(0xFFFFFFFFu, old, 0);
             if (old + 1u != (r / 16u + 1u) * P.n_local * T) return;
             __threadfence();                           // the other tiles' sums, after seeing the count
@@ -825,6 +831,10 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 red_release_add(&pc->a_done[16u + (r & 15u)].v, 1u);
             }
         };
+        auto complete = [&](const TaskId &t, int sq) {
+            uint32_t old = 0, r = 0;
+            if (complete_issue(t, sq, old, r)) complete_finish(old, r);
+        };
 
         for (uint32_t i = 0;; ++i) {
             const int s = (int)(i & 1);
@@ -833,9 +843,11 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
             // look-ahead only: a deeper one stretches every task's claim-to-completion time,
             // which is what dependent tasks wait for.  Task i-2 is signalled first: task i
             // may depend on it.
+            bool counting = false;
+            uint32_t cnt_old = 0, cnt_r = 0;
             if (i >= 1) {
                 bar_sync(3 + (s ^ 1), kPCtaThreads);
-                if (pend_valid[s]) { complete(pend[s], s); pend_valid[s] = false; }
+                if (pend_valid[s]) { counting = complete_issue(pend[s], s, cnt_old, cnt_r); pend_valid[s] = false; }
             }
             uint32_t q = 0, ab = 0;
             if (lane == 0) {
@@ -844,6 +856,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
             }
             q = __shfl_sync(0xFFFFFFFFu, q, 0);
             ab = __shfl_sync(0xFFFFFFFFu, ab, 0);
+            if (counting) complete_finish(cnt_old, cnt_r);
             bool have = (uint64_t)q < P.total_tasks && ab == 0;
             TaskId t;
             t.wb = t.idx = t.is_b = t.slot = t.gen = 0;
