@@ -292,7 +292,7 @@ def test_error_feedback_matches_oracle(k, d, n):
         assert np.array_equal(r.grads[i].cpu().numpy(), x[i] + ef[i].cpu().numpy())
 
 
-@pytest.mark.parametrize("n,nblk,tail", [(2, 14, 12_345), (3, 9, 0), (8, 6, 77)])
+@pytest.mark.parametrize("n,nblk,tail", [(1, 13, 5), (2, 14, 12_345), (3, 9, 0), (8, 6, 77), (13, 2, 4096)])
 def test_prepare_compress_fused_equals_the_two_calls(n, nblk, tail):
     """thc_prepare_compress (block norms summed inside the transform kernel, Section 5.3's
     overlap of the norm exchange with the RHT): its scales agree with thc_prepare's (fp64 sums
@@ -346,7 +346,7 @@ def test_prepare_compress_falls_back_where_the_fused_kernel_does_not_apply():
     inside the same entry point: results identical to calling them."""
     import torch
     from paper_2302_08545_b200 import runner
-    for k, d, n in [(16, 300_000, 3), (20, (1 << 20) + 5, 2)]:
+    for k, d, n in [(16, 300_000, 3), (20, (1 << 20) + 5, 2), (20, 2 * (1 << 20), 14)]:
         w = _mk(n, d, k)
         x, _ = _inputs(w)
         ctx = runner.context_for(w)
