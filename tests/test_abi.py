@@ -45,6 +45,7 @@ def test_sizes_match_the_paper_prototype_ratios():
     dict(table=T4_30[:-1] + (29,)), dict(table=(0, 3, 3) + T4_30[3:]), dict(t_p=0.0),
     dict(t_p=float("nan")), dict(log2_block=2), dict(log2_block=23), dict(in_dtype=7),
     dict(workers=0), dict(workers=65), dict(acc_bits=12), dict(workers=9, acc_bits=8),
+    dict(range_mode=2),
 ])
 def test_invalid_configurations_are_rejected(kw):
     with pytest.raises(thc.ThcError) as e:
@@ -55,6 +56,21 @@ def test_invalid_configurations_are_rejected(kw):
 def test_unsupported_granularity():
     with pytest.raises(thc.ThcError) as e:
         _ctx(bits=8, granularity=300, table=tuple(range(255)) + (300,))
+    assert e.value.code == thc.THC_EUNSUPPORTED
+
+
+def test_range_mode_sizes_and_limits():
+    """Exact-range contexts keep two floats per RHT block (minima, then maxima), never take
+    the fused scales path, and accept fp32 input only."""
+    c = _ctx(range_mode=1)
+    s = c.sizes(25_557_032, 8)
+    assert s.scales_count == 2 * s.nblocks and s.fused_scales == 0
+    n = _ctx().sizes(25_557_032, 8)
+    assert n.scales_count == n.nblocks and n.fused_scales == 1
+    assert _ctx().sizes(25_557_032, 14).fused_scales == 0        # ring would not fit in L2
+    assert _ctx(log2_block=16).sizes(25_557_032, 8).fused_scales == 0
+    with pytest.raises(thc.ThcError) as e:
+        _ctx(range_mode=1, in_dtype=thc.THC_BF16)
     assert e.value.code == thc.THC_EUNSUPPORTED
 
 
