@@ -448,3 +448,79 @@ def test_exact_range_flags_non_finite_blocks():
     assert s[1] == 0.0 and s[3 + 1] == 0.0 and s[2] == 0.0 and s[3 + 2] == 0.0 and s[3] > s[0]
     out = r.out.cpu().numpy()
     assert np.all(out[(1 << 16):] == 0.0) and np.all(np.isfinite(out))
+
+
+def test_error_feedback_loop_on_the_gpu_telescopes_and_matches_the_oracle():
+    """Algorithm 3's worker loop over several rounds, all on the GPU: x = grad + e,
+    compress, e = x - RHT^-1(X).  Every round's residual equals the oracle's run of the same
+    loop bit for bit, and what was sent telescopes: sum_r RHT^-1(X^r) = R grad - e^R
+    (up to fp32 rounding of the additions)."""
+    import torch
+    from paper_2302_08545_b200 import runner
+    k, d, n, R = 16, 100_000, 2, 4
+    w = _mk(n, d, k, t_p=0.9)                            # a tight clamp: large residuals
+    g, _ = _inputs(w)
+    ctx = runner.context_for(w)
+    r = runner.Round(ctx, n, d)
+    c = _ocfg(w)
+    ef = [torch.zeros(d, dtype=torch.float32, device=r.device) for _ in range(n)]
+    e_ref = np.zeros((n, d), np.float32)
+    sent = np.zeros((n, d), np.float64)
+    for rnd in range(R):
+        r.upload(g)
+        ctx.accumulate_error(r.grads, ef, d)             # x = grad + e
+        r.prepare()
+        r.compress(rnd)
+        ctx.error_feedback(r.grads, r.packed, d, rnd, r.scales, ef, r.workspace)
+        torch.cuda.synchronize()
+        x_ref = g + e_ref                                # one fp32 addition, as on the GPU
+        scl = r.scales.cpu().numpy()
+        for i in range(n):
+            assert np.array_equal(r.grads[i].cpu().numpy(), x_ref[i])
+            z = O.unpack(r.packed[i].cpu().numpy(), r.sz.d_pad, w.bits)
+            e_new = O.error_feedback(x_ref[i], z, scl, c, rnd)
+            assert np.array_equal(ef[i].cpu().numpy().view(np.uint32), e_new.view(np.uint32)), (rnd, i)
+            sent[i] += x_ref[i].astype(np.float64) - e_new.astype(np.float64)
+            e_ref[i] = e_new
+    assert ctx.status() == 0
+    resid = sent - (R * g.astype(np.float64) - e_ref.astype(np.float64))
+    assert np.abs(resid).max() <= 1e-5 * np.abs(g).max() * R
+
+
+def test_step_can_be_captured_in_a_cuda_graph_and_replayed():
+    """The hot calls only enqueue work on the given stream: after one eager step (which sets
+    kernel attributes) the whole step is captured into a CUDA graph; replays on new inputs
+    give the same bits as eager calls."""
+    import torch
+    from paper_2302_08545_b200 import runner
+    for k, d, n in [(16, 65_536 * 3, 4), (20, 14 * (1 << 20) + 17, 2)]:
+        w = _mk(n, d, k)
+        x, _ = _inputs(w)
+        ctx = runner.context_for(w)
+        r = runner.Round(ctx, n, d)
+        r.upload(x)
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            r.run(3, fused=True)                         # eager, on the capture stream
+        side.synchronize()
+        expect_packed = [p.clone() for p in r.packed]
+        expect_out = r.out.clone()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            r.run(3, fused=True)
+        for p in r.packed:
+            p.zero_()
+        r.out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for a, b in zip(r.packed, expect_packed):
+            assert torch.equal(a, b)
+        assert torch.equal(r.out, expect_out)
+        r.upload(x[::-1].copy())                         # other inputs, same graph
+        graph.replay()
+        torch.cuda.synchronize()
+        got_out = r.out.clone()
+        r.run(3, fused=True)
+        torch.cuda.synchronize()
+        assert torch.equal(got_out, r.out)
+        assert ctx.status() == 0
