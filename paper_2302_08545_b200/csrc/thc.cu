@@ -371,6 +371,142 @@ aggregate_b4w8_kernel(PtrArray in, uint32_t n, uint64_t units16, const DeviceBlo
     }
 }
 
+// The same with 16-bit sums (more workers than fit a byte: workers * g > 255).  Table values are
+// summed in byte lanes for CHUNK workers at a time (CHUNK * g <= 255), then widened into
+// 16-bit lanes (even and odd coordinates apart) and put back in order at the end.
+template <int CHUNK>
+__global__ void __launch_bounds__(kThreads)
+aggregate_b4w16_kernel(PtrArray in, uint32_t n, uint64_t units16, const DeviceBlock *dev,
+                       uint4 *__restrict__ sum)
+{
+    uint32_t t[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        t[q] = dev->table[4 * q] | (dev->table[4 * q + 1] << 8) | (dev->table[4 * q + 2] << 16) |
+               (dev->table[4 * q + 3] << 24);
+    for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < units16;
+         u += (uint64_t)gridDim.x * kThreads) {
+        uint32_t even[4] = {0u, 0u, 0u, 0u}, odd[4] = {0u, 0u, 0u, 0u};
+#pragma unroll 1
+        for (uint32_t i0 = 0; i0 < n; i0 += CHUNK) {
+            uint2 w[CHUNK];
+#pragma unroll
+            for (int j = 0; j < CHUNK; ++j)
+                w[j] = i0 + j < n ? __ldg(reinterpret_cast<const uint2 *>(in.p[i0 + j]) + u) : make_uint2(0u, 0u);
+            uint32_t acc[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int j = 0; j < CHUNK; ++j) {
+                const uint32_t words[2] = {w[j].x, w[j].y};   // index 0 everywhere adds T[0] = 0
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t a = words[h], b = a ^ 0x88888888u;
+                    acc[2 * h] += prmt(t[0], t[1], a) + prmt(t[2], t[3], b);
+                    acc[2 * h + 1] += prmt(t[0], t[1], a >> 16) + prmt(t[2], t[3], b >> 16);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                even[q] += acc[q] & 0x00FF00FFu;
+                odd[q] += (acc[q] >> 8) & 0x00FF00FFu;
+            }
+        }
+        uint32_t o[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            o[2 * q] = prmt(even[q], odd[q], 0x5410u);          // coordinates 4q, 4q+1
+            o[2 * q + 1] = prmt(even[q], odd[q], 0x7632u);      // coordinates 4q+2, 4q+3
+        }
+        sum[2 * u] = make_uint4(o[0], o[1], o[2], o[3]);
+        sum[2 * u + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
+// 1- and 2-bit indices with 8-bit sums: T[z] = g z for one bit, the identity table for two, so
+// the sum of table values is g times the sum of the indices.  Index fields are spread into
+// byte lanes by shift and mask (lane j of the k-th spread holds coordinate (8/BITS) j + k), added
+// across workers, and transposed into coordinate order at the end.  A thread handles 32
+// coordinates.
+template <int BITS>
+__global__ void __launch_bounds__(kThreads)
+aggregate_small_w8_kernel(PtrArray in, uint32_t n, uint64_t units32, uint32_t g_mult,
+                          uint4 *__restrict__ sum)
+{
+    constexpr int kWords = BITS;                       // 32 coordinates = BITS words
+    constexpr int kSpread = 8 / BITS;                  // spreads per word
+    constexpr uint32_t kMask = BITS == 1 ? 0x01010101u : 0x03030303u;
+    for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < units32;
+         u += (uint64_t)gridDim.x * kThreads) {
+        uint32_t acc[kWords][kSpread];
+#pragma unroll
+        for (int q = 0; q < kWords; ++q)
+#pragma unroll
+            for (int k = 0; k < kSpread; ++k) acc[q][k] = 0u;
+#pragma unroll 4
+        for (uint32_t i = 0; i < n; ++i) {
+            uint32_t words[kWords];
+            if constexpr (BITS == 1) {
+                words[0] = __ldg(reinterpret_cast<const uint32_t *>(in.p[i]) + u);
+            } else {
+                const uint2 w = __ldg(reinterpret_cast<const uint2 *>(in.p[i]) + u);
+                words[0] = w.x; words[1] = w.y;
+            }
+#pragma unroll
+            for (int q = 0; q < kWords; ++q)
+#pragma unroll
+                for (int k = 0; k < kSpread; ++k) acc[q][k] += (words[q] >> (k * BITS)) & kMask;
+        }
+        // byte j of acc[q][k] is coordinate (32/BITS) q + kSpread j + k: gather four consecutive
+        // coordinates into each output word
+        uint32_t o[8];
+#pragma unroll
+        for (int q = 0; q < kWords; ++q) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+#pragma unroll
+                for (int h = 0; h < kSpread / 4; ++h) {
+                    const uint32_t *a = &acc[q][4 * h];
+                    const uint32_t sel = (uint32_t)j | ((uint32_t)(4 + j) << 4);
+                    const uint32_t p01 = prmt(a[0], a[1], sel);            // bytes: a0[j], a1[j]
+                    const uint32_t p23 = prmt(a[2], a[3], sel);            // bytes: a2[j], a3[j]
+                    const uint32_t word = prmt(p01, p23, 0x5410u);         // a0[j], a1[j], a2[j], a3[j]
+                    o[(q * (32 / BITS) + kSpread * j + 4 * h) / 4] = word * g_mult;
+                }
+            }
+        }
+        sum[2 * u] = make_uint4(o[0], o[1], o[2], o[3]);
+        sum[2 * u + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
+// 8-bit indices with the identity table (g = 255) and 16-bit sums: bytes are widened into
+// 16-bit lanes (even and odd coordinates apart).  A thread handles 16 coordinates.
+__global__ void __launch_bounds__(kThreads)
+aggregate_b8w16_kernel(PtrArray in, uint32_t n, uint64_t units16, uint4 *__restrict__ sum)
+{
+    for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < units16;
+         u += (uint64_t)gridDim.x * kThreads) {
+        uint32_t even[4] = {0u, 0u, 0u, 0u}, odd[4] = {0u, 0u, 0u, 0u};
+#pragma unroll 4
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint4 w = __ldg(reinterpret_cast<const uint4 *>(in.p[i]) + u);
+            const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                even[q] += words[q] & 0x00FF00FFu;
+                odd[q] += (words[q] >> 8) & 0x00FF00FFu;
+            }
+        }
+        uint32_t o[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            o[2 * q] = prmt(even[q], odd[q], 0x5410u);
+            o[2 * q + 1] = prmt(even[q], odd[q], 0x7632u);
+        }
+        sum[2 * u] = make_uint4(o[0], o[1], o[2], o[3]);
+        sum[2 * u + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
 // ------------------------------------------------------------------------ error feedback
 // e <- x - e (e holds RHT^-1(X) on entry) and x <- x + e, 128-bit accesses with a scalar tail.
 __global__ void __launch_bounds__(kThreads)
@@ -1359,6 +1495,39 @@ int thc_aggregate(thc_ctx *ctx, const void *const *packed, uint32_t n, uint64_t 
         if (nb > cap16) nb = cap16;
         aggregate_b4w8_kernel<<<(unsigned)nb, kThreads, 0, st>>>(in, n, units16, ctx->dev,
                                                                   reinterpret_cast<uint4 *>(s));
+        THC_CUDA(cudaGetLastError());
+        return THC_OK;
+    }
+    const uint32_t bits = ctx->cfg.bits, g = ctx->cfg.granularity, w = ctx->acc_bits;
+    if (bits == 4 && w == 16 && g < 128 && sz.d_pad % 16 == 0) {
+        const uint64_t units16 = sz.d_pad / 16;
+        uint64_t nb = (units16 + kThreads - 1) / kThreads;
+        if (nb > (uint64_t)ctx->sm_count * 8) nb = (uint64_t)ctx->sm_count * 8;
+        uint4 *s4 = reinterpret_cast<uint4 *>(s);
+        if (g <= 31) aggregate_b4w16_kernel<8><<<(unsigned)nb, kThreads, 0, st>>>(in, n, units16, ctx->dev, s4);
+        else if (g <= 63) aggregate_b4w16_kernel<4><<<(unsigned)nb, kThreads, 0, st>>>(in, n, units16, ctx->dev, s4);
+        else aggregate_b4w16_kernel<2><<<(unsigned)nb, kThreads, 0, st>>>(in, n, units16, ctx->dev, s4);
+        THC_CUDA(cudaGetLastError());
+        return THC_OK;
+    }
+    if ((bits == 1 || (bits == 2 && ctx->identity)) && w == 8 && sz.d_pad % 32 == 0) {
+        const uint64_t units32 = sz.d_pad / 32;
+        uint64_t nb = (units32 + kThreads - 1) / kThreads;
+        if (nb > (uint64_t)ctx->sm_count * 8) nb = (uint64_t)ctx->sm_count * 8;
+        if (bits == 1)
+            aggregate_small_w8_kernel<1><<<(unsigned)nb, kThreads, 0, st>>>(in, n, units32, g,
+                                                                            reinterpret_cast<uint4 *>(s));
+        else
+            aggregate_small_w8_kernel<2><<<(unsigned)nb, kThreads, 0, st>>>(in, n, units32, 1u,
+                                                                            reinterpret_cast<uint4 *>(s));
+        THC_CUDA(cudaGetLastError());
+        return THC_OK;
+    }
+    if (bits == 8 && ctx->identity && w == 16 && sz.d_pad % 16 == 0) {
+        const uint64_t units16 = sz.d_pad / 16;
+        uint64_t nb = (units16 + kThreads - 1) / kThreads;
+        if (nb > (uint64_t)ctx->sm_count * 8) nb = (uint64_t)ctx->sm_count * 8;
+        aggregate_b8w16_kernel<<<(unsigned)nb, kThreads, 0, st>>>(in, n, units16, reinterpret_cast<uint4 *>(s));
         THC_CUDA(cudaGetLastError());
         return THC_OK;
     }

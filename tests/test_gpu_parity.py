@@ -524,3 +524,32 @@ def test_step_can_be_captured_in_a_cuda_graph_and_replayed():
         torch.cuda.synchronize()
         assert torch.equal(got_out, r.out)
         assert ctx.status() == 0
+
+
+@pytest.mark.parametrize("bits,g,table,n", [
+    (1, 1, (0, 1), 5), (1, 200, (0, 200), 1), (1, 3, (0, 3), 64), (2, 3, (0, 1, 2, 3), 64),
+    (4, 30, T4_30, 17), (4, 30, T4_30, 64), (4, 15, tuple(range(16)), 64), (4, 127, tuple(range(15)) + (127,), 3),
+    (8, 255, tuple(range(256)), 7), (8, 255, tuple(range(256)), 64),
+])
+def test_aggregate_fast_paths_on_random_indices(bits, g, table, n):
+    """The byte-lane (SWAR) aggregation kernels against the oracle's plain loop on uniformly
+    random packed indices: every index value, every lane, chunk boundaries of the 16-bit
+    widening, and a ragged number of thread units."""
+    import torch
+    from paper_2302_08545_b200 import runner
+    k = 7
+    d = 128 * 1237                                        # not a multiple of the grid stride
+    w = _mk(n, d, k, bits=bits, g=g, table=table)
+    ctx = runner.context_for(w)
+    sz = ctx.sizes(d, n)
+    rng = np.random.default_rng(1000 * bits + n)
+    packed = rng.integers(0, 256, size=(n, sz.packed_bytes), dtype=np.uint8)
+    dev = torch.device("cuda", 0)
+    bufs = [torch.from_numpy(packed[i]).to(dev) for i in range(n)]
+    total = torch.zeros(sz.sum_bytes, dtype=torch.uint8, device=dev)
+    ctx.aggregate(bufs, d, total)
+    torch.cuda.synchronize()
+    c = _ocfg(w)
+    ref = O.aggregate(packed, sz.d_pad, c, sz.acc_bits)
+    dt = {8: np.uint8, 16: np.uint16, 32: np.uint32}[sz.acc_bits]
+    assert np.array_equal(total.cpu().numpy().view(dt), ref)
