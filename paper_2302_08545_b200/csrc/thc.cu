@@ -356,21 +356,15 @@ aggregate_b4w8_kernel(PtrArray in, uint32_t n, uint64_t units16, const DeviceBlo
     for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < units16;
          u += (uint64_t)gridDim.x * kThreads) {
         uint32_t acc[4] = {0u, 0u, 0u, 0u};                  // 16 sums of 8 bits
-#pragma unroll 1
-        for (uint32_t i0 = 0; i0 < n; i0 += 8) {              // eight workers' loads in flight
-            uint2 w[8];
+#pragma unroll 4
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint2 w = __ldg(reinterpret_cast<const uint2 *>(in.p[i]) + u);   // 16 indices
+            const uint32_t words[2] = {w.x, w.y};
 #pragma unroll
-            for (int j = 0; j < 8; ++j)                       // index 0 everywhere adds T[0] = 0
-                w[j] = i0 + j < n ? __ldg(reinterpret_cast<const uint2 *>(in.p[i0 + j]) + u) : make_uint2(0u, 0u);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint32_t words[2] = {w[j].x, w[j].y};
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint32_t a = words[h], b = a ^ 0x88888888u;
-                    acc[2 * h] += prmt(t[0], t[1], a) + prmt(t[2], t[3], b);
-                    acc[2 * h + 1] += prmt(t[0], t[1], a >> 16) + prmt(t[2], t[3], b >> 16);
-                }
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t a = words[h], b = a ^ 0x88888888u;
+                acc[2 * h] += prmt(t[0], t[1], a) + prmt(t[2], t[3], b);
+                acc[2 * h + 1] += prmt(t[0], t[1], a >> 16) + prmt(t[2], t[3], b >> 16);
             }
         }
         sum[u] = make_uint4(acc[0], acc[1], acc[2], acc[3]);
