@@ -1152,19 +1152,21 @@ static encode_tiled_t get_encode_tiled()
     return fn;
 }
 
-// A 2-D map over `rows` rows of `cols` 32-bit words (row pitch in bytes), box 32 x box_rows,
-// 128-byte swizzle.  The data type is UINT32 so that bits travel unchanged.
+// A 2-D map over `rows` rows of `cols` 32-bit words (row pitch in bytes), box box_cols x
+// box_rows (32 columns with the 128-byte swizzle, 16 with the 64-byte one).  The data type is
+// UINT32 so that bits travel unchanged.
 static int encode_map(CUtensorMap *map, const void *base, uint64_t cols, uint64_t rows,
-                      uint64_t pitch_bytes, uint32_t box_rows)
+                      uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols = 32u)
 {
     encode_tiled_t enc = get_encode_tiled();
     if (enc == nullptr) return THC_ECUDA;
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {pitch_bytes};
-    const cuuint32_t box[2] = {32u, box_rows};
+    const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1u, 1u};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(base), dims, strides,
-                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           box_cols == 16u ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? THC_OK : THC_ECUDA;
 }
@@ -1218,10 +1220,23 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
     // loaded by the compute warps).
     TmaMaps maps;
     memset(&maps, 0, sizeof maps);
+    P.b_swz_mask = 7u;
     if (k == 20) {
         const int rc = encode_map(&maps.ring, workspace, (uint64_t)kPElems,
                                   (uint64_t)pl.ring << (k - kPLog2), (uint64_t)kPElems * 4, 128u);
         if (rc != THC_OK) return rc;
+    } else if (k == 22) {
+        // panels of 512 rows x 16 columns: boxes of 16 x 256, 64-byte swizzle
+        const int rc = encode_map(&maps.ring, workspace, (uint64_t)kPElems,
+                                  (uint64_t)pl.ring << (k - kPLog2), (uint64_t)kPElems * 4, 256u, 16u);
+        if (rc != THC_OK) return rc;
+        P.b_swz_mask = 3u;
+        P.b_tma = 2u;
+    } else if (k == 21) {
+        const int rc = encode_map(&maps.ring, workspace, (uint64_t)kPElems,
+                                  (uint64_t)pl.ring << (k - kPLog2), (uint64_t)kPElems * 4, 256u);
+        if (rc != THC_OK) return rc;
+        P.b_tma = 1u;
     }
     if (compress_f32 && (d >> 5) >= 256) {
         for (uint32_t i = 0; i < n_local; ++i) {

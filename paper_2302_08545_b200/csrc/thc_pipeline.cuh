@@ -95,6 +95,9 @@ struct PipeParams {
     uint32_t exact_range;      // scales = nblocks minima then nblocks maxima (else M per block)
     uint32_t nblocks;
     uint32_t *range_keys;      // range mode: nblocks min keys then nblocks max keys
+    uint32_t b_swz_mask;       // run-time geometry, pass-B tiles: chunk c sits at c ^ ((c >> 3) & mask)
+    uint32_t b_tma;            // ... and are fetched by TMA in this many boxes of 256 rows (k = 21: one;
+                               // k = 22: two, 64-byte rows with the 64-byte swizzle); 0: by the compute warps
 };
 
 struct PtrArrayP { const void *p[THC_MAX_WORKERS]; };
@@ -341,7 +344,7 @@ __device__ __forceinline__ float2 block_constants(BlockRange b, uint32_t g, uint
 // ------------------------------------------------------------------ in-place tile rounds
 // Butterfly stages on chunk-index bits [sp, sp+E) of a 2048-chunk tile (see fwht_round).
 template <int E>
-__device__ __forceinline__ void p_round(float4 *tile, int sp, int tid)
+__device__ __forceinline__ void p_round(float4 *tile, int sp, int tid, int mask)
 {
     constexpr int N = 1 << E;
     constexpr int kGroups = kPChunks >> E;
@@ -351,7 +354,7 @@ __device__ __forceinline__ void p_round(float4 *tile, int sp, int tid)
         const int base = ((G >> sp) << (sp + E)) | low;
         float4 v[N];
 #pragma unroll
-        for (int m = 0; m < N; ++m) v[m] = tile[pswz(base + (m << sp))];
+        for (int m = 0; m < N; ++m) { const int c = base + (m << sp); v[m] = tile[c ^ ((c >> 3) & mask)]; }
 #pragma unroll
         for (int t = 0; t < E; ++t) {
 #pragma unroll
@@ -359,20 +362,20 @@ __device__ __forceinline__ void p_round(float4 *tile, int sp, int tid)
                 if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
         }
 #pragma unroll
-        for (int m = 0; m < N; ++m) tile[pswz(base + (m << sp))] = v[m];
+        for (int m = 0; m < N; ++m) { const int c = base + (m << sp); tile[c ^ ((c >> 3) & mask)] = v[m]; }
     }
 }
 
-__device__ __forceinline__ void p_rounds(float4 *tile, int lo, int hi, int tid)
+__device__ __forceinline__ void p_rounds(float4 *tile, int lo, int hi, int tid, int mask)
 {
     int sp = lo;
     while (sp < hi) {
         const int e = min(4, hi - sp);
         switch (e) {
-        case 4: p_round<4>(tile, sp, tid); break;
-        case 3: p_round<3>(tile, sp, tid); break;
-        case 2: p_round<2>(tile, sp, tid); break;
-        default: p_round<1>(tile, sp, tid); break;
+        case 4: p_round<4>(tile, sp, tid, mask); break;
+        case 3: p_round<3>(tile, sp, tid, mask); break;
+        case 2: p_round<2>(tile, sp, tid, mask); break;
+        default: p_round<1>(tile, sp, tid, mask); break;
         }
         sp += e;
         compute_barrier();
@@ -618,7 +621,7 @@ __device__ __forceinline__ void epilogue_unit(const float4 &va, const float4 &vb
 // Last round of a pass-B tile, any geometry: the top E row bits, each thread owning 2^E rows
 // of one 8-coordinate unit, followed by the epilogue on the registers.
 template <int E, bool COMPRESS, int BITS, bool IDENTITY, bool RANGE>
-__device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, int ccl, int tid,
+__device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, int ccl, int tid, int mask,
                                                   const EpilogueCtx &ep, const PhiloxKeys &keys,
                                                   uint32_t &kmin, uint32_t &kmax)
 {
@@ -634,8 +637,8 @@ __device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, in
 #pragma unroll
         for (int m = 0; m < N; ++m) {
             const int c = ((row_low + (m << rl)) << ccl) + 2 * uu;
-            a[m] = tile[pswz(c)];
-            b[m] = tile[pswz(c + 1)];
+            a[m] = tile[c ^ ((c >> 3) & mask)];
+            b[m] = tile[(c + 1) ^ ((c >> 3) & mask)];
         }
 #pragma unroll
         for (int t = 0; t < E; ++t) {
@@ -729,6 +732,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
     const uint32_t T = 1u << kb;                      // tiles (= panels) per worker-block
     const uint64_t B = 1ull << P.k;
     const int ccl = 11 - kb;                          // log2 chunks per pass-B row
+    const int bmask = (int)P.b_swz_mask;              // swizzle of run-time-geometry pass-B tiles
     const uint64_t d_rows32 = P.d >> 5;               // whole 32-coordinate rows of a gradient
 
     if (tid == 0) {
@@ -975,6 +979,16 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                         tma_load_2d(bufs[s], &maps.ring, x0, y0, &s_mbar[s], pol_ring);
                         tma_load_2d(bufs[s] + 1024, &maps.ring, x0 + 32, y0, &s_mbar[s], pol_ring);
                         tma = 1; phase = uses[s] & 1u; ++uses[s];
+                    } else if (P.b_tma) {
+                        // k = 21: 256 ring rows x 32 columns, one box; k = 22: 512 rows x 16
+                        // columns, two boxes of 256 rows
+                        mbar_expect_tx(&s_mbar[s], kPElems * 4);
+                        const int x0 = (int)(t.idx << (kPLog2 - kb));
+                        const int y0 = (int)(t.slot << kb);
+                        for (uint32_t bx = 0; bx < P.b_tma; ++bx)
+                            tma_load_2d(bufs[s] + (kPChunks / P.b_tma) * bx, &maps.ring, x0, y0 + 256 * (int)bx,
+                                        &s_mbar[s], pol_ring);
+                        tma = 1; phase = uses[s] & 1u; ++uses[s];
                     }
                 }
                 ti.tma = tma;
@@ -1003,7 +1017,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 for (int i = 0; i < kPChunks / kPThreads; ++i) {
                     const int c = tid + i * kPThreads;
                     const int row = c >> ccl, cc = c & ((1 << ccl) - 1);
-                    cp_async16(&tile[pswz(c)], src + ((size_t)row << kPLog2) + 4 * cc);
+                    cp_async16(&tile[c ^ ((c >> 3) & bmask)], src + ((size_t)row << kPLog2) + 4 * cc);
                 }
                 return;
             }
@@ -1119,9 +1133,9 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     round_rows_0_3(tile, tid);
                 } else {
                     switch (e1) {
-                    case 4: p_round<4>(tile, ccl, tid); break;
-                    case 3: p_round<3>(tile, ccl, tid); break;
-                    default: p_round<2>(tile, ccl, tid); break;
+                    case 4: p_round<4>(tile, ccl, tid, bmask); break;
+                    case 3: p_round<3>(tile, ccl, tid, bmask); break;
+                    default: p_round<2>(tile, ccl, tid, bmask); break;
                     }
                 }
                 compute_barrier();
@@ -1131,12 +1145,12 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 } else {
                     const int rem = kb - e1;
                     const int e_last = rem < 3 ? rem : 3;
-                    if (rem > e_last) p_rounds(tile, ccl + e1, ccl + kb - e_last, tid);
+                    if (rem > e_last) p_rounds(tile, ccl + e1, ccl + kb - e_last, tid, bmask);
                     switch (e_last) {
-                    case 3: pass_b_last_round<3, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, ep, keys, kmin, kmax); break;
-                    case 2: pass_b_last_round<2, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, ep, keys, kmin, kmax); break;
-                    case 1: pass_b_last_round<1, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, ep, keys, kmin, kmax); break;
-                    default: pass_b_last_round<0, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, ep, keys, kmin, kmax); break;
+                    case 3: pass_b_last_round<3, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, bmask, ep, keys, kmin, kmax); break;
+                    case 2: pass_b_last_round<2, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, bmask, ep, keys, kmin, kmax); break;
+                    case 1: pass_b_last_round<1, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, bmask, ep, keys, kmin, kmax); break;
+                    default: pass_b_last_round<0, kCompress, BITS, IDENTITY, kRange>(tile, kb, ccl, tid, bmask, ep, keys, kmin, kmax); break;
                     }
                 }
                 if (kRange) {

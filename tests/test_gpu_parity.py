@@ -109,7 +109,7 @@ def test_single_pass_blocks(k, d, n):
 
 @pytest.mark.parametrize("k,d,n", [
     (15, 32_768, 2), (15, 100_000, 2), (16, 65_536 * 2 + 5, 3), (18, 300_000, 2),
-    (20, (1 << 20) + 777, 2), (22, (1 << 22), 1),
+    (20, (1 << 20) + 777, 2), (21, (1 << 22) + 3, 2), (22, (1 << 22), 1), (22, (1 << 23) + 11, 2),
 ])
 def test_two_pass_blocks(k, d, n):
     check_round(_mk(n, d, k))
