@@ -440,6 +440,49 @@ __device__ __forceinline__ double pass_a_round1(float4 *tile, const uint32_t *sw
     return sq;
 }
 
+// First round of a pass-A tile of a bf16 gradient that lies wholly inside the vector: the thread
+// fetches its two rows (64 bytes each) straight from global memory (the control warp has
+// pulled the lines into L2), widens them to fp32 in registers (exact) and goes on as
+// pass_a_round1 does: no staging pass through shared memory, no block barrier.
+__device__ __forceinline__ void pass_a_round1_bf16(float4 *tile, const uint16_t *src, const uint32_t *sw, int tid)
+{
+    const int x = tid & 7;
+    const int r0 = ((tid >> 5) << 6) | (tid & 31);
+    float4 v[16];
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+        const uint4 *p = reinterpret_cast<const uint4 *>(src + (size_t)(r0 + 32 * g) * 32);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint4 t4 = __ldg(p + q);
+            v[8 * g + 2 * q] = make_float4(__uint_as_float(t4.x << 16), __uint_as_float(t4.x & 0xFFFF0000u),
+                                           __uint_as_float(t4.y << 16), __uint_as_float(t4.y & 0xFFFF0000u));
+            v[8 * g + 2 * q + 1] = make_float4(__uint_as_float(t4.z << 16), __uint_as_float(t4.z & 0xFFFF0000u),
+                                               __uint_as_float(t4.w << 16), __uint_as_float(t4.w & 0xFFFF0000u));
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+        const uint32_t w = sw[r0 + 32 * g];
+#pragma unroll
+        for (int m = 0; m < 8; ++m) v[8 * g + m] = flip4(v[8 * g + m], w >> (m * 4));
+    }
+#pragma unroll
+    for (int m = 0; m < 16; ++m) v[m] = stages01(v[m]);
+#pragma unroll
+    for (int t = 0; t < 3; ++t) {
+#pragma unroll
+        for (int m = 0; m < 16; ++m)
+            if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
+    }
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+        float4 *row = tile + (r0 + 32 * g) * 8;
+#pragma unroll
+        for (int m = 0; m < 8; ++m) row[m ^ x] = v[8 * g + m];
+    }
+}
+
 // First round of a pass-A tile of the inverse transform (decompress, error feedback): the same
 // stages as pass_a_round1, but the thread fetches its two rows straight from global memory
 // (the control warp has pulled the lines into L2) and de-quantises them in registers:
@@ -1071,12 +1114,14 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     atomicOr(&P.dev->status, THC_STATUS_WAIT_TIMEOUT);
                     atomicExch(&pc->abort, 1u);
                 }
-            } else if (kCompress || me.is_b) {
+            } else if ((kCompress || me.is_b) &&
+                       !(MODE == kCompressBF16 && !me.is_b &&
+                         (uint64_t)me.r * B + ((uint64_t)me.idx << kPLog2) + kPElems <= P.d)) {
                 load_tile(me, tile);
                 cp_async_commit();
                 cp_async_wait_all();
                 compute_barrier();
-            }                                          // inverse pass A: round 1 fetches its own rows
+            }           // inverse pass A, whole bf16 tiles: round 1 fetches its own rows
             const bool is_b = me.is_b != 0;
             const uint32_t wl = me.wl;
             const uint64_t r = me.r;
@@ -1090,7 +1135,13 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
             if (!is_b) {
                 // ================================ pass A: tile idx of worker-block wb
                 double sq = 0.0;
-                if constexpr (kCompress) {
+                if constexpr (MODE == kCompressBF16) {
+                    const uint64_t j0 = r * B + ((uint64_t)idx << kPLog2);
+                    if (j0 + kPElems <= P.d)
+                        pass_a_round1_bf16(tile, static_cast<const uint16_t *>(in.p[wl]) + j0, sw + 256 * cur, tid);
+                    else
+                        pass_a_round1<true, false>(tile, sw + 256 * cur, tid);
+                } else if constexpr (kCompress) {
                     sq = pass_a_round1<true, kFused>(tile, sw + 256 * cur, tid);
                 } else {
                     constexpr int kInBits = MODE == kDecompress8 ? 8 : MODE == kDecompress16 ? 16
