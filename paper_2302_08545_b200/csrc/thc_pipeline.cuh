@@ -844,29 +844,27 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
             old = __shfl_sync(0xFFFFFFFFu, old, 0);
             if (old + 1u != (r / 16u + 1u) * P.n_local * T) return;
             __threadfence();                           // the other tiles' sums, after seeing the count
+            // Eight workers at a time, four lanes per worker: each lane adds every fourth of
+            // its worker's T tile sums (all loads in flight together), the four lanes are
+            // combined, one square root per worker, then the maximum over the workers.
             double ell = 0.0;
+#pragma unroll 1
             for (uint32_t i0 = 0; i0 < P.n_local; i0 += 8u) {
-                // eight workers at a time: all loads in flight together (T = 128: four per lane)
-                double v[8][4];
+                const uint32_t i = i0 + ((uint32_t)lane >> 2);
+                const bool live = i < P.n_local;
+                const double *p = P.tile_sq + ((size_t)(r * P.n_local + (live ? i : 0u)) << kb) + (lane & 3);
+                double acc = 0.0;
+#pragma unroll 8
+                for (uint32_t c2 = 0; c2 < T; c2 += 4u) acc += __ldcg(p + c2);
+                acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 1);
+                acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 2);
+                double norm = live ? sqrt(acc) : 0.0;
 #pragma unroll
-                for (int w = 0; w < 8; ++w) {
-                    const uint32_t i = i0 + w < P.n_local ? i0 + w : P.n_local - 1u;
-                    const double *p = P.tile_sq + ((size_t)(r * P.n_local + i) << kb);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t c2 = (uint32_t)lane + 32u * j;
-                        v[w][j] = c2 < T ? __ldcg(p + c2) : 0.0;
-                    }
+                for (int off = 4; off < 32; off <<= 1) {
+                    const double other = __shfl_xor_sync(0xFFFFFFFFu, norm, off);
+                    if (other > norm || other != other) norm = other;     // a NaN norm sticks
                 }
-#pragma unroll
-                for (int w = 0; w < 8; ++w) {
-                    double acc = 0.0;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) acc += v[w][j];
-                    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
-                    const double norm = sqrt(acc);
-                    if (i0 + w < P.n_local && (norm > ell || norm != norm)) ell = norm;   // a NaN norm sticks
-                }
+                if (norm > ell || norm != norm) ell = norm;
             }
             if (lane == 0) {
                 float M = (float)(P.t_p * ell / sqrt((double)B));

@@ -553,3 +553,43 @@ def test_aggregate_fast_paths_on_random_indices(bits, g, table, n):
     ref = O.aggregate(packed, sz.d_pad, c, sz.acc_bits)
     dt = {8: np.uint8, 16: np.uint16, 32: np.uint32}[sz.acc_bits]
     assert np.array_equal(total.cpu().numpy().view(dt), ref)
+
+
+def test_prepare_compress_fused_degenerate_blocks():
+    """All-zero and non-finite blocks through the fused scales path: the same scales, status
+    bits and indices as the two separate calls."""
+    import torch
+    from paper_2302_08545_b200 import runner, thc
+    k, n, nblk = 20, 2, 14
+    d = nblk << k
+    w = _mk(n, d, k)
+    x, _ = _inputs(w)
+    x[:, 3 << k:4 << k] = 0.0
+    x[1, (7 << k) + 12345] = np.inf
+    x[0, (9 << k) + 5] = np.nan
+    ctx = runner.context_for(w)
+    r = runner.Round(ctx, n, d)
+    assert r.sz.fused_scales == 1
+    r.upload(x)
+    r.prepare(); r.compress(2)
+    torch.cuda.synchronize()
+    f0 = ctx.status()
+    s0 = r.scales.cpu().numpy().copy(); p0 = [p.cpu().numpy().copy() for p in r.packed]
+    r.scales.fill_(-1.0)
+    for p in r.packed:
+        p.fill_(255)
+    r.prepare_compress(2)
+    torch.cuda.synchronize()
+    f1 = ctx.status()
+    assert f0 == f1 == (thc.STATUS_NONFINITE | thc.STATUS_ZERO_BLOCK)
+    s1 = r.scales.cpu().numpy()
+    assert s1[3] == 0.0 and s1[7] == 0.0 and s1[9] == 0.0
+    ulp = np.abs(s1.view(np.int32).astype(np.int64) - s0.view(np.int32).astype(np.int64))
+    assert ulp.max() <= 1
+    if ulp.max() == 0:
+        for i in range(n):
+            assert np.array_equal(r.packed[i].cpu().numpy(), p0[i])
+    for blk in (3, 7, 9):
+        for i in range(n):
+            seg = r.packed[i].cpu().numpy()[(blk << k) // 2:((blk + 1) << k) // 2]
+            assert not seg.any()
