@@ -39,13 +39,13 @@ KERNELS_PER_STEP = {"prepare": 2, "compress": 1, "prepare_compress": 1, "aggrega
 # variant, measured with ncu on the d=2^24, n=4, b=4 sweep point
 # (profiles/thc_pipeline_kernel_sweep_d2p24_b4_n4.md); traffic grows in proportion to n*d_pad,
 # so a full launch is this times n*d_pad.
-NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.293}
-NCU_FUSED_DRAM_BYTES_PER_COORD = {("f32", 4): 6.213}
+NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.277}
+NCU_FUSED_DRAM_BYTES_PER_COORD = {("f32", 4): 6.227}
 # Executed thread-instructions per (worker, padded coordinate) from the same captures
 # (smsp__inst_executed x 32 / coordinates): the kernel is bound by instruction issue and the
 # shared-memory pipe rather than by HBM, so the issue rate is reported beside the HBM fraction.
-NCU_COMPRESS_THREAD_INST_PER_COORD = {("f32", 4): 47.7}
-NCU_FUSED_THREAD_INST_PER_COORD = {("f32", 4): 50.9}
+NCU_COMPRESS_THREAD_INST_PER_COORD = {("f32", 4): 47.5}
+NCU_FUSED_THREAD_INST_PER_COORD = {("f32", 4): 50.7}
 
 
 def pick_workload(name: str) -> W.Workload:
