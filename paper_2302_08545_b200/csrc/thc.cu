@@ -592,8 +592,10 @@ prepare_partial_kernel(PtrArray in, uint64_t d, uint32_t chunk_log2, uint64_t ch
 }
 
 // M per block from the partial sums (Section 5.3: M = t_p * max_i ||x_i|| / sqrt(B)).  One warp
-// per RHT block; the summation order is fixed (strided per lane, then a butterfly of
-// shuffles), so the result does not depend on timing.
+// per RHT block, eight workers at a time with four lanes per worker: a lane adds every fourth
+// partial sum of its worker (loads independent of each other), the four lanes are combined,
+// one square root per worker, then the maximum over workers.  The order is fixed, so the
+// result does not depend on timing.
 __global__ void __launch_bounds__(128)
 prepare_final_kernel(const double *__restrict__ partial, uint32_t n, uint64_t nblocks,
                      uint64_t chunks_per_block, uint64_t chunks_per_worker, double t_p, uint32_t k,
@@ -603,13 +605,20 @@ prepare_final_kernel(const double *__restrict__ partial, uint32_t n, uint64_t nb
     const int lane = threadIdx.x & 31;
     if (blk >= nblocks) return;
     double ell = 0.0;
-    for (uint32_t i = 0; i < n; ++i) {
+    for (uint32_t i0 = 0; i0 < n; i0 += 8u) {
+        const uint32_t i = i0 + ((uint32_t)lane >> 2);
+        const bool live = i < n;
+        const double *p = partial + (uint64_t)(live ? i : 0u) * chunks_per_worker + blk * chunks_per_block;
         double s = 0.0;
-        const double *p = partial + (uint64_t)i * chunks_per_worker + blk * chunks_per_block;
-        for (uint64_t c = lane; c < chunks_per_block; c += 32) s += p[c];
-        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
-        const double norm = sqrt(s);
-        if (norm > ell || norm != norm) ell = norm;    // a NaN norm sticks
+        for (uint64_t c = (uint64_t)(lane & 3); c < chunks_per_block; c += 4) s += p[c];
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, 1);
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, 2);
+        double norm = live ? sqrt(s) : 0.0;
+        for (int off = 4; off < 32; off <<= 1) {
+            const double other = __shfl_xor_sync(0xFFFFFFFFu, norm, off);
+            if (other > norm || other != other) norm = other;      // a NaN norm sticks
+        }
+        if (norm > ell || norm != norm) ell = norm;
     }
     if (lane != 0) return;
     float M = (float)(t_p * ell / sqrt((double)((uint64_t)1 << k)));
