@@ -15,11 +15,21 @@
 // and returns.
 //
 // Each CTA is four compute warps and one control warp, a producer/consumer pair over two tile
-// buffers.  The control warp claims the next task, waits for its dependency, computes the
-// tile's sign words, starts the TMA load of its tile into the free buffer (completion on an
-// mbarrier) and hands the descriptor over through a full/empty named-barrier handshake; the
-// compute warps wait for the data, run the rounds and signal completion.  Tiles sit in shared
+// buffers.  The control warp claims the next task, starts what does not depend on anything
+// (sign words, the TMA load of a pass-A gradient tile, L2 prefetch of tiles the compute warps
+// fetch themselves), waits for the task's dependency, starts the TMA load of a pass-B panel
+// (completion on an mbarrier) and hands the descriptor over through a full/empty named-barrier
+// handshake; the compute warps wait for the data, run the rounds and report on a `done`
+// mbarrier.  The control warp also signals completions to the other CTAs, so that the release
+// fence is not on the compute warps' path; it does so at the next hand-shake or, while it
+// waits for a dependency, as soon as the `done` mbarrier says so: a wait never holds back the
+// signal of an earlier task, which may be the very thing waited for.  Tiles sit in shared
 // memory in TMA's 128-byte swizzle: 16-byte chunk c at c ^ ((c >> 3) & 7).
+//
+// Modes: compress (fp32 or bf16 gradients in, packed indices out), the same with fused scales,
+// exact range (pass A as compress, the epilogue only takes min / max), decompress (sums of 8,
+// 16 or 32 bits in, fp32 out) and error feedback (a worker's own packed indices in,
+// x - RHT^-1(X) out).  The 2^20 block has a compile-time geometry (KB = 7).
 //
 // Fused scales (kCompressF32Fused; Section 5.3 notes that the norm exchange can run beside the
 // RHT).  Pass A does not need the clamp bound M, only the epilogue of pass B does.  So every
@@ -158,7 +168,6 @@ __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
 
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
 // Named barriers: 1,2 = task slot full; 3,4 = task slot consumed; 5 = compute warps only.
 // bar.sync / bar.arrive are warp-aligned instructions: the __syncwarp() makes sure the warp
@@ -174,17 +183,6 @@ __device__ __forceinline__ void bar_arrive(int id, int count)
     asm volatile("bar.arrive %0, %1;" :: "r"(id), "r"(count) : "memory");
 }
 __device__ __forceinline__ void compute_barrier() { bar_sync(5, kPThreads); }
-
-// Barrier over the compute warps that also ORs a predicate: every thread gets the same answer.
-__device__ __forceinline__ bool compute_barrier_or(bool pred)
-{
-    uint32_t out;
-    __syncwarp();
-    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\t"
-                 "barrier.cta.red.or.pred q, 5, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
-                 : "=r"(out) : "r"((uint32_t)pred), "r"(kPThreads) : "memory");
-    return out != 0;
-}
 
 __device__ __forceinline__ uint32_t atom_release_add(uint32_t *p, uint32_t v)
 {
