@@ -110,6 +110,7 @@ typedef struct thc_sizes_t {
 /* Validate `cfg` (host only) and build a context.  If a CUDA device is present, the
  * context's device block is allocated on the current device; without a device the context
  * still answers thc_sizes() and validation, and every launching call returns THC_ECUDA.
+ * Launching calls must be made with that device current (THC_EINVAL otherwise).
  * Errors: THC_EINVAL (see thc_config), THC_EUNSUPPORTED, THC_ECUDA. */
 int thc_create(const thc_config *cfg, thc_ctx **ctx);
 int thc_destroy(thc_ctx *ctx);

@@ -975,6 +975,10 @@ static int check_launch_ctx(const thc_ctx *ctx)
 {
     if (ctx == nullptr) return THC_EINVAL;
     if (ctx->device < 0 || ctx->dev == nullptr) { g_last_cuda = cudaSuccess; return THC_ECUDA; }
+    // the context's device block, tables and counters live on the device it was created on
+    int cur = -1;
+    THC_CUDA(cudaGetDevice(&cur));
+    if (cur != ctx->device) return THC_EINVAL;
     return THC_OK;
 }
 
