@@ -1169,7 +1169,7 @@ static encode_tiled_t get_encode_tiled()
 // box_rows (32 columns with the 128-byte swizzle, 16 with the 64-byte one).  The data type is
 // UINT32 so that bits travel unchanged.
 static int encode_map(CUtensorMap *map, const void *base, uint64_t cols, uint64_t rows,
-                      uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols = 32u)
+                      uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols = 32u, bool half_words = false)
 {
     encode_tiled_t enc = get_encode_tiled();
     if (enc == nullptr) return THC_ECUDA;
@@ -1177,9 +1177,13 @@ static int encode_map(CUtensorMap *map, const void *base, uint64_t cols, uint64_
     const cuuint64_t strides[1] = {pitch_bytes};
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1u, 1u};
-    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(base), dims, strides,
+    // 16-bit elements (bf16 gradients as rows of 32: 64 bytes) or 32-bit words; rows of 64
+    // bytes take the 64-byte swizzle
+    const bool rows64 = half_words ? box_cols == 32u : box_cols == 16u;
+    const CUresult r = enc(map, half_words ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32, 2,
+                           const_cast<void *>(base), dims, strides,
                            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           box_cols == 16u ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                           rows64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? THC_OK : THC_ECUDA;
 }
@@ -1188,7 +1192,7 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
                            const thc_sizes_t &sz, uint64_t d, uint32_t n_local, uint32_t worker_base, uint32_t round, uint32_t divisor,
                            const float *scales, void *workspace, const PtrArrayP &in,
                            const MutPtrArrayP &out, const MutPtrArrayP &rot, cudaStream_t st,
-                           float *fused_scales_out = nullptr)
+                           float *fused_scales_out = nullptr, bool compress_bf16 = false)
 {
     const uint32_t k = ctx->cfg.log2_block;
     PipeParams P;
@@ -1254,6 +1258,12 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
     if (compress_f32 && (d >> 5) >= 256) {
         for (uint32_t i = 0; i < n_local; ++i) {
             const int rc = encode_map(&maps.in[i], in.p[i], 32u, d >> 5, 128u, 256u);
+            if (rc != THC_OK) return rc;
+        }
+    }
+    if (compress_bf16 && (d >> 5) >= 256) {
+        for (uint32_t i = 0; i < n_local; ++i) {
+            const int rc = encode_map(&maps.in[i], in.p[i], 32u, d >> 5, 64u, 256u, 32u, true);
             if (rc != THC_OK) return rc;
         }
     }
@@ -1368,7 +1378,7 @@ int thc_compress(thc_ctx *ctx, const void *const *grads, uint32_t n_local, uint3
     pipe_kernel_t kern = bf16 ? pick_pipe_kernel<kCompressBF16>(ctx->cfg.bits, ctx->identity, k)
                               : pick_pipe_kernel<kCompressF32>(ctx->cfg.bits, ctx->identity, k);
     return launch_pipeline(ctx, kern, !bf16, sz, d, n_local, worker_base, round, 1, scales, workspace,
-                           pin, pout, prot, st);
+                           pin, pout, prot, st, nullptr, bf16);
 }
 
 // Scales and compress in one launch (see thc.h).  Falls back to the two separate calls where

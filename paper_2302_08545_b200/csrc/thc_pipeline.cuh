@@ -438,26 +438,32 @@ __device__ __forceinline__ double pass_a_round1(float4 *tile, const uint32_t *sw
     return sq;
 }
 
-// First round of a pass-A tile of a bf16 gradient that lies wholly inside the vector: the thread
-// fetches its two rows (64 bytes each) straight from global memory (the control warp has
-// pulled the lines into L2), widens them to fp32 in registers (exact) and goes on as
-// pass_a_round1 does: no staging pass through shared memory, no block barrier.
-__device__ __forceinline__ void pass_a_round1_bf16(float4 *tile, const uint16_t *src, const uint32_t *sw, int tid)
+// First round of a pass-A tile of a bf16 gradient that lies wholly inside the vector: the TMA
+// unit has put the 16 KB of bf16 (256 rows of 64 bytes, 64-byte swizzle) into the upper half of
+// the tile buffer.  Every thread reads its two rows into registers; after a block barrier
+// (the fp32 rows written next overlap other threads' bf16 rows) the values are widened to fp32
+// (exact) and the round goes on as pass_a_round1 does.
+__device__ __forceinline__ void pass_a_round1_bf16(float4 *tile, const uint32_t *sw, int tid)
 {
     const int x = tid & 7;
     const int r0 = ((tid >> 5) << 6) | (tid & 31);
-    float4 v[16];
+    const uint4 *stage = reinterpret_cast<const uint4 *>(tile) + kPChunks / 2;
+    uint4 raw[8];
 #pragma unroll
     for (int g = 0; g < 2; ++g) {
-        const uint4 *p = reinterpret_cast<const uint4 *>(src + (size_t)(r0 + 32 * g) * 32);
+        const int row = r0 + 32 * g;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint4 t4 = __ldg(p + q);
-            v[8 * g + 2 * q] = make_float4(__uint_as_float(t4.x << 16), __uint_as_float(t4.x & 0xFFFF0000u),
-                                           __uint_as_float(t4.y << 16), __uint_as_float(t4.y & 0xFFFF0000u));
-            v[8 * g + 2 * q + 1] = make_float4(__uint_as_float(t4.z << 16), __uint_as_float(t4.z & 0xFFFF0000u),
-                                               __uint_as_float(t4.w << 16), __uint_as_float(t4.w & 0xFFFF0000u));
-        }
+        for (int q = 0; q < 4; ++q) raw[4 * g + q] = stage[row * 4 + (q ^ ((row >> 1) & 3))];
+    }
+    compute_barrier();
+    float4 v[16];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint4 t4 = raw[i];
+        v[2 * i] = make_float4(__uint_as_float(t4.x << 16), __uint_as_float(t4.x & 0xFFFF0000u),
+                               __uint_as_float(t4.y << 16), __uint_as_float(t4.y & 0xFFFF0000u));
+        v[2 * i + 1] = make_float4(__uint_as_float(t4.z << 16), __uint_as_float(t4.z & 0xFFFF0000u),
+                                   __uint_as_float(t4.w << 16), __uint_as_float(t4.w & 0xFFFF0000u));
     }
 #pragma unroll
     for (int g = 0; g < 2; ++g) {
@@ -926,7 +932,12 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                         tma_load_2d(bufs[s], &maps.in[wl], 0, (int)(j0 >> 5), &s_mbar[s], pol_stream);
                         tma = 1; phase = uses[s] & 1u; ++uses[s];
                     }
-                    if (!kF32In) {
+                    if (lane == 0 && MODE == kCompressBF16 && (j0 >> 5) + 256 <= d_rows32) {
+                        mbar_expect_tx(&s_mbar[s], kPElems * 2);
+                        tma_load_2d(bufs[s] + kPChunks / 2, &maps.in[wl], 0, (int)(j0 >> 5), &s_mbar[s], pol_stream);
+                        tma = 1; phase = uses[s] & 1u; ++uses[s];
+                    }
+                    if (!kF32In && !(MODE == kCompressBF16 && (j0 >> 5) + 256 <= d_rows32)) {
                         // tiles the compute warps load themselves: pull the lines into L2 now
                         const uint32_t in_bits = MODE == kCompressBF16 ? 16u : MODE == kDecompress8 ? 8u
                                                  : MODE == kDecompress16 ? 16u : MODE == kDecompress32 ? 32u
@@ -1110,14 +1121,12 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     atomicOr(&P.dev->status, THC_STATUS_WAIT_TIMEOUT);
                     atomicExch(&pc->abort, 1u);
                 }
-            } else if ((kCompress || me.is_b) &&
-                       !(MODE == kCompressBF16 && !me.is_b &&
-                         (uint64_t)me.r * B + ((uint64_t)me.idx << kPLog2) + kPElems <= P.d)) {
+            } else if (kCompress || me.is_b) {
                 load_tile(me, tile);
                 cp_async_commit();
                 cp_async_wait_all();
                 compute_barrier();
-            }           // inverse pass A, whole bf16 tiles: round 1 fetches its own rows
+            }                                          // inverse pass A: round 1 fetches its own rows
             const bool is_b = me.is_b != 0;
             const uint32_t wl = me.wl;
             const uint64_t r = me.r;
@@ -1133,8 +1142,9 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 double sq = 0.0;
                 if constexpr (MODE == kCompressBF16) {
                     const uint64_t j0 = r * B + ((uint64_t)idx << kPLog2);
-                    if (j0 + kPElems <= P.d)
-                        pass_a_round1_bf16(tile, static_cast<const uint16_t *>(in.p[wl]) + j0, sw + 256 * cur, tid);
+                    (void)j0;
+                    if (me.tma)
+                        pass_a_round1_bf16(tile, sw + 256 * cur, tid);
                     else
                         pass_a_round1<true, false>(tile, sw + 256 * cur, tid);
                 } else if constexpr (kCompress) {
