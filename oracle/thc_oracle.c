@@ -351,7 +351,8 @@ void thc_oracle_estimate_range(const void *sum, uint32_t w, uint32_t divisor, ui
     uint64_t B = (uint64_t)1 << k;
     for (uint64_t j = 0; j < d_pad; ++j) {
         float m = lo[j / B], M = hi[j / B];
-        if (!(M > m) || !isfinite(M) || !isfinite(m)) { v[j] = 0.0f; continue; }   /* R8 */
+        if (!(M >= m) || !isfinite(M) || !isfinite(m)) { v[j] = 0.0f; continue; }  /* R8 */
+        /* M == m (a constant block: every index is 0): the estimate line gives m itself */
         uint32_t y = w == 8 ? ((const uint8_t *)sum)[j]
                    : w == 16 ? ((const uint16_t *)sum)[j]
                              : ((const uint32_t *)sum)[j];
@@ -409,7 +410,7 @@ void thc_oracle_error_feedback_range(const float *x, const uint8_t *z, uint64_t 
     float *back = (float *)malloc(sizeof(float) * d);
     for (uint64_t j = 0; j < d_pad; ++j) {
         float m = lo[j / B], M = hi[j / B];
-        if (!(M > m) || !isfinite(M) || !isfinite(m)) { v[j] = 0.0f; continue; }   /* R8 */
+        if (!(M >= m) || !isfinite(M) || !isfinite(m)) { v[j] = 0.0f; continue; }  /* R8 */
         float step = (float)(((double)M - (double)m) / (double)g);
         v[j] = fmaf((float)table[z[j]], step, m);
     }

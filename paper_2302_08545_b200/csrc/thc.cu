@@ -645,7 +645,7 @@ __global__ void range_final_kernel(const uint32_t *keys, uint64_t nblocks, float
     float lo = key_float(keys[i]), hi = key_float(keys[nblocks + i]);
     uint32_t flags = 0;
     if (!isfinite(lo) || !isfinite(hi)) { lo = 0.0f; hi = 0.0f; flags |= THC_STATUS_NONFINITE; }
-    if (!(hi > lo)) flags |= THC_STATUS_ZERO_BLOCK;
+    if (hi == 0.0f && lo == 0.0f) flags |= THC_STATUS_ZERO_BLOCK;   // a constant block decodes exactly
     scales[i] = lo;
     scales[nblocks + i] = hi;
     if (flags) atomicOr(&dev->status, flags);

@@ -93,10 +93,11 @@ __device__ __forceinline__ float2 compress_constants(BlockRange b)
 }
 
 // (step, base) of v = fma(Y, step, base): (hi - lo)/(g * divisor) and lo; (0, 0) for a
-// degenerate block (decodes to zeros).
+// degenerate block (decodes to zeros).  hi == lo (a constant block: every index is 0) gives
+// step 0 and base lo: the estimate line of Algorithm 2 with M = m.
 __device__ __forceinline__ float2 decode_constants(BlockRange b, uint32_t g, uint32_t divisor)
 {
-    if (!(b.hi > b.lo) || !isfinite(b.hi) || !isfinite(b.lo)) return make_float2(0.f, 0.f);
+    if (!(b.hi >= b.lo) || !isfinite(b.hi) || !isfinite(b.lo)) return make_float2(0.f, 0.f);
     const double w = (double)b.hi - (double)b.lo;
     return make_float2((float)(w / ((double)g * (double)divisor)), b.lo);
 }

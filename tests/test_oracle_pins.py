@@ -695,3 +695,20 @@ def test_exact_range_round_has_no_truncation_error_on_heavy_tails():
     e_norm = ((out_norm - base) ** 2).sum() / (base.astype(np.float64) ** 2).sum()
     e_exact = ((out_exact - base) ** 2).sum() / (base.astype(np.float64) ** 2).sum()
     assert e_exact < 0.05 and e_norm > 5 * e_exact
+
+
+def test_exact_range_constant_block_decodes_to_the_constant():
+    """One non-zero coordinate in the first position of a block rotates to a constant block
+    (column 0 of H is all ones): min = max, every index is 0, and the estimate line
+    m + X (M - m)/g with M = m returns m, so the round reproduces the input."""
+    k = 4
+    c = cfg(k=k)
+    x = np.zeros((1, 48), np.float32)
+    x[0, 16] = 3.25                                       # first coordinate of block 1
+    x[0, 5] = -1.0
+    lo, hi = O.ranges(x, c, 2)
+    assert lo[1] == hi[1] and abs(abs(lo[1]) - 3.25 / 4.0) < 1e-7 and lo[2] == 0.0 == hi[2]
+    out = O.thc_round(x, c, 2, exact_range=True)
+    z = O.unpack(out["packed"][0], 48, 4)
+    assert not z[16:48].any()
+    assert out["out"][16] == np.float32(3.25) and not out["out"][17:].any()
