@@ -83,3 +83,39 @@ def test_random_configuration(case):
         z = O.unpack(packed[i], r.sz.d_pad, w.bits)
         e = O.error_feedback(x[i], z, hi, c, rnd, lo=lo)
         assert np.array_equal(ef[i].cpu().numpy().view(np.uint32), e.view(np.uint32)), (p, i)
+
+
+@pytest.mark.parametrize("case", range(12))
+def test_random_bf16_configuration(case):
+    """The same for bf16 gradients (widened exactly to fp32 on both sides)."""
+    import torch
+    from paper_2302_08545_b200 import runner
+    rng = np.random.default_rng(70_000 + case)
+    k = int(rng.choice([4, 9, 13, 14, 15, 16, 18, 20, 21, 22]))
+    B = 1 << k
+    nblk = int(rng.integers(1, 4 if k <= 18 else 3))
+    d = (nblk - 1) * B + int(rng.integers(1, B + 1))
+    n = int(rng.integers(1, 6 if k <= 18 else 3))
+    rnd = int(rng.integers(0, 1 << 16))
+    w = W.Workload(f"randbf{case}", n=n, d=d, log2_block=k, bits=4, granularity=30, table=W.TABLES[(4, 30)],
+                   in_dtype="bf16", data_seed=case, t_p=W.T_P["1/32"])
+    xf = (rng.standard_normal((n, d)) * 1e-2).astype(np.float32)
+    bits16 = (xf.view(np.uint32) >> 16).astype(np.uint16)             # truncate to bf16
+    x = O.bf16_to_f32(bits16)
+    c = O.Config(bits=4, granularity=30, table=tuple(w.table), t_p=w.t_p, log2_block=k, seed=w.seed)
+    ctx = runner.context_for(w)
+    r = runner.Round(ctx, n, d, "bf16")
+    r.upload(bits16)
+    r.run(rnd)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    s = r.scales.cpu().numpy()
+    ulp = np.abs(s.view(np.int32).astype(np.int64) - O.scales(x, c).view(np.int32).astype(np.int64))
+    assert ulp.max() <= 1
+    packed = np.stack([q.cpu().numpy() for q in r.packed])
+    exp_packed, _ = O.compress(x, s, c, rnd)
+    assert np.array_equal(packed, exp_packed), (k, d, n)
+    total = r.sum_numpy()
+    assert np.array_equal(total, O.aggregate(packed, r.sz.d_pad, c, r.sz.acc_bits))
+    out_ref = O.decompress(total, n, d, s, c, rnd)
+    assert np.array_equal(r.out.cpu().numpy().view(np.uint32), out_ref.view(np.uint32))
