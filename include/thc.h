@@ -192,9 +192,13 @@ int thc_prepare_noalloc(const void *const *grads, uint32_t n, uint64_t d, uint32
  * counterpart in THC_RANGE_NORM mode).  thc_compress, thc_quantize_rotated, thc_decompress and
  * thc_error_feedback of such a context read `scales` in this layout and use the range
  * [m, M] of Algorithm 2 as given: no coordinate is clamped.  Costs one transform pass over the
- * inputs.  A block with a non-finite rotated coordinate gets (0, 0) and THC_STATUS_NONFINITE. */
+ * inputs.  A block with a non-finite rotated coordinate gets (0, 0) and THC_STATUS_NONFINITE.
+ * rotated_or_null: host array of n device pointers (d_pad fp32 each) that receive the rotated
+ * coordinates, so that thc_quantize_rotated can finish the compression without a second
+ * transform; null (or a null entry) to skip. */
 int thc_prepare_minmax(thc_ctx *ctx, const void *const *grads, uint32_t n, uint64_t d, uint32_t round,
-                       float *scales, void *workspace, uint64_t workspace_bytes, void *stream);
+                       float *scales, float *const *rotated_or_null, void *workspace,
+                       uint64_t workspace_bytes, void *stream);
 
 /* thc_prepare and thc_compress in one launch, for callers that hold all n workers' gradients
  * (the simulated cluster): same arguments and results as the two calls in a row, `scales`

@@ -267,6 +267,7 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
             const uint64_t j = chunk_coord(g, base, c);
             if (j >= g.d_pad) continue;
             const float4 v = scale4(tile[swz(c)], g.c_block);
+            if (rotated.p[wl] != nullptr) *reinterpret_cast<float4 *>(static_cast<float *>(rotated.p[wl]) + j) = v;
             const uint32_t k0 = float_key(v.x), k1 = float_key(v.y), k2 = float_key(v.z), k3 = float_key(v.w);
             uint32_t kmin = min(min(k0, k1), min(k2, k3));
             uint32_t kmax = max(max(k0, k1), max(k2, k3));
@@ -1277,7 +1278,8 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
 // the keys become the (lo, hi) planes of `scales`.  This costs about as much as the transform
 // half of thc_compress: the price of a range that clamps nothing.
 int thc_prepare_minmax(thc_ctx *ctx, const void *const *grads, uint32_t n, uint64_t d, uint32_t round,
-                       float *scales, void *workspace, uint64_t workspace_bytes, void *stream)
+                       float *scales, float *const *rotated, void *workspace, uint64_t workspace_bytes,
+                       void *stream)
 {
     int rc0 = check_launch_ctx(ctx);
     if (rc0 != THC_OK) return rc0;
@@ -1305,7 +1307,13 @@ int thc_prepare_minmax(thc_ctx *ctx, const void *const *grads, uint32_t n, uint6
         memset(&in, 0, sizeof in);
         memset(&out, 0, sizeof out);
         memset(&rot, 0, sizeof rot);
-        for (uint32_t i = 0; i < n; ++i) in.p[i] = grads[i];
+        for (uint32_t i = 0; i < n; ++i) {
+            in.p[i] = grads[i];
+            if (rotated != nullptr && rotated[i] != nullptr) {
+                if (!aligned16(rotated[i])) return THC_EINVAL;
+                rot.p[i] = rotated[i];
+            }
+        }
         out.p[0] = keys;
         TileGeom g = base_geom(ctx, sz, d, round);
         geom_pass_a(g);
@@ -1318,7 +1326,13 @@ int thc_prepare_minmax(thc_ctx *ctx, const void *const *grads, uint32_t n, uint6
         memset(&pin, 0, sizeof pin);
         memset(&pout, 0, sizeof pout);
         memset(&prot, 0, sizeof prot);
-        for (uint32_t i = 0; i < n; ++i) pin.p[i] = grads[i];
+        for (uint32_t i = 0; i < n; ++i) {
+            pin.p[i] = grads[i];
+            if (rotated != nullptr && rotated[i] != nullptr) {
+                if (!aligned16(rotated[i])) return THC_EINVAL;
+                prot.p[i] = rotated[i];
+            }
+        }
         rc = launch_pipeline(ctx, pick_pipe_kernel<kRangeF32>(4, true, k), true, sz, d, n, 0, round,
                              1, scales, workspace, pin, pout, prot, st);
     }

@@ -618,6 +618,10 @@ __device__ __forceinline__ void epilogue_unit(const float4 &va, const float4 &vb
     const float4 ra = scale4(va, ep.c_block);
     const float4 rb = scale4(vb, ep.c_block);
     if constexpr (RANGE) {
+        if (ep.rotated != nullptr) {
+            *reinterpret_cast<float4 *>(ep.rotated + j) = ra;
+            *reinterpret_cast<float4 *>(ep.rotated + j + 4) = rb;
+        }
         const float r[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
 #pragma unroll
         for (int e = 0; e < 8; ++e) {

@@ -56,7 +56,8 @@ class Round:
         self.ctx.prepare(self.grads, self.d, self.scales, self.workspace, stream)
 
     def prepare_minmax(self, rnd: int = 0, stream=None):
-        self.ctx.prepare_minmax(self.grads, self.d, rnd, self.scales, self.workspace, stream)
+        self.ctx.prepare_minmax(self.grads, self.d, rnd, self.scales, self.workspace,
+                                rotated=self.rotated, stream=stream)
 
     def compress(self, rnd: int = 0, stream=None):
         self.ctx.compress(self.grads, self.d, rnd, self.scales, self.packed, self.workspace,
@@ -65,6 +66,9 @@ class Round:
     def prepare_compress(self, rnd: int = 0, stream=None):
         self.ctx.prepare_compress(self.grads, self.d, rnd, self.scales, self.packed, self.workspace,
                                   rotated=self.rotated, stream=stream)
+
+    def quantize_rotated(self, rnd: int = 0, stream=None):
+        self.ctx.quantize_rotated(self.rotated, self.d, rnd, self.scales, self.packed, stream=stream)
 
     def aggregate(self, stream=None):
         self.ctx.aggregate(self.packed, self.d, self.total, stream)

@@ -80,7 +80,7 @@ def lib():
     L.thc_aggregate.argtypes = [vp, pp, u32, u64, vp, vp]
     L.thc_decompress.argtypes = [vp, vp, u32, u64, u32, vp, vp, vp, u64, vp]
     L.thc_prepare_noalloc.argtypes = [pp, u32, u64, u32, u32, ctypes.c_double, vp, vp, vp]
-    L.thc_prepare_minmax.argtypes = [vp, pp, u32, u64, u32, vp, vp, u64, vp]
+    L.thc_prepare_minmax.argtypes = [vp, pp, u32, u64, u32, vp, pp, vp, u64, vp]
     L.thc_prepare_compress.argtypes = [vp, pp, u32, u32, u64, u32, vp, pp, pp, vp, u64, vp]
     L.thc_error_feedback.argtypes = [vp, pp, pp, u32, u64, u32, vp, pp, vp, u64, vp]
     L.thc_accumulate_error.argtypes = [vp, pp, pp, u32, u64, vp]
@@ -186,9 +186,10 @@ class Context:
                                  workspace.numel() * workspace.element_size(), _stream(stream)),
                "thc_prepare")
 
-    def prepare_minmax(self, grads, d: int, rnd: int, scales, workspace, stream=None):
+    def prepare_minmax(self, grads, d: int, rnd: int, scales, workspace, rotated=None, stream=None):
         arr = _ptr_array([_dp(g) for g in grads])
-        _check(lib().thc_prepare_minmax(self._h, arr, len(grads), d, rnd, _dp(scales), _dp(workspace),
+        ra = _ptr_array([_dp(r) for r in rotated]) if rotated is not None else None
+        _check(lib().thc_prepare_minmax(self._h, arr, len(grads), d, rnd, _dp(scales), ra, _dp(workspace),
                                         workspace.numel() * workspace.element_size(), _stream(stream)),
                "thc_prepare_minmax")
 

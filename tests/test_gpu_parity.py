@@ -593,3 +593,30 @@ def test_prepare_compress_fused_degenerate_blocks():
         for i in range(n):
             seg = r.packed[i].cpu().numpy()[(blk << k) // 2:((blk + 1) << k) // 2]
             assert not seg.any()
+
+
+@pytest.mark.parametrize("k,d,n", [(10, 33_001, 2), (16, 150_000, 2), (20, (1 << 21) + 99, 2)])
+def test_exact_range_with_rotated_output_needs_one_transform(k, d, n):
+    """thc_prepare_minmax can hand out the rotated coordinates; thc_quantize_rotated on them
+    gives the same packed indices as thc_compress (which transforms again)."""
+    import torch
+    from paper_2302_08545_b200 import runner
+    w = _mk(n, d, k)
+    x, _ = _inputs(w)
+    ctx = runner.context_for(w, exact_range=True)
+    r = runner.Round(ctx, n, d, want_rotated=True)
+    r.upload(x)
+    r.prepare_minmax(6)
+    r.quantize_rotated(6)
+    torch.cuda.synchronize()
+    one_pass = [p.cpu().numpy().copy() for p in r.packed]
+    rot = [t.cpu().numpy().copy() for t in r.rotated]
+    for p in r.packed:
+        p.zero_()
+    r.compress(6)
+    torch.cuda.synchronize()
+    c = _ocfg(w)
+    for i in range(n):
+        assert np.array_equal(one_pass[i], r.packed[i].cpu().numpy())
+        assert np.array_equal(rot[i].view(np.uint32), O.rht_forward(x[i], c, 6).view(np.uint32))
+    assert ctx.status() == 0
