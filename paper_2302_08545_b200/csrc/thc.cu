@@ -300,6 +300,8 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
     }
 }
 
+constexpr int kQrBlockCache = 1024;
+
 // Quantise + pack coordinates that are already rotated (the epilogue of compress alone).
 template <int BITS, bool IDENTITY>
 __global__ void __launch_bounds__(kThreads)
@@ -307,23 +309,34 @@ quantize_rotated_kernel(PtrArray rotated, MutPtrArray packed, uint64_t d_pad, ui
                         uint32_t granularity, uint32_t round, uint32_t worker_base, uint32_t exact_range,
                         const float *__restrict__ scales, const DeviceBlock *dev, PhiloxKeys keys)
 {
-    __shared__ uint4 lut[256];
-    for (int f = threadIdx.x; f <= (int)granularity; f += kThreads) lut[f] = dev->lut[f];
+    // dynamic shared memory: the quantiser table, one copy per lane group, then the block
+    // constants of the first kQrBlockCache RHT blocks (the fp64 division is done once per block)
+    extern __shared__ __align__(16) unsigned char qr_smem[];
+    uint4 *lut = reinterpret_cast<uint4 *>(qr_smem);
+    float2 *bc = reinterpret_cast<float2 *>(qr_smem + (size_t)(granularity + 1) * kLutRep * 16);
+    for (int idx = threadIdx.x; idx < (int)(granularity + 1) * kLutRep; idx += kThreads)
+        lut[idx] = dev->lut[idx / kLutRep];
+    const uint64_t nblocks = d_pad >> k;
+    const uint32_t cached = nblocks < (uint64_t)kQrBlockCache ? (uint32_t)nblocks : (uint32_t)kQrBlockCache;
+    for (uint32_t b = threadIdx.x; b < cached; b += kThreads)
+        bc[b] = compress_constants(block_range(scales, b, nblocks, exact_range));
     __syncthreads();
     const uint32_t wl = blockIdx.y;
     const float *rot = static_cast<const float *>(rotated.p[wl]);
     unsigned char *pk = static_cast<unsigned char *>(packed.p[wl]);
     const float gf = (float)granularity;
+    const uint4 *my_lut = lut + (threadIdx.x & (kLutRep - 1));
     for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < d_pad / 8;
          u += (uint64_t)gridDim.x * kThreads) {
         const uint64_t j = u * 8;
         const float4 a = __ldg(reinterpret_cast<const float4 *>(rot + j));
         const float4 b = __ldg(reinterpret_cast<const float4 *>(rot + j + 4));
         const float r[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-        const float2 kc = compress_constants(block_range(scales, j >> k, d_pad >> k, exact_range));
+        const uint64_t blk = j >> k;
+        const float2 kc = blk < cached ? bc[blk] : compress_constants(block_range(scales, blk, nblocks, exact_range));
         const float kappa = kc.x, offset = kc.y;
         const uint4 rnd = round_call(j, worker_base + wl, round, keys);
-        const uint64_t z = quantize8<BITS, IDENTITY>(r, kappa, offset, gf, rnd, lut, 1);
+        const uint64_t z = quantize8<BITS, IDENTITY>(r, kappa, offset, gf, rnd, my_lut, kLutRep);
         if constexpr (BITS == 8) *reinterpret_cast<uint2 *>(pk + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
         else if constexpr (BITS == 4) *reinterpret_cast<uint32_t *>(pk + j / 2) = (uint32_t)z;
         else if constexpr (BITS == 2) *reinterpret_cast<uint16_t *>(pk + j / 4) = (uint16_t)z;
@@ -1506,7 +1519,8 @@ int thc_quantize_rotated(thc_ctx *ctx, const float *const *rotated, uint32_t n_l
     if (blocks > cap) blocks = cap;
     const dim3 grid((unsigned)blocks, n_local);
     const uint32_t k = ctx->cfg.log2_block, g = ctx->cfg.granularity;
-#define THC_QR(B, I) quantize_rotated_kernel<B, I><<<grid, kThreads, 0, st>>>( \
+    const size_t qr_smem = (size_t)(g + 1) * kLutRep * 16 + (size_t)kQrBlockCache * 8;
+#define THC_QR(B, I) quantize_rotated_kernel<B, I><<<grid, kThreads, qr_smem, st>>>( \
         in, out, sz.d_pad, k, g, round, worker_base,                         \
         ctx->cfg.range_mode == THC_RANGE_MINMAX ? 1u : 0u, scales, ctx->dev, ctx->keys)
     switch (ctx->cfg.bits) {
