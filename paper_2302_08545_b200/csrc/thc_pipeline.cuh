@@ -922,15 +922,6 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 if (!t.is_b) {
                     // pass A reads only the caller's input: start the load before looking at
                     // the ring slot, which only the end of the task writes to
-                    if (kCompress) {
-                        // sign words of the tile: 64 Philox calls, two per lane
-#pragma unroll
-                        for (int c = 0; c < 2; ++c) {
-                            const int call = lane + 32 * c;
-                            const uint4 ph = sign_call(j0 + 128ull * call, P.round, keys);
-                            *reinterpret_cast<uint4 *>(sw + 256 * s + 4 * call) = ph;
-                        }
-                    }
                     if (lane == 0 && kF32In && (j0 >> 5) + 256 <= d_rows32) {
                         mbar_expect_tx(&s_mbar[s], kPElems * 4);
                         tma_load_2d(bufs[s], &maps.in[wl], 0, (int)(j0 >> 5), &s_mbar[s], pol_stream);
@@ -952,6 +943,15 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                         const uint32_t lines = (uint32_t)kPElems * in_bits / 8 / 128;
                         for (uint32_t l = (uint32_t)lane; l < lines; l += 32u)
                             if (first + 128ull * l < limit) prefetch_l2(src + first + 128ull * l);
+                    }
+                    if (kCompress) {
+                        // sign words of the tile (64 Philox calls, two per lane), while the copy is in flight
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            const int call = lane + 32 * c;
+                            const uint4 ph = sign_call(j0 + 128ull * call, P.round, keys);
+                            *reinterpret_cast<uint4 *>(sw + 256 * s + 4 * call) = ph;
+                        }
                     }
                 }
                 // pass B needs its worker-block's tiles (fused scales: the block's M, which
@@ -996,25 +996,6 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 ti.gen = t.gen;
                 pend[s] = t;
                 pend_valid[s] = true;
-                if (t.is_b && !kCompress && KB == 7) {
-                    // inverse transform: sign words of the panel's 128 rows x 64 columns (two
-                    // words per row), and for error feedback the x values the epilogue will read
-                    const uint64_t j_panel = (uint64_t)r * B + ((uint64_t)t.idx << 6);
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const int row = lane + 32 * c;
-                        const uint64_t jr = j_panel + ((uint64_t)row << kPLog2);
-                        const uint4 ph = sign_call(jr, P.round, keys);
-                        const bool hi = ((jr >> 5) & 3u) != 0;         // words 2,3 of the call
-                        sw[256 * s + 2 * row] = hi ? ph.z : ph.x;
-                        sw[256 * s + 2 * row + 1] = hi ? ph.w : ph.y;
-                        if (kEF) {
-                            const float *xr = static_cast<const float *>(rotated.p[t.wb - r * P.n_local]) + jr;
-                            if (jr < P.d) prefetch_l2(xr);
-                            if (jr + 32 < P.d) prefetch_l2(xr + 32);
-                        }
-                    }
-                }
                 if (lane == 0 && t.is_b) {
                     if (kFused) {
                         BlockRange br;
@@ -1043,6 +1024,25 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                             tma_load_2d(bufs[s] + (kPChunks / P.b_tma) * bx, &maps.ring, x0, y0 + 256 * (int)bx,
                                         &s_mbar[s], pol_ring);
                         tma = 1; phase = uses[s] & 1u; ++uses[s];
+                    }
+                }
+                if (t.is_b && !kCompress && KB == 7) {
+                    // inverse transform: sign words of the panel's 128 rows x 64 columns (two
+                    // words per row), and for error feedback the x values the epilogue will read
+                    const uint64_t j_panel = (uint64_t)r * B + ((uint64_t)t.idx << 6);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int row = lane + 32 * c;
+                        const uint64_t jr = j_panel + ((uint64_t)row << kPLog2);
+                        const uint4 ph = sign_call(jr, P.round, keys);
+                        const bool hi = ((jr >> 5) & 3u) != 0;         // words 2,3 of the call
+                        sw[256 * s + 2 * row] = hi ? ph.z : ph.x;
+                        sw[256 * s + 2 * row + 1] = hi ? ph.w : ph.y;
+                        if (kEF) {
+                            const float *xr = static_cast<const float *>(rotated.p[t.wb - r * P.n_local]) + jr;
+                            if (jr < P.d) prefetch_l2(xr);
+                            if (jr + 32 < P.d) prefetch_l2(xr + 32);
+                        }
                     }
                 }
                 ti.tma = tma;
