@@ -7,6 +7,9 @@
  *     thc_compress    RHT -> truncate -> stochastic quantisation to b-bit table indices -> pack
  *     thc_aggregate   the parameter server's only job: Y = sum_i T[Z_i], in integers
  *     thc_decompress  Y/n -> real values -> inverse RHT
+ * and around them: thc_prepare_compress (the first two in one launch), thc_prepare_minmax (the
+ * exact range of Algorithm 1's preliminary stage instead of the norm-based one),
+ * thc_quantize_rotated, thc_error_feedback / thc_accumulate_error (Algorithm 3's residual).
  *
  * Conventions shared by every call
  *   - "device" pointers are CUDA device addresses on the device that was current when the
@@ -17,7 +20,8 @@
  *   - Every device buffer is owned by the caller.  Device buffers must be 16-byte aligned.
  *     The library owns only the context (a few hundred bytes of device memory for the
  *     status word and scheduling counters, allocated by thc_create).
- *   - The four round calls and thc_quantize_rotated only enqueue work on `stream`
+ *   - The round calls (and thc_quantize_rotated, thc_prepare_compress, thc_prepare_minmax,
+ *     thc_error_feedback, thc_accumulate_error) only enqueue work on `stream`
  *     (a cudaStream_t passed as void*; NULL = the legacy default stream) and return without
  *     synchronising.  They allocate nothing.  Calls that share a context must be issued
  *     on one stream (or be ordered by the caller): they share the context's counters.
@@ -27,7 +31,8 @@
  *
  * Layouts (coordinate j = 0 .. d_pad-1, d_pad = d rounded up to a multiple of B = 2^k)
  *   gradient   d elements, fp32 or bf16, contiguous; coordinates d..d_pad-1 count as zero
- *   scales     one fp32 M per block, nblocks = d_pad / B entries
+ *   scales     one fp32 M per block, nblocks = d_pad / B entries (THC_RANGE_MINMAX contexts:
+ *              nblocks minima followed by nblocks maxima; thc_sizes_t.scales_count)
  *   packed     d_pad*b/8 bytes per worker; index j in bits [(j mod 8/b)*b, +b) of byte j*b/8
  *   sum        d_pad little-endian unsigned integers of acc_bits bits
  *   rotated    d_pad fp32 per worker: the RHT output before truncation (optional)
@@ -56,6 +61,7 @@ extern "C" {
 /* thc_status() bits */
 #define THC_STATUS_NONFINITE     1u  /* a block's norm was NaN/Inf: its scale was set to 0        */
 #define THC_STATUS_ZERO_BLOCK    2u  /* a block had scale 0 (all-zero input): indices 0, output 0 */
+                                     /* (exact range: a block whose range is [0, 0])              */
 #define THC_STATUS_WAIT_TIMEOUT  4u  /* an on-device wait gave up; the call's output is invalid   */
 
 typedef struct thc_ctx thc_ctx;   /* opaque */
