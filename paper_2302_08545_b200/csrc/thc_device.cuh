@@ -25,7 +25,7 @@ constexpr int kLutRep = 8;                     // lane replication of the quanti
 struct DeviceBlock {
     uint32_t status;             // THC_STATUS_* bits
     uint32_t pad_[31];
-    uint32_t counters[1024];     // scheduling counters (self-resetting), 128-byte aligned
+    uint32_t counters[5632];     // scheduling counters (self-resetting), 128-byte aligned
     uint4    lut[256];           // by floor(u*g): (-T[z0] as float, 65536/(T[z0+1]-T[z0]), z0, 0)
     uint32_t table[256];         // T
 };

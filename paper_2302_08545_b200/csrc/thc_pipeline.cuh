@@ -57,7 +57,7 @@ constexpr int kPChunks = kPElems / 4;
 constexpr int kPThreads = 128;                // compute threads of a CTA
 constexpr int kPCtaThreads = 160;             // plus one control warp that runs the queue
 constexpr int kPSignWords = 512;            // sign words: two slots of 256 (pass A) or one of 512
-constexpr int kMaxRing = 56;
+constexpr int kMaxRing = 320;                // ring slots: blocks of 2^15 need up to 280 to cover the tasks in flight
 constexpr int kBlockConstMax = 256;         // per-block constants cached in shared memory
 constexpr uint32_t kMaxPolls = 1u << 21;
 
