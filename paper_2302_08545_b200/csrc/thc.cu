@@ -567,32 +567,38 @@ prepare_partial_kernel(PtrArray in, uint64_t d, uint32_t chunk_log2, uint64_t ch
     const uint64_t j0 = chunk << chunk_log2;
     const int n4 = 1 << (chunk_log2 - 2);
     double s = 0.0;
-    for (int c = threadIdx.x; c < n4; c += kThreads) {
-        const uint64_t j = j0 + (uint64_t)c * 4;
-        if (j >= d) break;
-        float4 v;
-        if (BF16) {
-            const uint16_t *x = static_cast<const uint16_t *>(in.p[wl]);
-            uint32_t w0 = 0, w1 = 0;
-            if (j + 4 <= d) {
-                const uint2 q = __ldg(reinterpret_cast<const uint2 *>(x + j));
-                w0 = q.x; w1 = q.y;
+    if (BF16) {
+        // eight bf16 (16 bytes) per load
+        const uint16_t *x = static_cast<const uint16_t *>(in.p[wl]);
+        for (int c = threadIdx.x; c < n4 / 2; c += kThreads) {
+            const uint64_t j = j0 + (uint64_t)c * 8;
+            if (j >= d) break;
+            uint32_t w[4] = {0u, 0u, 0u, 0u};
+            if (j + 8 <= d) {
+                const uint4 q = __ldg(reinterpret_cast<const uint4 *>(x + j));
+                w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
             } else {
-                for (int e = 0; e < 4; ++e)
-                    if (j + e < d) {
-                        const uint32_t h = (uint32_t)__ldg(x + j + e) << ((e & 1) * 16);
-                        if (e < 2) w0 |= h; else w1 |= h;
-                    }
+                for (int e = 0; e < 8; ++e)
+                    if (j + e < d) w[e >> 1] |= (uint32_t)__ldg(x + j + e) << ((e & 1) * 16);
             }
-            v = make_float4(__uint_as_float(w0 << 16), __uint_as_float(w0 & 0xFFFF0000u),
-                            __uint_as_float(w1 << 16), __uint_as_float(w1 & 0xFFFF0000u));
-        } else {
-            v = load_f32x4_masked(static_cast<const float *>(in.p[wl]), j, d);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const double lo = (double)__uint_as_float(w[q] << 16);
+                const double hi = (double)__uint_as_float(w[q] & 0xFFFF0000u);
+                s = fma(lo, lo, s);
+                s = fma(hi, hi, s);
+            }
         }
-        s = fma((double)v.x, (double)v.x, s);
-        s = fma((double)v.y, (double)v.y, s);
-        s = fma((double)v.z, (double)v.z, s);
-        s = fma((double)v.w, (double)v.w, s);
+    } else {
+        for (int c = threadIdx.x; c < n4; c += kThreads) {
+            const uint64_t j = j0 + (uint64_t)c * 4;
+            if (j >= d) break;
+            const float4 v = load_f32x4_masked(static_cast<const float *>(in.p[wl]), j, d);
+            s = fma((double)v.x, (double)v.x, s);
+            s = fma((double)v.y, (double)v.y, s);
+            s = fma((double)v.z, (double)v.z, s);
+            s = fma((double)v.w, (double)v.w, s);
+        }
     }
     __shared__ double red[kThreads / 32];
     for (int off = 16; off > 0; off >>= 1) s += __shfl_down_sync(0xFFFFFFFFu, s, off);
