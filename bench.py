@@ -279,11 +279,16 @@ def run_gpu(args):
     clocks.mark_start()
     start.record(stream)
     for _ in range(args.steps):
-        step(events)
+        step()
     end.record(stream)
     torch.cuda.synchronize()
     clocks.mark_end()
     clocks.close()
+    # per-call times: a second pass with an event pair around every call (kept out of the
+    # timed region, where the extra records would sit between the launches)
+    for _ in range(min(args.steps, 50)):
+        step(events)
+    torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     ms_local = start.elapsed_time(end) / args.steps
@@ -312,6 +317,36 @@ def run_gpu(args):
         for name, a, b in split_events:
             acc.setdefault(name, []).append(a.elapsed_time(b))
         split_ms.update({k: float(np.mean(v)) for k, v in acc.items()})
+
+    # ---- the same step replayed as a CUDA graph (launch cost off the critical path; matters
+    # for the launch-bound small configurations)
+    graph_ms = None
+    try:
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            for _, fn in calls:
+                fn()
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _, fn in calls:
+                fn()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = max(10, min(args.steps, 100))
+        g0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        g1.record(stream)
+        torch.cuda.synchronize()
+        graph_ms = g0.elapsed_time(g1) / reps
+        del graph
+    except Exception as exc:                            # report, do not fail the benchmark
+        graph_ms = None
+        sys.stderr.write(f"graph replay skipped: {exc}\n")
 
     # ---- end to end: every step's gradients come from pinned host memory and its result goes
     # back to the host.  Steps are pipelined as a training loop would: two sets of device
@@ -435,6 +470,7 @@ def run_gpu(args):
         "gpu_launches": args.steps * sum(KERNELS_PER_STEP[name] for name, _ in calls),
         "roofline": roofline,
         "per_call_ms": per_call_ms,
+        "graph_replay_ms_per_step": graph_ms,
         "split_calls_ms": {k: split_ms[k] for k in ("prepare", "compress") if k in split_ms},
         "round_excl_prepare": {
             "ms": round_ms, "gradient_gbs": grad_bytes / (round_ms * 1e-3) / 1e9,
