@@ -33,7 +33,8 @@
  *   gradient   d elements, fp32 or bf16, contiguous; coordinates d..d_pad-1 count as zero
  *   scales     one fp32 M per block, nblocks = d_pad / B entries (THC_RANGE_MINMAX contexts:
  *              nblocks minima followed by nblocks maxima; thc_sizes_t.scales_count)
- *   packed     d_pad*b/8 bytes per worker; index j in bits [(j mod 8/b)*b, +b) of byte j*b/8
+ *   packed     d_pad*b/8 bytes per worker; index j in bits [j*b, j*b + b) of the little-endian bit
+ *              stream, i.e. bits [(j mod 8/b)*b, +b) of byte j*b/8 where b divides 8
  *   sum        d_pad little-endian unsigned integers of acc_bits bits
  *   rotated    d_pad fp32 per worker: the RHT output before truncation (optional)
  *   out        d fp32
@@ -68,7 +69,7 @@ typedef struct thc_ctx thc_ctx;   /* opaque */
 
 /*
  * Parameters of the method (Algorithm 3, "Input" line) plus the layout choices.
- *   bits         b in {1, 2, 4, 8}: bits per table index (Section 4.3)
+ *   bits         b in {1, 2, 3, 4, 8}: bits per table index (Section 4.3)
  *   granularity  g with 2^b - 1 <= g <= 255 (Section 4.3, "granularity")
  *   table        T[0 .. 2^b - 1], 0 = T[0] < T[1] < ... < T[2^b - 1] = g (Section 4.3);
  *                the identity table with g = 2^b - 1 is Uniform THC (Section 4.2)

@@ -295,24 +295,37 @@ void thc_oracle_quantize_at(const float *r, uint64_t d_pad, uint32_t k, const fl
     free(lo);
 }
 
-/* Bit-packing (Section 3; reading R7). packed has d_pad*b/8 bytes. */
+/* Bit-packing (Section 3; reading R7): index j occupies bits [j*b, j*b + b) of a little-endian
+ * bit stream, i.e. for b dividing 8 bits [(j mod 8/b)*b, +b) of byte j*b/8; for b = 3 an index
+ * may straddle two bytes.  packed has d_pad*b/8 bytes (d_pad is a multiple of 8). */
+static void put_index(uint8_t *packed, uint64_t j, uint32_t b, uint32_t z)
+{
+    for (uint32_t t = 0; t < b; ++t) {
+        uint64_t bit = j * b + t;
+        if ((z >> t) & 1u) packed[bit >> 3] |= (uint8_t)(1u << (bit & 7));
+    }
+}
+
+static uint32_t get_index(const uint8_t *packed, uint64_t j, uint32_t b)
+{
+    uint32_t z = 0;
+    for (uint32_t t = 0; t < b; ++t) {
+        uint64_t bit = j * b + t;
+        z |= (uint32_t)((packed[bit >> 3] >> (bit & 7)) & 1u) << t;
+    }
+    return z;
+}
+
 void thc_oracle_pack(const uint8_t *z, uint64_t d_pad, uint32_t b, uint8_t *packed)
 {
     uint64_t nbytes = d_pad * b / 8;
     memset(packed, 0, nbytes);
-    uint32_t per_byte = 8 / b;
-    for (uint64_t j = 0; j < d_pad; ++j) {
-        packed[j / per_byte] |= (uint8_t)(z[j] << ((j % per_byte) * b));
-    }
+    for (uint64_t j = 0; j < d_pad; ++j) put_index(packed, j, b, z[j]);
 }
 
 void thc_oracle_unpack(const uint8_t *packed, uint64_t d_pad, uint32_t b, uint8_t *z)
 {
-    uint32_t per_byte = 8 / b;
-    uint32_t mask = (1u << b) - 1u;
-    for (uint64_t j = 0; j < d_pad; ++j) {
-        z[j] = (uint8_t)((packed[j / per_byte] >> ((j % per_byte) * b)) & mask);
-    }
+    for (uint64_t j = 0; j < d_pad; ++j) z[j] = (uint8_t)get_index(packed, j, b);
 }
 
 /* ------------------------------------------------------------------------------------
@@ -324,15 +337,9 @@ void thc_oracle_aggregate(const uint8_t *packed, uint32_t n, uint64_t d_pad, uin
                           const uint16_t *table, uint32_t w, void *sum)
 {
     uint64_t stride = d_pad * b / 8;
-    uint32_t per_byte = 8 / b;
-    uint32_t mask = (1u << b) - 1u;
     for (uint64_t j = 0; j < d_pad; ++j) {
         uint32_t y = 0;
-        for (uint32_t i = 0; i < n; ++i) {
-            uint8_t byte = packed[(uint64_t)i * stride + j / per_byte];
-            uint32_t zi = (byte >> ((j % per_byte) * b)) & mask;
-            y += table[zi];
-        }
+        for (uint32_t i = 0; i < n; ++i) y += table[get_index(packed + (uint64_t)i * stride, j, b)];
         if (w == 8) ((uint8_t *)sum)[j] = (uint8_t)y;
         else if (w == 16) ((uint16_t *)sum)[j] = (uint16_t)y;
         else ((uint32_t *)sum)[j] = y;

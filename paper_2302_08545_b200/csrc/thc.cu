@@ -104,6 +104,15 @@ __device__ __forceinline__ float4 load_f32x4_masked(const float *x, uint64_t j, 
     return v;
 }
 
+// Eight 3-bit indices (24 bits, coordinate 0 in the low bits) go to bytes 3 (j/8) .. +2.
+__device__ __forceinline__ void store_packed3(unsigned char *pk, uint64_t j, uint32_t z)
+{
+    unsigned char *p = pk + 3 * (j >> 3);
+    p[0] = (unsigned char)z;
+    p[1] = (unsigned char)(z >> 8);
+    p[2] = (unsigned char)(z >> 16);
+}
+
 __device__ __forceinline__ float sum_to_float(uint32_t y)   // exact for y < 2^23
 {
     return __uint_as_float(0x4B000000u | y) - 8388608.0f;
@@ -253,6 +262,7 @@ rht_tile_kernel(TileGeom g, PtrArray in, MutPtrArray out, MutPtrArray rotated,
             const uint64_t z = quantize8<BITS, IDENTITY>(r, bc.x, bc.y, gf, rnd, my_lut, kLutRep);
             if constexpr (BITS == 8) *reinterpret_cast<uint2 *>(pk + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
             else if constexpr (BITS == 4) *reinterpret_cast<uint32_t *>(pk + j / 2) = (uint32_t)z;
+            else if constexpr (BITS == 3) store_packed3(pk, j, (uint32_t)z);
             else if constexpr (BITS == 2) *reinterpret_cast<uint16_t *>(pk + j / 4) = (uint16_t)z;
             else pk[j / 8] = (unsigned char)z;
         }
@@ -339,6 +349,7 @@ quantize_rotated_kernel(PtrArray rotated, MutPtrArray packed, uint64_t d_pad, ui
         const uint64_t z = quantize8<BITS, IDENTITY>(r, kappa, offset, gf, rnd, my_lut, kLutRep);
         if constexpr (BITS == 8) *reinterpret_cast<uint2 *>(pk + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
         else if constexpr (BITS == 4) *reinterpret_cast<uint32_t *>(pk + j / 2) = (uint32_t)z;
+        else if constexpr (BITS == 3) store_packed3(pk, j, (uint32_t)z);
         else if constexpr (BITS == 2) *reinterpret_cast<uint16_t *>(pk + j / 4) = (uint16_t)z;
         else pk[j / 8] = (unsigned char)z;
     }
@@ -686,8 +697,11 @@ aggregate_kernel(PtrArray in, uint32_t n, uint64_t units, uint64_t d_pad, const 
         for (uint64_t j = units * 32; j < d_pad; ++j) {
             uint32_t acc = 0;
             for (uint32_t i = 0; i < n; ++i) {
-                const unsigned char byte = static_cast<const unsigned char *>(in.p[i])[j * BITS / 8];
-                acc += T[(byte >> ((j % (8 / BITS)) * BITS)) & ((1u << BITS) - 1u)];
+                const unsigned char *pb = static_cast<const unsigned char *>(in.p[i]);
+                const uint64_t bit = j * BITS;
+                uint32_t two = pb[bit >> 3];
+                if (((bit & 7) + BITS) > 8) two |= (uint32_t)pb[(bit >> 3) + 1] << 8;
+                acc += T[(two >> (bit & 7)) & ((1u << BITS) - 1u)];
             }
             if constexpr (W == 8) sum[j] = (unsigned char)acc;
             else if constexpr (W == 16) reinterpret_cast<uint16_t *>(sum)[j] = (uint16_t)acc;
@@ -712,6 +726,8 @@ aggregate_kernel(PtrArray in, uint32_t n, uint64_t units, uint64_t d_pad, const 
             } else if constexpr (BITS == 4) {
                 const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src));
                 w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w;
+            } else if constexpr (BITS == 3) {
+                w[0] = __ldg(src); w[1] = __ldg(src + 1); w[2] = __ldg(src + 2);
             } else if constexpr (BITS == 2) {
                 const uint2 a = __ldg(reinterpret_cast<const uint2 *>(src));
                 w[0] = a.x; w[1] = a.y;
@@ -721,7 +737,9 @@ aggregate_kernel(PtrArray in, uint32_t n, uint64_t units, uint64_t d_pad, const 
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
                 const int bit = e * BITS;
-                const uint32_t z = (w[bit >> 5] >> (bit & 31)) & ((1u << BITS) - 1u);
+                // a 3-bit index may straddle two words: funnel shift over the pair
+                const uint32_t lo = w[bit >> 5], hi = w[((bit >> 5) + 1) < kInWords ? (bit >> 5) + 1 : (bit >> 5)];
+                const uint32_t z = __funnelshift_r(lo, hi, bit & 31) & ((1u << BITS) - 1u);
                 acc[e] += T[z];
             }
         }
@@ -807,7 +825,7 @@ const char *thc_strerror(int code)
 static int validate_config(const thc_config *c, uint32_t *acc_bits, bool *identity)
 {
     if (c == nullptr) return THC_EINVAL;
-    if (!(c->bits == 1 || c->bits == 2 || c->bits == 4 || c->bits == 8)) return THC_EINVAL;
+    if (!(c->bits == 1 || c->bits == 2 || c->bits == 3 || c->bits == 4 || c->bits == 8)) return THC_EINVAL;
     const uint32_t levels = 1u << c->bits;
     if (c->granularity < levels - 1) return THC_EINVAL;
     if (c->granularity > 255) return THC_EUNSUPPORTED;
@@ -1056,6 +1074,7 @@ static tile_kernel_t pick_tile_kernel(uint32_t bits, bool identity)
     switch (bits) {
     case 1: return identity ? rht_tile_kernel<LOAD, STORE, 1, true> : rht_tile_kernel<LOAD, STORE, 1, false>;
     case 2: return identity ? rht_tile_kernel<LOAD, STORE, 2, true> : rht_tile_kernel<LOAD, STORE, 2, false>;
+    case 3: return identity ? rht_tile_kernel<LOAD, STORE, 3, true> : rht_tile_kernel<LOAD, STORE, 3, false>;
     case 4: return identity ? rht_tile_kernel<LOAD, STORE, 4, true> : rht_tile_kernel<LOAD, STORE, 4, false>;
     default: return identity ? rht_tile_kernel<LOAD, STORE, 8, true> : rht_tile_kernel<LOAD, STORE, 8, false>;
     }
@@ -1143,6 +1162,7 @@ static pipe_kernel_t pick_pipe_kernel_kb(uint32_t bits, bool identity)
         switch (bits) {
         case 1: return thc_pipeline_kernel<MODE, 1, true, KB>;
         case 2: return thc_pipeline_kernel<MODE, 2, true, KB>;
+        case 3: return thc_pipeline_kernel<MODE, 3, true, KB>;
         case 4: return thc_pipeline_kernel<MODE, 4, true, KB>;
         default: return thc_pipeline_kernel<MODE, 8, true, KB>;
         }
@@ -1152,6 +1172,7 @@ static pipe_kernel_t pick_pipe_kernel_kb(uint32_t bits, bool identity)
         switch (bits) {
         case 1: return identity ? thc_pipeline_kernel<MODE, 1, true, KB> : thc_pipeline_kernel<MODE, 1, false, KB>;
         case 2: return identity ? thc_pipeline_kernel<MODE, 2, true, KB> : thc_pipeline_kernel<MODE, 2, false, KB>;
+        case 3: return identity ? thc_pipeline_kernel<MODE, 3, true, KB> : thc_pipeline_kernel<MODE, 3, false, KB>;
         case 4: return identity ? thc_pipeline_kernel<MODE, 4, true, KB> : thc_pipeline_kernel<MODE, 4, false, KB>;
         default: return identity ? thc_pipeline_kernel<MODE, 8, true, KB> : thc_pipeline_kernel<MODE, 8, false, KB>;
         }
@@ -1532,6 +1553,7 @@ int thc_quantize_rotated(thc_ctx *ctx, const float *const *rotated, uint32_t n_l
     switch (ctx->cfg.bits) {
     case 1: if (ctx->identity) THC_QR(1, true); else THC_QR(1, false); break;
     case 2: if (ctx->identity) THC_QR(2, true); else THC_QR(2, false); break;
+    case 3: if (ctx->identity) THC_QR(3, true); else THC_QR(3, false); break;
     case 4: if (ctx->identity) THC_QR(4, true); else THC_QR(4, false); break;
     default: if (ctx->identity) THC_QR(8, true); else THC_QR(8, false); break;
     }
@@ -1613,6 +1635,7 @@ int thc_aggregate(thc_ctx *ctx, const void *const *packed, uint32_t n, uint64_t 
     switch (ctx->cfg.bits) {
     case 1: THC_AGW(1); break;
     case 2: THC_AGW(2); break;
+    case 3: THC_AGW(3); break;
     case 4: THC_AGW(4); break;
     default: THC_AGW(8); break;
     }

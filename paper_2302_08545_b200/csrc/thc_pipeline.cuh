@@ -511,6 +511,10 @@ __device__ __forceinline__ void pass_a_round1_inverse(float4 *tile, const unsign
                 const uint4 t4 = __ldg(reinterpret_cast<const uint4 *>(p) + q);
                 w[4 * q] = t4.x; w[4 * q + 1] = t4.y; w[4 * q + 2] = t4.z; w[4 * q + 3] = t4.w;
             }
+        } else if constexpr (IN_BITS == 3) {
+            w[0] = __ldg(reinterpret_cast<const uint32_t *>(p));
+            w[1] = __ldg(reinterpret_cast<const uint32_t *>(p) + 1);
+            w[2] = __ldg(reinterpret_cast<const uint32_t *>(p) + 2);
         } else if constexpr (IN_BITS == 2) {
             const uint2 t2 = __ldg(reinterpret_cast<const uint2 *>(p));
             w[0] = t2.x; w[1] = t2.y;
@@ -523,8 +527,9 @@ __device__ __forceinline__ void pass_a_round1_inverse(float4 *tile, const unsign
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int bit = (m * 4 + e) * IN_BITS;
+                const uint32_t nxt = w[((bit >> 5) + 1) < IN_BITS ? (bit >> 5) + 1 : (bit >> 5)];
                 const uint32_t val = IN_BITS == 32 ? w[bit >> 5]
-                                                   : (w[bit >> 5] >> (bit & 31)) & ((1u << (IN_BITS & 31)) - 1u);
+                                     : __funnelshift_r(w[bit >> 5], nxt, bit & 31) & ((1u << (IN_BITS & 31)) - 1u);
                 float yf;
                 if (MODE == kErrorFeedback) yf = ft[val * FREP];
                 else if (MODE == kDecompress32) yf = (float)val;
@@ -643,6 +648,8 @@ __device__ __forceinline__ void epilogue_unit(const float4 &va, const float4 &vb
             *reinterpret_cast<uint2 *>(ep.packed + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
         else if constexpr (BITS == 4)
             *reinterpret_cast<uint32_t *>(ep.packed + j / 2) = (uint32_t)z;
+        else if constexpr (BITS == 3)
+            store_packed3(ep.packed, j, (uint32_t)z);
         else if constexpr (BITS == 2)
             *reinterpret_cast<uint16_t *>(ep.packed + j / 4) = (uint16_t)z;
         else

@@ -7,9 +7,8 @@ paper's training gradients.
 
 Every point builds the optimal lookup table for (b, g, p) with the solver of tables.py
 (Section 5.2), runs one full round of the library on the GPU (scales, compress, aggregate,
-decompress) and reports  NMSE = ||out - mean_i x_i||^2 / ||mean_i x_i||^2.  Index widths are
-those the packing supports (1, 2, 4, 8 bits; the paper's 3-bit curve has no counterpart).
-One JSON line per point.
+decompress) and reports  NMSE = ||out - mean_i x_i||^2 / ||mean_i x_i||^2 for 2, 3 and 4 bits
+per index (the paper's three curves).  One JSON line per point.
 """
 from __future__ import annotations
 
@@ -19,7 +18,7 @@ import json
 from . import tables
 from .workloads import Workload
 
-DEFAULT_POINTS = {2: (3, 4, 5, 6, 8, 10), 4: (15, 18, 22, 26, 30, 36, 44, 52)}
+DEFAULT_POINTS = {2: (3, 4, 5, 6, 8, 10), 3: (7, 8, 10, 12, 14, 18, 22), 4: (15, 18, 22, 26, 30, 36, 44, 52)}
 
 
 def lognormal_gradients(n: int, d: int, seed: int, device):

@@ -41,7 +41,7 @@ def test_sizes_match_the_paper_prototype_ratios():
 
 
 @pytest.mark.parametrize("kw", [
-    dict(bits=3), dict(bits=0), dict(granularity=14), dict(table=(1,) + T4_30[1:]),
+    dict(bits=5), dict(bits=0), dict(granularity=14), dict(table=(1,) + T4_30[1:]),
     dict(table=T4_30[:-1] + (29,)), dict(table=(0, 3, 3) + T4_30[3:]), dict(t_p=0.0),
     dict(t_p=float("nan")), dict(log2_block=2), dict(log2_block=23), dict(in_dtype=7),
     dict(workers=0), dict(workers=65), dict(acc_bits=12), dict(workers=9, acc_bits=8),

@@ -11,13 +11,16 @@ pytestmark = pytest.mark.gpu
 
 def test_nmse_falls_with_granularity_and_by_much_more_with_bits():
     from paper_2302_08545_b200 import nmse_experiment as E
-    rows = E.run({2: (3, 6, 10), 4: (15, 30, 52)}, log2_d=21, workers=10)
+    rows = E.run({2: (3, 6, 10), 3: (7, 14), 4: (15, 30, 52)}, log2_d=21, workers=10)
     nm = {(r["bits"], r["granularity"]): r["nmse"] for r in rows}
     # more grid points for the same number of bits: no worse (optimal tables nest in quality)
     assert nm[(2, 6)] <= nm[(2, 3)] * 1.02 and nm[(2, 10)] <= nm[(2, 6)] * 1.02
     assert nm[(4, 30)] <= nm[(4, 15)] * 1.02 and nm[(4, 52)] <= nm[(4, 30)] * 1.02
     # two more bits: far more than the gain from granularity (the paper: about 10x per bit)
     assert min(nm[(4, g)] for g in (15, 30, 52)) < 0.05 * min(nm[(2, g)] for g in (3, 6, 10))
+    # three bits sit in between, each bit worth a large factor
+    best = {b: min(v for (bb, _), v in nm.items() if bb == b) for b in (2, 3, 4)}
+    assert best[4] < 0.5 * best[3] < 0.25 * best[2]
     assert all(0.0 < v < 1.0 for v in nm.values())
 
 

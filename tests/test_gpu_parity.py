@@ -117,6 +117,7 @@ def test_two_pass_blocks(k, d, n):
 
 @pytest.mark.parametrize("bits,g,table", [
     (1, 1, (0, 1)), (1, 30, (0, 30)), (2, 3, (0, 1, 2, 3)), (2, 4, (0, 1, 3, 4)),
+    (3, 7, tuple(range(8))), (3, 12, (0, 2, 4, 5, 6, 7, 9, 12)),
     (4, 15, tuple(range(16))), (4, 30, T4_30), (8, 255, tuple(range(256))),
     (4, 200, tuple(int(round(v)) for v in np.linspace(0, 200, 16))),
 ])
@@ -366,7 +367,7 @@ def test_prepare_compress_falls_back_where_the_fused_kernel_does_not_apply():
             assert np.array_equal(r.packed[i].cpu().numpy(), p0[i])
 
 
-@pytest.mark.parametrize("bits,g", [(1, 1), (2, 3), (8, 255)])
+@pytest.mark.parametrize("bits,g", [(1, 1), (2, 3), (3, 7), (8, 255)])
 def test_error_feedback_other_index_widths(bits, g):
     """The one-launch error-feedback path unpacks 1-, 2- and 8-bit indices as well."""
     import torch
@@ -530,6 +531,7 @@ def test_step_can_be_captured_in_a_cuda_graph_and_replayed():
     (1, 1, (0, 1), 5), (1, 200, (0, 200), 1), (1, 3, (0, 3), 64), (2, 3, (0, 1, 2, 3), 64),
     (4, 30, T4_30, 17), (4, 30, T4_30, 64), (4, 15, tuple(range(16)), 64), (4, 127, tuple(range(15)) + (127,), 3),
     (8, 255, tuple(range(256)), 7), (8, 255, tuple(range(256)), 64),
+    (3, 7, tuple(range(8)), 9), (3, 20, (0, 1, 5, 8, 10, 13, 17, 20), 13), (3, 60, (0, 9, 17, 26, 30, 41, 50, 60), 64),
 ])
 def test_aggregate_fast_paths_on_random_indices(bits, g, table, n):
     """The byte-lane (SWAR) aggregation kernels against the oracle's plain loop on uniformly

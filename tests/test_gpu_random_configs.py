@@ -18,7 +18,7 @@ def _random_case(rng):
         nblk = int(rng.integers(1, 3))
     d = (nblk - 1) * B + int(rng.integers(1, B + 1))
     n = int(rng.integers(1, 10 if k <= 18 else 4))
-    bits = int(rng.choice([1, 2, 4, 8]))
+    bits = int(rng.choice([1, 2, 3, 4, 8]))
     levels = 1 << bits
     if rng.random() < 0.4:
         g = levels - 1

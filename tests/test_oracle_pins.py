@@ -382,9 +382,10 @@ def test_quantizer_edges_and_degenerate_blocks():
 
 
 # ------------------------------------------------------------------- pack / aggregate
-@pytest.mark.parametrize("bits", [1, 2, 4, 8])
+@pytest.mark.parametrize("bits", [1, 2, 3, 4, 8])
 def test_pack_layout_brute_force(bits):
-    """Index j sits at bit offset (j mod 8/b)*b of byte j*b/8."""
+    """Index j sits at bits [j*b, j*b+b) of the little-endian bit stream: for b dividing 8 at
+    bit offset (j mod 8/b)*b of byte j*b/8; three-bit indices straddle bytes."""
     per = 8 // bits
     d_pad = 64
     rng = np.random.default_rng(bits)
@@ -395,7 +396,12 @@ def test_pack_layout_brute_force(bits):
     for j in range(d_pad):
         val = sum(int(bitstream[j * bits + t]) << t for t in range(bits))
         assert val == z[j]
-        assert (int(packed[j // per]) >> ((j % per) * bits)) & ((1 << bits) - 1) == z[j]
+        if 8 % bits == 0:
+            assert (int(packed[j // per]) >> ((j % per) * bits)) & ((1 << bits) - 1) == z[j]
+    if bits == 3:                                        # eight indices are one 24-bit integer
+        for u in range(d_pad // 8):
+            word = int(packed[3 * u]) | int(packed[3 * u + 1]) << 8 | int(packed[3 * u + 2]) << 16
+            assert word == sum(int(z[8 * u + e]) << (3 * e) for e in range(8))
     assert np.array_equal(O.unpack(packed, d_pad, bits), z)
 
 
