@@ -718,3 +718,77 @@ def test_exact_range_constant_block_decodes_to_the_constant():
     z = O.unpack(out["packed"][0], 48, 4)
     assert not z[16:48].any()
     assert out["out"][16] == np.float32(3.25) and not out["out"][17:].any()
+
+
+# -------------------------------------- error feedback on a general (asymmetric) range [m, M]
+def _dense_inverse_rht(v, d, c, rnd):
+    """D (1/sqrt B) H v per block, written out with SciPy's dense Sylvester matrix in float64."""
+    B = c.block
+    H = hadamard(B).astype(np.float64)
+    out = np.zeros(v.size)
+    for blk in range(v.size // B):
+        s = O.signs(c.seed, rnd, blk * B, B).astype(np.float64)
+        out[blk * B:(blk + 1) * B] = s * (H @ v[blk * B:(blk + 1) * B]) / np.sqrt(B)
+    return out[:d]
+
+
+def test_error_feedback_on_an_asymmetric_range_follows_algorithm_2s_estimate_line():
+    """Algorithm 3's e_i = x_i - RHT^-1(X_i) with Algorithm 2's quantisation values on [m, M]:
+    X[j] = m + T[z[j]] (M - m)/g.  The range here is the exact, asymmetric one (m != -M) and
+    differs per block.  Checked three ways: bit for bit against x minus the decompression of
+    the worker's own one-worker aggregate with divisor 1 on the same range; against the
+    formula written out densely in float64 (a step of 2M/g or a base of -M instead of m is
+    off by a sizeable fraction of the range and fails); and by the size of the residual."""
+    k, d, rnd = 6, 150, 7                                  # three blocks of 64, the last ragged
+    c = cfg(k=k)
+    rng = np.random.default_rng(41)
+    x = (rng.standard_normal((2, d)) + 0.6 * rng.standard_normal((2, 1))).astype(np.float32)
+    x[:, 70] += 9.0                                       # one-sided outlier: a lopsided range
+    lo, hi = O.ranges(x, c, rnd)
+    assert np.all(np.abs(lo + hi) > 0.05 * (hi - lo))      # really asymmetric, every block
+    T = np.array(T4_30, np.float64)
+    B = 1 << k
+    for i in range(2):
+        z = O.quantize(O.rht_forward(x[i], c, rnd), hi, c, rnd, i, lo=lo)
+        e = O.error_feedback(x[i], z, hi, c, rnd, lo=lo)
+        one = O.aggregate(O.pack(z, 4)[None, :], c.d_pad(d), c, 8)
+        back = O.decompress(one, 1, d, hi, c, rnd, lo=lo)
+        assert np.array_equal(e.view(np.uint32), (x[i] - back).view(np.uint32))
+        m = np.repeat(lo.astype(np.float64), B)
+        M = np.repeat(hi.astype(np.float64), B)
+        X = m + T[z] * (M - m) / 30.0
+        dense = x[i].astype(np.float64) - _dense_inverse_rht(X, d, c, rnd)
+        width = float((hi - lo).max())
+        assert np.abs(e - dense).max() <= 2e-6 * width
+        # the two plausible slips are far outside that tolerance
+        wrong_step = x[i].astype(np.float64) - _dense_inverse_rht(m + T[z] * (2.0 * M) / 30.0, d, c, rnd)
+        wrong_base = x[i].astype(np.float64) - _dense_inverse_rht(-M + T[z] * (M - m) / 30.0, d, c, rnd)
+        assert np.abs(e - wrong_step).max() > 1e-2 * width
+        assert np.abs(e - wrong_base).max() > 1e-2 * width
+        # nothing is clamped on the exact range, so the residual is quantisation noise only:
+        # per rotated coordinate at most (gap/g)^2 (M-m)^2 / 4, gap <= 3 of g = 30
+        nmse_bound = ((3.0 / 30.0) ** 2 / 4.0) * (width ** 2) * c.d_pad(d)
+        assert (e.astype(np.float64) ** 2).sum() <= nmse_bound
+
+
+def test_error_feedback_telescopes_over_rounds_on_the_exact_range():
+    """Algorithm 3 with the exact range of Algorithm 1's preliminary stage: x^r = grad + e^r,
+    e^{r+1} = x^r - RHT^-1(X^r), so sum_r RHT^-1(X^r) = R grad - e^R; nothing is truncated, so
+    e stays at quantisation-noise size and the running mean converges to grad."""
+    k, d, R = 6, 128, 40
+    c = cfg(k=k)
+    rng = np.random.default_rng(43)
+    grad = (rng.standard_normal(d) + 0.8).astype(np.float32)   # a mean offset: m != -M in block 0
+    e = np.zeros(d, np.float32)
+    sent = np.zeros(d)
+    for r in range(R):
+        x = (grad + e).astype(np.float32)
+        lo, hi = O.ranges(x[None, :], c, r)
+        z = O.quantize(O.rht_forward(x, c, r), hi, c, r, 0, lo=lo)
+        one = O.aggregate(O.pack(z, 4)[None, :], d, c, 8)
+        sent += O.decompress(one, 1, d, hi, c, r, lo=lo)
+        e = O.error_feedback(x, z, hi, c, r, lo=lo)
+    g64 = grad.astype(np.float64)
+    assert np.allclose(sent, R * g64 - e, atol=2e-5 * R)
+    assert np.linalg.norm(e) < 0.5 * np.linalg.norm(g64)
+    assert np.linalg.norm(sent / R - g64) < 0.02 * np.linalg.norm(g64)
