@@ -39,8 +39,8 @@
  *       <g+1> is the real number u*g, which is never rounded on its own.
  *   R6  Rounding decision: z0 = the largest index <= 2^b - 2 with T[z0] <= floor(u*g)
  *       (capped so that u = 1 falls in the last interval); delta = fma(u, g, -T[z0]);
- *       up iff u16 < RN(2^16 * delta / (T[z0+1] - T[z0])), the product taken as one fused
- *       multiply-add of delta with R16[z0] = 65536 / (T[z0+1]-T[z0]).
+ *       up iff u16 < RN(delta * R16[z0]) with R16[z0] = (float)(65536 / (T[z0+1]-T[z0])):
+ *       the exact product rounded once to the nearest integer, ties to even.
  *       So P(up) is the paper's (a - q0)/(q1 - q0) rounded to a multiple of 2^-16.
  *   R7  Packing: index j occupies bits [(j mod 8/b) * b, +b) of byte j*b/8; sums are
  *       little-endian unsigned w-bit integers in coordinate order.
@@ -269,8 +269,9 @@ void thc_oracle_quantize_range_at(const float *r, uint64_t d_pad, uint32_t k, co
         float gap = (float)((int)table[z0 + 1] - (int)table[z0]);
         float r16 = 65536.0f / gap;
         float delta = fmaf(pos, (float)g, -(float)table[z0]);
-        float tau = fmaf(delta, r16, 8388608.0f);                         /* RN to integer */
-        uint32_t threshold = (uint32_t)(tau - 8388608.0f);
+        /* RN(delta * r16) to an integer, ties to even: the product of two fp32 numbers is
+         * exact in double (24 + 24 bits) and rint() rounds it once */
+        uint32_t threshold = (uint32_t)rint((double)delta * (double)r16);
         uint32_t u = thc_oracle_u16(seed, round, worker, j_base + j);
         z[j] = (uint8_t)(z0 + (u < threshold ? 1u : 0u));
     }

@@ -792,3 +792,63 @@ def test_error_feedback_telescopes_over_rounds_on_the_exact_range():
     assert np.allclose(sent, R * g64 - e, atol=2e-5 * R)
     assert np.linalg.norm(e) < 0.5 * np.linalg.norm(g64)
     assert np.linalg.norm(sent / R - g64) < 0.02 * np.linalg.norm(g64)
+
+
+# ------------------------------------------------ the rounding threshold, in exact arithmetic
+def _rn32(q):
+    """Nearest fp32 (ties to even) of a positive rational, as a Fraction (normal range)."""
+    q = Fraction(q)
+    e = 0
+    while q / Fraction(2) ** e >= 1 << 24:
+        e += 1
+    while q / Fraction(2) ** e < 1 << 23:
+        e -= 1
+    scaled = q / Fraction(2) ** e
+    m = scaled.numerator // scaled.denominator
+    rem = scaled - m
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and m % 2 == 1):
+        m += 1
+    return Fraction(m) * Fraction(2) ** e
+
+
+def test_rounding_threshold_is_the_probability_of_section_4_1_in_sixteen_bits():
+    """Section 4.1: a in [q0, q1] goes up with probability (a - q0)/(q1 - q0).  For every
+    coordinate the oracle rounds up exactly for the 16-bit variates below a threshold; over
+    many workers (independent variates, same rotated value) the largest variate that went up
+    and the smallest that did not bracket that threshold.  The bracket must contain
+    RN(2^16 delta / gap) evaluated in exact rational arithmetic from the fp32 inputs
+    (position u = RN(r/(2M) + 1/2), delta = RN(u g - T[z0]), R16 = RN(65536/gap))."""
+    k, g = 6, 30
+    c = cfg(k=k)
+    rng = np.random.default_rng(47)
+    r = (rng.standard_normal(64) * 0.4).astype(np.float32)
+    M = np.array([1.0], np.float32)                      # kappa = 1/2, offset = 1/2: both exact
+    workers = 6000
+    zs = np.stack([O.quantize(r, M, c, rnd=9, worker=w) for w in range(workers)])
+    us = np.array([[O.u16(c.seed, 9, w, j) for j in range(64)] for w in range(0, workers, 60)])
+    T = T4_30
+    checked = 0
+    for j in range(64):
+        u = _rn32(Fraction(float(r[j])) / 2 + Fraction(1, 2)) if r[j] > -1.0 else Fraction(0)
+        u = min(max(u, Fraction(0)), Fraction(1))
+        f = min(int(u * g), g - 1)
+        z0 = max(z for z in range(15) if T[z] <= f)
+        gap = T[z0 + 1] - T[z0]
+        exact = u * g - T[z0]
+        delta = _rn32(exact) if exact > 0 else Fraction(0)
+        r16 = _rn32(Fraction(65536, gap))
+        prod = delta * r16
+        thr = prod.numerator // prod.denominator
+        rem = prod - thr
+        if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and thr % 2 == 1):
+            thr += 1
+        assert set(np.unique(zs[:, j])) <= {z0, z0 + 1}
+        # every sampled worker's decision agrees with u16 < thr
+        for row, w in enumerate(range(0, workers, 60)):
+            assert (zs[w, j] == z0 + 1) == (us[row, j] < thr)
+            checked += 1
+        # and the up-frequency over all workers is thr / 65536 within sampling error
+        freq = (zs[:, j] == z0 + 1).mean()
+        p = thr / 65536.0
+        assert abs(freq - p) <= 4.5 * np.sqrt(max(p * (1 - p), 1e-4) / workers)
+    assert checked == 64 * 100
