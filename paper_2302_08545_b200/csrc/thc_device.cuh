@@ -19,7 +19,6 @@ constexpr int kTileElems = 1 << kTileLog2;
 constexpr int kTileChunks = kTileElems / 4;    // 16-byte chunks
 constexpr int kThreads = 256;
 constexpr int kSignWordsMax = 1024;            // sign words a tile can need
-constexpr int kLutRep = 8;                     // lane replication of the quantiser table
 
 // Lives in the context's device block.
 struct DeviceBlock {
@@ -213,6 +212,42 @@ __device__ __forceinline__ void fwht_rounds(float4 *tile, int lo, int hi, int ti
 }
 
 // --------------------------------------------------------------------------- quantiser
+// The quantiser's table in shared memory, indexed by f = floor(u g): what the rounding rule
+// needs about the table interval [T[z0], T[z0+1]] that holds f.  Consecutive entries are 128
+// bytes apart and every entry is replicated over lanes so that a warp's look-ups (random f per
+// lane) never meet in a bank:
+//   indices of up to 4 bits   16 copies of 8 bytes   (R16 = 65536 / gap as fp32,
+//                                                     bf16(-T[z0]) << 16 | z0: table values up to
+//                                                     255 are exact in bf16)
+//   8-bit indices              8 copies of 16 bytes  (-T[z0] as fp32, R16, z0, 0)
+constexpr int kLutEntryBytes = 128;
+
+template <int BITS, bool IDENTITY>
+struct LutKind { static constexpr bool k8 = !IDENTITY && BITS <= 4; };
+
+template <bool LUT8>
+__device__ __forceinline__ void lut_fill(unsigned char *lut, const DeviceBlock *dev, uint32_t g, int tid, int nthreads)
+{
+    if (LUT8) {
+        for (int idx = tid; idx < (int)(g + 1) * 16; idx += nthreads) {
+            const uint4 e = dev->lut[idx / 16];
+            reinterpret_cast<uint2 *>(lut)[idx] = make_uint2(e.y, (e.x & 0xFFFF0000u) | e.z);
+        }
+    } else {
+        for (int idx = tid; idx < (int)(g + 1) * 8; idx += nthreads)
+            reinterpret_cast<uint4 *>(lut)[idx] = dev->lut[idx / 8];
+    }
+}
+
+// Shared-space byte address of this lane's copy of entry 0, minus 0x4B000000 * 128: the bits of
+// the float 2^23 + f, times 128, plus this value is the address of entry f.
+template <bool LUT8>
+__device__ __forceinline__ uint32_t lut_lane_addr(const unsigned char *lut, int lane)
+{
+    const uint32_t copy = LUT8 ? (uint32_t)(lane & 15) * 8u : (uint32_t)(lane & 7) * 16u;
+    return (uint32_t)__cvta_generic_to_shared(lut) + copy - 0x4B000000u * (uint32_t)kLutEntryBytes;
+}
+
 // Stochastic quantisation of eight consecutive rotated coordinates to table indices
 // (Algorithm 2, worker lines; Section 4.1 for the rounding rule):
 //   u = sat(fma(r, kappa, offset))          position in [m, M] on the unit interval, truncated
@@ -220,45 +255,56 @@ __device__ __forceinline__ void fwht_rounds(float4 *tile, int lo, int hi, int ti
 //   z0 = index of the table value at or below u*g, delta = fma(u, g, -T[z0])
 //   up iff u16 < RN(2^16 delta / gap)        (one fma onto 2^23, integer compare)
 // kappa = 1/(2M) and offset = 1/2; kappa = offset = 0 encodes a degenerate block (index 0).
-// `lut` points at this lane's copy of the (-T[z0], 65536/gap, z0) entries, `lut_stride`
-// entries apart per floor value.  Returns the indices packed BITS apiece, coordinate 0 in
-// the low bits.
+// `lut_addr` comes from lut_lane_addr (unused for the identity table).  Returns the indices
+// packed BITS apiece, coordinate 0 in the low bits.
 template <int BITS, bool IDENTITY>
 __device__ __forceinline__ uint64_t quantize8(const float (&r)[8], float kappa, float offset,
-                                              float gf, uint4 rnd, const uint4 *lut,
-                                              int lut_stride)
+                                              float gf, uint4 rnd, uint32_t lut_addr)
 {
+    constexpr bool kLut8 = LutKind<BITS, IDENTITY>::k8;
     const uint32_t words[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
     // Indices are accumulated as z * 2^(BITS*slot) with multiply-adds into two 32-bit halves
-    // (coordinates 0-3 and 4-7 for BITS = 8, otherwise everything in the low half).
+    // (coordinates 0-3 and 4-7).  With the 8-byte entries the whole second word is multiplied
+    // in: what its upper half leaves above bit 16 is cut off at the end (4 BITS <= 16 valid bits).
     uint32_t acc[2] = {0u, 0u};
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
         float u;
         asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(u) : "f"(r[e]), "f"(kappa), "f"(offset));
         const float t = __fmaf_rd(u, gf, 8388608.0f);          // 2^23 + floor(u * g)
-        const uint32_t u16 = (e & 1) ? (words[e >> 1] >> 16) : (words[e >> 1] & 0xFFFFu);
-        const uint32_t ub = u16 | 0x4B000000u;                 // bits of 2^23 + u16
-        uint32_t z0;
+        // bits of 2^23 + u16
+        const uint32_t ub = (e & 1) ? __byte_perm(words[e >> 1], 0x4B000000u, 0x7432)
+                                    : __byte_perm(words[e >> 1], 0x4B000000u, 0x7410);
+        uint32_t zw;
         float tau;
         if (IDENTITY) {
-            z0 = __float_as_uint(t) & 0xFFu;
+            zw = __float_as_uint(t) & 0xFFu;
             const float delta = fmaf(u, gf, 8388608.0f - t);
             tau = fmaf(delta, 65536.0f, 8388608.0f);
+        } else if (kLut8) {
+            const uint32_t a = __float_as_uint(t) * (uint32_t)kLutEntryBytes + lut_addr;
+            uint32_t x, y;
+            asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(x), "=r"(y) : "r"(a));
+            const float delta = fmaf(u, gf, __uint_as_float(y & 0xFFFF0000u));
+            tau = fmaf(delta, __uint_as_float(x), 8388608.0f);
+            zw = y;
         } else {
-            const uint4 entry = lut[(__float_as_uint(t) & 0xFFu) * lut_stride];
-            z0 = entry.z;
-            const float delta = fmaf(u, gf, __uint_as_float(entry.x));
-            tau = fmaf(delta, __uint_as_float(entry.y), 8388608.0f);
+            const uint32_t a = __float_as_uint(t) * (uint32_t)kLutEntryBytes + lut_addr;
+            uint32_t x, y, z, w;
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "r"(a));
+            const float delta = fmaf(u, gf, __uint_as_float(x));
+            tau = fmaf(delta, __uint_as_float(y), 8388608.0f);
+            zw = z;
         }
-        constexpr int half = BITS == 8 ? 1 : 0;
-        const int slot = BITS == 8 ? (e & 3) : e;
-        const int h = half ? (e >> 2) : 0;
-        const uint32_t weight = 1u << (BITS * slot);
-        acc[h] = z0 * weight + acc[h];
+        const int h = e >> 2;
+        const uint32_t weight = 1u << (BITS * (e & 3));
+        acc[h] = zw * weight + acc[h];
         if (ub < __float_as_uint(tau)) acc[h] += weight;
     }
-    return (uint64_t)acc[0] | ((uint64_t)acc[1] << 32);
+    if constexpr (BITS == 8) return (uint64_t)acc[0] | ((uint64_t)acc[1] << 32);
+    if constexpr (BITS == 4) return (uint64_t)__byte_perm(acc[0], acc[1], 0x5410);
+    constexpr uint32_t mask = (1u << (4 * BITS)) - 1u;
+    return (uint64_t)((acc[0] & mask) | ((acc[1] & mask) << (4 * BITS)));
 }
 
 }  // namespace thc

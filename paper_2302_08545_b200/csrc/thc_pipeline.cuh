@@ -108,6 +108,7 @@ struct PipeParams {
     uint32_t b_swz_mask;       // run-time geometry, pass-B tiles: chunk c sits at c ^ ((c >> 3) & mask)
     uint32_t b_tma;            // ... and are fetched by TMA in this many boxes of 256 rows (k = 21: one;
                                // k = 22: two, 64-byte rows with the 64-byte swizzle); 0: by the compute warps
+    uint32_t nbuf;             // thc_warp_pipeline_kernel: tile buffers per CTA
 };
 
 struct PtrArrayP { const void *p[THC_MAX_WORKERS]; };
@@ -602,7 +603,7 @@ __device__ __forceinline__ void pass_a_round3_store(const float4 *tile, float *d
 struct EpilogueCtx {
     uint64_t j_tile;        // coordinate of (row 0, column 0) of the tile in the worker's vector
     float kappa, half_g, gf, c_block;
-    const uint4 *lut;
+    uint32_t lut;           // this lane's address into the quantiser table (lut_lane_addr)
     uint32_t worker, round;
     unsigned char *packed;
     float *rotated;
@@ -643,7 +644,7 @@ __device__ __forceinline__ void epilogue_unit(const float4 &va, const float4 &vb
         }
         const float r[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
         const uint4 rnd = round_call(j, ep.worker, ep.round, keys);
-        const uint64_t z = quantize8<BITS, IDENTITY>(r, ep.kappa, ep.half_g, ep.gf, rnd, ep.lut, kLutRep);
+        const uint64_t z = quantize8<BITS, IDENTITY>(r, ep.kappa, ep.half_g, ep.gf, rnd, ep.lut);
         if constexpr (BITS == 8)
             *reinterpret_cast<uint2 *>(ep.packed + j) = make_uint2((uint32_t)z, (uint32_t)(z >> 32));
         else if constexpr (BITS == 4)
@@ -776,9 +777,9 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
     float4 *bufs[2] = {reinterpret_cast<float4 *>(pipe_smem),
                        reinterpret_cast<float4 *>(pipe_smem + kPElems * 4)};
     uint32_t *sw = reinterpret_cast<uint32_t *>(pipe_smem + 2 * kPElems * 4);
-    uint4 *lut = reinterpret_cast<uint4 *>(pipe_smem + 2 * kPElems * 4 + kPSignWords * 4);
+    unsigned char *lut = pipe_smem + 2 * kPElems * 4 + kPSignWords * 4;
     float2 *blk_const = reinterpret_cast<float2 *>(pipe_smem + 2 * kPElems * 4 + kPSignWords * 4 +
-                                                   (size_t)(P.granularity + 1) * kLutRep * 16);
+                                                   (size_t)(P.granularity + 1) * kLutEntryBytes);
     __shared__ TaskInfo s_info[2];
     __shared__ __align__(8) uint64_t s_mbar[2];
     __shared__ __align__(8) uint64_t s_done;           // one phase per finished task (compute warps arrive)
@@ -799,10 +800,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
         mbar_init(&s_done, kPThreads);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (kCompress && !IDENTITY && !kRange) {
-        for (int idx = tid; idx < (int)(P.granularity + 1) * kLutRep; idx += kPCtaThreads)
-            lut[idx] = P.dev->lut[idx / kLutRep];
-    }
+    if (kCompress && !IDENTITY && !kRange) lut_fill<LutKind<BITS, IDENTITY>::k8>(lut, P.dev, P.granularity, tid, kPCtaThreads);
     // error feedback: table values as floats, one copy per lane (8 copies for 8-bit indices)
     constexpr int kFRep = BITS <= 4 ? 32 : 8;
     float *ftab = reinterpret_cast<float *>(lut);
@@ -1181,7 +1179,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 EpilogueCtx ep;
                 ep.j_tile = j_tile;
                 ep.kappa = bc.x; ep.half_g = bc.y; ep.gf = (float)P.granularity; ep.c_block = P.c_block;
-                ep.lut = lut + (tid & (kLutRep - 1));
+                ep.lut = lut_lane_addr<LutKind<BITS, IDENTITY>::k8>(lut, tid);
                 ep.worker = P.worker_base + wl; ep.round = P.round;
                 ep.packed = kCompress ? static_cast<unsigned char *>(outp.p[wl]) : nullptr;
                 ep.rotated = kCompress ? static_cast<float *>(rotated.p[wl]) : nullptr;
