@@ -864,7 +864,7 @@ int thc_create(const thc_config *cfg, thc_ctx **out)
     ctx->device = -1;
     ctx->dev = nullptr;
     ctx->sm_count = 148;
-    ctx->legacy_pipeline = true;
+    ctx->legacy_pipeline = false;
     uint32_t k0 = (uint32_t)cfg->seed, k1 = (uint32_t)(cfg->seed >> 32);
     for (int r = 0; r < 10; ++r) {
         ctx->keys.k[2 * r] = k0;

@@ -745,16 +745,21 @@ __device__ __forceinline__ void pass_b_last_round_kb7(float4 *tile, int tid,
                     butterfly(b[m], b[m | (1 << t)]);
                 }
         }
-        // back to the thread's own slots: the epilogue below is a compact loop (code size)
+        // The epilogue is a loop of two iterations over four rows each (unrolled over all eight
+        // it does not fit the instruction cache): the second iteration's rows move down the
+        // register arrays in between.
+        const int uu = 4 * h + u;
+        const uint64_t j0 = ep.j_tile + ((uint64_t)rl << kPLog2) + 8 * uu;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
 #pragma unroll
-        for (int m = 0; m < 8; ++m) { pa[m << 7] = a[m]; pb[m << 7] = b[m]; }
+            for (int m = 0; m < 4; ++m)
+                epilogue_unit<COMPRESS, BITS, IDENTITY, RANGE>(a[m], b[m], j0 + ((uint64_t)(4 * half + m) << (kPLog2 + 4)),
+                                                               rl + 16 * (4 * half + m), uu, ep, keys, kmin, kmax);
+#pragma unroll
+            for (int m = 0; m < 4; ++m) { a[m] = a[m + 4]; b[m] = b[m + 4]; }
+        }
     }
-    const int uu = 4 * h + u;
-    const uint64_t j0 = ep.j_tile + ((uint64_t)rl << kPLog2) + 8 * uu;
-#pragma unroll 2
-    for (int m = 0; m < 8; ++m)
-        epilogue_unit<COMPRESS, BITS, IDENTITY, RANGE>(pa[m << 7], pb[m << 7], j0 + ((uint64_t)m << (kPLog2 + 4)),
-                                                       rl + 16 * m, uu, ep, keys, kmin, kmax);
 }
 
 // ------------------------------------------------------------------------------ the kernel

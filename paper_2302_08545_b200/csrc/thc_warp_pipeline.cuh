@@ -284,8 +284,8 @@ thc_warp_pipeline_kernel(const __grid_constant__ WarpMaps maps, PipeParams P, Pt
             if (__any_sync(0xFFFFFFFFu, progress)) {
                 idle = 0;
             } else {
-                __nanosleep(32);
-                if (++idle > (1u << 25)) {              // about a second without any progress
+                __nanosleep(256);                       // tasks take microseconds: poll a few times per task
+                if (++idle > (1u << 22)) {              // about a second without any progress
                     if (lane == 0) { atomicOr(&P.dev->status, THC_STATUS_WAIT_TIMEOUT); atomicExch(&pc->abort, 1u); }
                     break;
                 }
