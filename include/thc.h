@@ -249,11 +249,6 @@ int thc_status(thc_ctx *ctx, uint32_t *flags, void *stream);
  * context still usable; the outputs of that call are undefined.  Synchronises the device. */
 int thc_debug_skip_tasks(thc_ctx *ctx, uint32_t count);
 
-/* Test hook (no counterpart in the paper): with on != 0, thc_compress on this context keeps to
- * the general large-block kernel also where the specialised kernel for 2^20-coordinate blocks of
- * fp32 gradients applies; both must produce the same bytes.  Host only. */
-int thc_debug_legacy_pipeline(thc_ctx *ctx, int on);
-
 const char *thc_strerror(int code);
 
 /* Library build identification, e.g. "thc-b200 sm_100a". */

@@ -769,7 +769,6 @@ aggregate_kernel(PtrArray in, uint32_t n, uint64_t units, uint64_t d_pad, const 
 }  // namespace thc
 
 #include "thc_pipeline.cuh"
-#include "thc_warp_pipeline.cuh"
 
 // =========================================================================== host side
 using namespace thc;
@@ -783,7 +782,6 @@ struct thc_ctx {
     PhiloxKeys keys;
     uint32_t lut_rep;
     int sm_count;
-    bool legacy_pipeline;       // test hook: keep thc_compress on thc_pipeline_kernel
 };
 
 static thread_local cudaError_t g_last_cuda = cudaSuccess;
@@ -864,7 +862,6 @@ int thc_create(const thc_config *cfg, thc_ctx **out)
     ctx->device = -1;
     ctx->dev = nullptr;
     ctx->sm_count = 148;
-    ctx->legacy_pipeline = false;
     uint32_t k0 = (uint32_t)cfg->seed, k1 = (uint32_t)(cfg->seed >> 32);
     for (int r = 0; r < 10; ++r) {
         ctx->keys.k[2 * r] = k0;
@@ -1312,114 +1309,6 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
     return THC_OK;
 }
 
-// ---- warp-pipeline dispatch (2^20-coordinate blocks, fp32 gradients in, indices out)
-typedef void (*warp_kernel_t)(const WarpMaps, PipeParams, PtrArrayP, MutPtrArrayP, MutPtrArrayP, PhiloxKeys);
-
-static warp_kernel_t pick_warp_kernel(uint32_t bits, bool identity)
-{
-    switch (bits) {
-    case 1: return identity ? thc_warp_pipeline_kernel<1, true> : thc_warp_pipeline_kernel<1, false>;
-    case 2: return identity ? thc_warp_pipeline_kernel<2, true> : thc_warp_pipeline_kernel<2, false>;
-    case 3: return identity ? thc_warp_pipeline_kernel<3, true> : thc_warp_pipeline_kernel<3, false>;
-    case 4: return identity ? thc_warp_pipeline_kernel<4, true> : thc_warp_pipeline_kernel<4, false>;
-    default: return identity ? thc_warp_pipeline_kernel<8, true> : thc_warp_pipeline_kernel<8, false>;
-    }
-}
-
-static bool warp_pipeline_applies(const thc_ctx *ctx)
-{
-    return ctx->cfg.log2_block == 20 && ctx->cfg.in_dtype == THC_F32 && !ctx->legacy_pipeline;
-}
-
-// Schedule for one CTA per SM with kWMaxBuf tasks in flight each.  Never asks for more ring
-// slots than plan_pipeline, which sizes the workspace.
-static PipePlan plan_warp_pipeline(const thc_ctx *ctx, uint64_t wb_count)
-{
-    const uint64_t T = 128;
-    const uint64_t tasks = wb_count * T * 2;
-    PipePlan p;
-    p.grid = (uint32_t)(tasks < (uint64_t)ctx->sm_count ? tasks : (uint64_t)ctx->sm_count);
-    const uint64_t inflight = (uint64_t)ctx->sm_count * (kWMaxBuf + 1);
-    uint64_t lag = (inflight + 2 * T - 1) / (2 * T) + 1;
-    uint64_t ring = lag + (inflight + 2 * T - 1) / (2 * T) + 1;
-    const PipePlan legacy = plan_pipeline(ctx, wb_count);
-    if (ring > legacy.ring) { ring = legacy.ring; if (lag > ring - 2 && ring > 2) lag = ring - 2; }
-    if (lag > wb_count) lag = wb_count;
-    if (ring > wb_count) ring = wb_count;
-    p.lag = (uint32_t)lag;
-    p.ring = (uint32_t)ring;
-    return p;
-}
-
-static int launch_warp_pipeline(const thc_ctx *ctx, const thc_sizes_t &sz, uint64_t d, uint32_t n_local,
-                                uint32_t worker_base, uint32_t round, const float *scales, void *workspace,
-                                const PtrArrayP &in, const MutPtrArrayP &out, const MutPtrArrayP &rot,
-                                cudaStream_t st)
-{
-    const uint32_t k = 20;
-    PipeParams P;
-    memset(&P, 0, sizeof P);
-    P.d = d;
-    P.d_pad = sz.d_pad;
-    P.wb_count = sz.nblocks * n_local;
-    P.total_tasks = P.wb_count * 256;
-    if (P.wb_count >= 0x7FFFFFFFull || P.total_tasks >= 0x7FFFFFFFull) return THC_EUNSUPPORTED;
-    const PipePlan pl = plan_warp_pipeline(ctx, P.wb_count);
-    P.ring = static_cast<float *>(workspace);
-    P.scales = scales;
-    P.dev = ctx->dev;
-    P.k = k;
-    P.kb = k - kPLog2;
-    P.n_local = n_local;
-    P.lag = pl.lag;
-    P.ring_slots = pl.ring;
-    P.granularity = ctx->cfg.granularity;
-    P.divisor = 1;
-    P.round = round;
-    P.worker_base = worker_base;
-    P.c_block = (float)(1.0 / sqrt((double)(1ull << k)));
-    P.exact_range = ctx->cfg.range_mode == THC_RANGE_MINMAX ? 1u : 0u;
-    P.nblocks = (uint32_t)sz.nblocks;
-    P.nbuf = kWMaxBuf;
-    const uint64_t nblk_cached = sz.nblocks < (uint64_t)kBlockConstMax ? sz.nblocks : (uint64_t)kBlockConstMax;
-    const size_t smem = (size_t)1024 + (size_t)kWMaxBuf * kWBufBytes + (size_t)(ctx->cfg.granularity + 1) * 128 +
-                        (size_t)nblk_cached * 8;
-    warp_kernel_t kern = pick_warp_kernel(ctx->cfg.bits, ctx->identity);
-    { const int rc = ensure_dynamic_smem(reinterpret_cast<const void *>(kern), smem); if (rc != THC_OK) return rc; }
-    encode_tiled_t enc = get_encode_tiled();
-    if (enc == nullptr) return THC_ECUDA;
-    WarpMaps maps;
-    memset(&maps, 0, sizeof maps);
-    {
-        // ring: rows of 4096 floats (one per pass-A half tile), 256 per slot; box 32 columns x 256 rows
-        const cuuint64_t dims[2] = {4096, (cuuint64_t)pl.ring * 256};
-        const cuuint64_t strides[1] = {16384};
-        const cuuint32_t box[2] = {32, 256};
-        const cuuint32_t es[2] = {1, 1};
-        if (enc(&maps.ring, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, workspace, dims, strides, box, es,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return THC_ECUDA;
-    }
-    if ((d >> 7) >= 64) {
-        // gradient as (32 floats, 4 rows, groups of 4 rows): a box takes one of the four rows of
-        // 32 consecutive groups, i.e. every fourth 128-byte row of half a tile
-        for (uint32_t i = 0; i < n_local; ++i) {
-            const cuuint64_t dims[3] = {32, 4, d >> 7};
-            const cuuint64_t strides[2] = {128, 512};
-            const cuuint32_t box[3] = {32, 1, 32};
-            const cuuint32_t es[3] = {1, 1, 1};
-            if (enc(&maps.in[i], CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void *>(in.p[i]), dims, strides,
-                    box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-                return THC_ECUDA;
-        }
-    }
-    kern<<<pl.grid, kWThreads, smem, st>>>(maps, P, in, out, rot, ctx->keys);
-    THC_CUDA(cudaGetLastError());
-    return THC_OK;
-}
-
 // thc_prepare in exact-range mode (Algorithm 1's preliminary stage on the rotated coordinates):
 // one transform pass over all workers whose epilogue only takes the minimum and maximum, then
 // the keys become the (lo, hi) planes of `scales`.  This costs about as much as the transform
@@ -1536,8 +1425,6 @@ int thc_compress(thc_ctx *ctx, const void *const *grads, uint32_t n_local, uint3
     memcpy(&pin, &in, sizeof pin);
     memcpy(&pout, &out, sizeof pout);
     memcpy(&prot, &rot, sizeof prot);
-    if (warp_pipeline_applies(ctx))
-        return launch_warp_pipeline(ctx, sz, d, n_local, worker_base, round, scales, workspace, pin, pout, prot, st);
     pipe_kernel_t kern = bf16 ? pick_pipe_kernel<kCompressBF16>(ctx->cfg.bits, ctx->identity, k)
                               : pick_pipe_kernel<kCompressF32>(ctx->cfg.bits, ctx->identity, k);
     return launch_pipeline(ctx, kern, !bf16, sz, d, n_local, worker_base, round, 1, scales, workspace,
@@ -1832,13 +1719,6 @@ int thc_debug_skip_tasks(thc_ctx *ctx, uint32_t count)
     THC_CUDA(cudaDeviceSynchronize());
     PipeCounters *pc = reinterpret_cast<PipeCounters *>(ctx->dev->counters);
     THC_CUDA(cudaMemcpy(&pc->head, &count, sizeof count, cudaMemcpyHostToDevice));
-    return THC_OK;
-}
-
-int thc_debug_legacy_pipeline(thc_ctx *ctx, int on)
-{
-    if (ctx == nullptr) return THC_EINVAL;
-    ctx->legacy_pipeline = on != 0;
     return THC_OK;
 }
 

@@ -108,7 +108,6 @@ struct PipeParams {
     uint32_t b_swz_mask;       // run-time geometry, pass-B tiles: chunk c sits at c ^ ((c >> 3) & mask)
     uint32_t b_tma;            // ... and are fetched by TMA in this many boxes of 256 rows (k = 21: one;
                                // k = 22: two, 64-byte rows with the 64-byte swizzle); 0: by the compute warps
-    uint32_t nbuf;             // thc_warp_pipeline_kernel: tile buffers per CTA
 };
 
 struct PtrArrayP { const void *p[THC_MAX_WORKERS]; };

@@ -21,7 +21,7 @@ STATUS_NONFINITE, STATUS_ZERO_BLOCK, STATUS_WAIT_TIMEOUT = 1, 2, 4
 
 EXPORTS = ("thc_create", "thc_destroy", "thc_sizes", "thc_prepare", "thc_compress",
            "thc_quantize_rotated", "thc_aggregate", "thc_decompress", "thc_prepare_noalloc",
-           "thc_error_feedback", "thc_accumulate_error", "thc_prepare_compress", "thc_prepare_minmax", "thc_debug_skip_tasks", "thc_debug_legacy_pipeline", "thc_status", "thc_strerror", "thc_version")
+           "thc_error_feedback", "thc_accumulate_error", "thc_prepare_compress", "thc_prepare_minmax", "thc_debug_skip_tasks", "thc_status", "thc_strerror", "thc_version")
 NOALLOC_SCRATCH_BYTES = 4 << 20
 
 
@@ -85,7 +85,6 @@ def lib():
     L.thc_error_feedback.argtypes = [vp, pp, pp, u32, u64, u32, vp, pp, vp, u64, vp]
     L.thc_accumulate_error.argtypes = [vp, pp, pp, u32, u64, vp]
     L.thc_debug_skip_tasks.argtypes = [vp, u32]
-    L.thc_debug_legacy_pipeline.argtypes = [vp, ctypes.c_int]
     L.thc_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
     for name in EXPORTS[:-2]:
         getattr(L, name).restype = ctypes.c_int
@@ -249,10 +248,6 @@ class Context:
     def debug_skip_tasks(self, count: int):
         """Test hook: the next pipeline launch starts its task queue at `count`."""
         _check(lib().thc_debug_skip_tasks(self._h, count), "thc_debug_skip_tasks")
-
-    def debug_legacy_pipeline(self, on: bool):
-        """Test hook: keep thc_compress on the general large-block kernel."""
-        _check(lib().thc_debug_legacy_pipeline(self._h, 1 if on else 0), "thc_debug_legacy_pipeline")
 
     def status(self, stream=None) -> int:
         flags = ctypes.c_uint32(0)
