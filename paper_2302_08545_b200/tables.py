@@ -78,36 +78,3 @@ def optimal_table(bits: int, g: int, p: float):
     if abs(table_cost(mirror, g, tp) - table_cost(table, g, tp)) <= 1e-13 and mirror < table:
         table = mirror
     return table, table_cost(table, g, tp)
-
-
-def stars_and_bars(n: int, k: int):
-    """All ways to throw n identical balls into k bins (Appendix B's enumeration), in the
-    order of its Algorithm 4: start with everything in bin 0; each step moves one ball from
-    the first non-empty bin to the next bin and returns the rest of that bin to bin 0."""
-    b = [0] * k
-    b[0] = n
-    yield tuple(b)
-    total = math.comb(n + k - 1, k - 1)
-    for _ in range(total - 1):
-        a = next(i for i in range(k) if b[i] > 0)
-        b[a + 1] += 1
-        rest = b[a] - 1
-        b[a] = 0
-        b[0] = rest
-        yield tuple(b)
-
-
-def brute_force_table(bits: int, g: int, p: float):
-    """Exhaustive search over all strictly increasing tables (small cases only)."""
-    levels = 1 << bits
-    tp = t_p(p)
-    best = None
-    for extra in stars_and_bars(g - (levels - 1), levels - 1):
-        table = [0]
-        for e in extra:
-            table.append(table[-1] + 1 + e)
-        c = table_cost(table, g, tp)
-        key = (round(c, 13), tuple(table))
-        if best is None or key < best:
-            best = key
-    return best[1], best[0]

@@ -1,6 +1,7 @@
 """The lookup-table solver (Section 5.2 / Appendix B) against brute force and the paper's
 printed facts, and the tables the workloads use against the solver."""
 import math
+from itertools import combinations
 
 import pytest
 from scipy import integrate
@@ -35,19 +36,45 @@ def test_paper_worked_integral_is_the_interval_sum():
     assert abs(tables.table_cost((0, 1, 3, 4), 4, tp) - ref) < 1e-12
 
 
-def test_stars_and_bars_enumeration_is_complete_and_duplicate_free():
-    for n, k in ((0, 3), (3, 1), (4, 3), (5, 4)):
-        seen = list(tables.stars_and_bars(n, k))
-        assert len(seen) == math.comb(n + k - 1, k - 1) == len(set(seen))
-        assert all(sum(b) == n and min(b) >= 0 for b in seen)
-    assert next(iter(tables.stars_and_bars(4, 3))) == (4, 0, 0)
+def increasing_tables(bits: int, g: int):
+    """Every table 0 = T[0] < T[1] < ... < T[2^b - 1] = g: the inner values are a subset of
+    {1, ..., g - 1} in increasing order.  (Appendix B counts them as g - 2^b + 1 balls in
+    2^b - 1 bins, the balls being the grid points skipped between neighbours.)"""
+    for inner in combinations(range(1, g), (1 << bits) - 2):
+        yield (0,) + inner + (g,)
+
+
+def brute_force_table(bits: int, g: int, p: float):
+    """Exhaustive search over all strictly increasing tables (small cases only)."""
+    tp = tables.t_p(p)
+    best = None
+    for table in increasing_tables(bits, g):
+        key = (round(tables.table_cost(table, g, tp), 13), table)
+        if best is None or key < best:
+            best = key
+    return best[1], best[0]
+
+
+def test_enumeration_counts_match_appendix_b():
+    """The number of candidate tables is C(g - 1, 2^b - 2), which is Appendix B's stars-and-bars
+    count C(n + k - 1, k - 1) with n = g - 2^b + 1 balls and k = 2^b - 1 bins; for b = 4, g = 51 the
+    paper quotes about 4.8e11 candidates, and 100947 after its symmetry reduction for the
+    example it works out."""
+    for bits, g in ((1, 5), (2, 4), (2, 9), (3, 12)):
+        levels = 1 << bits
+        tabs = list(increasing_tables(bits, g))
+        n, k = g - levels + 1, levels - 1
+        assert len(tabs) == len(set(tabs)) == math.comb(n + k - 1, k - 1) == math.comb(g - 1, levels - 2)
+        assert all(t[0] == 0 and t[-1] == g and all(a < b for a, b in zip(t, t[1:])) for t in tabs)
+    assert abs(math.comb(48, 14) / 4.8e11 - 1) < 0.01
+    assert math.comb(23, 6) == 100947
 
 
 @pytest.mark.parametrize("bits,g", [(1, 1), (1, 5), (2, 3), (2, 4), (2, 9), (3, 7), (3, 12), (3, 14)])
 def test_dp_equals_brute_force(bits, g):
     for p in (1 / 32, 1 / 1024):
         t_dp, c_dp = tables.optimal_table(bits, g, p)
-        t_bf, c_bf = tables.brute_force_table(bits, g, p)
+        t_bf, c_bf = brute_force_table(bits, g, p)
         assert abs(c_dp - c_bf) < 1e-12
         assert t_dp == t_bf
 
