@@ -169,6 +169,20 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
                    const float *scales, float *out, void *workspace, uint64_t workspace_bytes,
                    void *stream);
 
+/* thc_aggregate followed by thc_decompress as one call, for a caller that holds all n workers'
+ * packed indices on this GPU (the simulated cluster): Algorithm 2's PS line, Y = sum_i T[Z_i],
+ * feeding the worker's estimate line and the inverse RHT (Algorithm 3) directly.  For RHT blocks
+ * above 2^14 coordinates this is one launch and the sums never travel through memory; they are
+ * written (d_pad unsigned integers of acc_bits bits, as thc_aggregate writes them) only if
+ * sum_or_null is given.  `out` is bit for bit what the two calls give with divisor n.  The paper's
+ * PS is another machine, so the separate calls remain the general form.
+ *   packed       host array of n device pointers (n <= thc_config.workers)
+ *   out          device, d fp32, written
+ *   sum_or_null  device, sum_bytes, written if not NULL                                      */
+int thc_aggregate_decompress(thc_ctx *ctx, const void *const *packed, uint32_t n, uint64_t d,
+                             uint32_t round, const float *scales, float *out, void *sum_or_null,
+                             void *workspace, uint64_t workspace_bytes, void *stream);
+
 /* Preliminary stage without any allocation, for callers that may not call cudaMalloc (a
  * plugin inside a host framework's fixed memory plan, code running under a frozen memory
  * budget) and so can use neither thc_create (which allocates the context's device block)
@@ -178,7 +192,8 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
  * GPU that loads the library, until the process exits).
  *   grads            host array of n device pointers (16-byte aligned), d elements each
  *   log2_block, in_dtype, t_p   as in thc_config
- *   scales           device, ceil(d / 2^log2_block) fp32, written; same values as thc_prepare
+ *   scales           device, ceil(d / 2^log2_block) fp32, written; the values of thc_prepare up to
+ *                    the last bit (the fp64 partial sums are added in another fixed order)
  *   status_or_null   device word that THC_STATUS_NONFINITE / THC_STATUS_ZERO_BLOCK are OR-ed
  *                    into, or NULL
  * Limit: n * ceil(d_pad / 2^min(log2_block,14)) partial sums must fit the array (524,288
@@ -186,7 +201,8 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
  * cudaFree or any allocating routine never.  The first call on a device looks up the
  * array's device address (cudaGetSymbolAddress); make that call before any stream capture.
  * All calls share the array: calls that overlap on the GPU race; calls on one stream do
- * not.  Nothing in the array has to be cleared between calls. */
+ * not.  Nothing in the array has to be cleared between calls.  d > 2^40 is THC_EINVAL like
+ * everywhere else; device ordinals of 64 and above are not served (THC_ECUDA). */
 #define THC_NOALLOC_SCRATCH_BYTES (4u << 20)
 int thc_prepare_noalloc(const void *const *grads, uint32_t n, uint64_t d, uint32_t log2_block,
                         uint32_t in_dtype, double t_p, float *scales, uint32_t *status_or_null,
@@ -225,8 +241,10 @@ int thc_prepare_compress(thc_ctx *ctx, const void *const *grads, uint32_t n, uin
  * workers, the residual between what it compressed and what its own indices stand for,
  *     ef[i] = x_i - RHT^-1( m + T[Z_i] (M - m)/g ),
  * to be added to the next round's gradient (thc_accumulate_error).  fp32 contexts only
- * (THC_EUNSUPPORTED for bf16 inputs).  Built from the library's own kernels: table values
- * of one worker (thc_aggregate with n = 1), thc_decompress with divisor 1, one subtraction.
+ * (THC_EUNSUPPORTED for bf16 inputs).  For RHT blocks above 2^14 coordinates this is one launch
+ * over all workers (indices in, de-quantised in registers, inverse transform, x - result out);
+ * for smaller blocks it is composed per worker of thc_aggregate with n = 1, thc_decompress with
+ * divisor 1 and one subtraction.  Both give the same bits.
  *   grads    host array of n_local device pointers: the x_i that were compressed
  *   packed   host array of n_local device pointers: their packed indices
  *   ef       host array of n_local device pointers, d fp32 each, written
@@ -245,7 +263,7 @@ int thc_status(thc_ctx *ctx, uint32_t *flags, void *stream);
 /* Test hook for the bounded waits of the large-block pipeline (no counterpart in the paper).
  * The next thc_compress / thc_decompress on this context starts its task queue at position
  * `count` instead of 0, so tasks that depend on the skipped ones can never be satisfied: the
- * kernel must notice (about two seconds), set THC_STATUS_WAIT_TIMEOUT, and return with the
+ * kernel must notice (about one second), set THC_STATUS_WAIT_TIMEOUT, and return with the
  * context still usable; the outputs of that call are undefined.  Synchronises the device. */
 int thc_debug_skip_tasks(thc_ctx *ctx, uint32_t count);
 

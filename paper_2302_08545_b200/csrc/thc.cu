@@ -366,7 +366,7 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 }
 
 __global__ void __launch_bounds__(kThreads)
-aggregate_b4w8_kernel(PtrArray in, uint32_t n, uint64_t units16, const DeviceBlock *dev,
+aggregate_b4w8_kernel(PtrArray in, uint32_t n, uint64_t units32, const DeviceBlock *dev,
                       uint4 *__restrict__ sum)
 {
     uint32_t t[4];
@@ -374,21 +374,30 @@ aggregate_b4w8_kernel(PtrArray in, uint32_t n, uint64_t units16, const DeviceBlo
     for (int q = 0; q < 4; ++q)
         t[q] = dev->table[4 * q] | (dev->table[4 * q + 1] << 8) | (dev->table[4 * q + 2] << 16) |
                (dev->table[4 * q + 3] << 24);
-    for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < units16;
+    // A thread sums 32 coordinates: 16 bytes of indices per worker, the loads of up to eight
+    // workers in flight together, 32 bytes of sums out.
+    for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < units32;
          u += (uint64_t)gridDim.x * kThreads) {
-        uint32_t acc[4] = {0u, 0u, 0u, 0u};                  // 16 sums of 8 bits
-#pragma unroll 4
-        for (uint32_t i = 0; i < n; ++i) {
-            const uint2 w = __ldg(reinterpret_cast<const uint2 *>(in.p[i]) + u);   // 16 indices
-            const uint32_t words[2] = {w.x, w.y};
+        uint32_t acc[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};     // 32 sums of 8 bits
+#pragma unroll 1
+        for (uint32_t i0 = 0; i0 < n; i0 += 8) {
+            uint4 w[8];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const uint32_t a = words[h], b = a ^ 0x88888888u;
-                acc[2 * h] += prmt(t[0], t[1], a) + prmt(t[2], t[3], b);
-                acc[2 * h + 1] += prmt(t[0], t[1], a >> 16) + prmt(t[2], t[3], b >> 16);
+            for (int j = 0; j < 8; ++j)         // index 0 everywhere adds T[0] = 0
+                w[j] = i0 + j < n ? __ldcs(reinterpret_cast<const uint4 *>(in.p[i0 + j]) + u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t words[4] = {w[j].x, w[j].y, w[j].z, w[j].w};
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    const uint32_t a = words[h], b = a ^ 0x88888888u;
+                    acc[2 * h] += prmt(t[0], t[1], a) + prmt(t[2], t[3], b);
+                    acc[2 * h + 1] += prmt(t[0], t[1], a >> 16) + prmt(t[2], t[3], b >> 16);
+                }
             }
         }
-        sum[u] = make_uint4(acc[0], acc[1], acc[2], acc[3]);
+        __stcs(sum + 2 * u, make_uint4(acc[0], acc[1], acc[2], acc[3]));
+        __stcs(sum + 2 * u + 1, make_uint4(acc[4], acc[5], acc[6], acc[7]));
     }
 }
 
@@ -397,7 +406,7 @@ aggregate_b4w8_kernel(PtrArray in, uint32_t n, uint64_t units16, const DeviceBlo
 // 16-bit lanes (even and odd coordinates apart) and put back in order at the end.
 template <int CHUNK>
 __global__ void __launch_bounds__(kThreads)
-aggregate_b4w16_kernel(PtrArray in, uint32_t n, uint64_t units16, const DeviceBlock *dev,
+aggregate_b4w16_kernel(PtrArray in, uint32_t n, uint64_t units32, const DeviceBlock *dev,
                        uint4 *__restrict__ sum)
 {
     uint32_t t[4];
@@ -405,40 +414,43 @@ aggregate_b4w16_kernel(PtrArray in, uint32_t n, uint64_t units16, const DeviceBl
     for (int q = 0; q < 4; ++q)
         t[q] = dev->table[4 * q] | (dev->table[4 * q + 1] << 8) | (dev->table[4 * q + 2] << 16) |
                (dev->table[4 * q + 3] << 24);
-    for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < units16;
+    // A thread sums 32 coordinates: 16 bytes of indices per worker, 64 bytes of sums out.
+    for (uint64_t u = (uint64_t)blockIdx.x * kThreads + threadIdx.x; u < units32;
          u += (uint64_t)gridDim.x * kThreads) {
-        uint32_t even[4] = {0u, 0u, 0u, 0u}, odd[4] = {0u, 0u, 0u, 0u};
+        uint32_t even[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u}, odd[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
 #pragma unroll 1
         for (uint32_t i0 = 0; i0 < n; i0 += CHUNK) {
-            uint2 w[CHUNK];
+            uint4 w[CHUNK];
 #pragma unroll
-            for (int j = 0; j < CHUNK; ++j)
-                w[j] = i0 + j < n ? __ldg(reinterpret_cast<const uint2 *>(in.p[i0 + j]) + u) : make_uint2(0u, 0u);
-            uint32_t acc[4] = {0u, 0u, 0u, 0u};
+            for (int j = 0; j < CHUNK; ++j)      // index 0 everywhere adds T[0] = 0
+                w[j] = i0 + j < n ? __ldcs(reinterpret_cast<const uint4 *>(in.p[i0 + j]) + u) : make_uint4(0u, 0u, 0u, 0u);
+            uint32_t acc[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
 #pragma unroll
             for (int j = 0; j < CHUNK; ++j) {
-                const uint32_t words[2] = {w[j].x, w[j].y};   // index 0 everywhere adds T[0] = 0
+                const uint32_t words[4] = {w[j].x, w[j].y, w[j].z, w[j].w};
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
+                for (int h = 0; h < 4; ++h) {
                     const uint32_t a = words[h], b = a ^ 0x88888888u;
                     acc[2 * h] += prmt(t[0], t[1], a) + prmt(t[2], t[3], b);
                     acc[2 * h + 1] += prmt(t[0], t[1], a >> 16) + prmt(t[2], t[3], b >> 16);
                 }
             }
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+            for (int q = 0; q < 8; ++q) {
                 even[q] += acc[q] & 0x00FF00FFu;
                 odd[q] += (acc[q] >> 8) & 0x00FF00FFu;
             }
         }
-        uint32_t o[8];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            o[2 * q] = prmt(even[q], odd[q], 0x5410u);          // coordinates 4q, 4q+1
-            o[2 * q + 1] = prmt(even[q], odd[q], 0x7632u);      // coordinates 4q+2, 4q+3
+        for (int q4 = 0; q4 < 4; ++q4) {
+            uint32_t o[4];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                o[2 * q] = prmt(even[2 * q4 + q], odd[2 * q4 + q], 0x5410u);          // coordinates 4q, 4q+1
+                o[2 * q + 1] = prmt(even[2 * q4 + q], odd[2 * q4 + q], 0x7632u);      // coordinates 4q+2, 4q+3
+            }
+            __stcs(sum + 4 * u + q4, make_uint4(o[0], o[1], o[2], o[3]));
         }
-        sum[2 * u] = make_uint4(o[0], o[1], o[2], o[3]);
-        sum[2 * u + 1] = make_uint4(o[4], o[5], o[6], o[7]);
     }
 }
 
@@ -1154,7 +1166,7 @@ static pipe_kernel_t pick_pipe_kernel_kb(uint32_t bits, bool identity)
 {
     if constexpr (MODE == kRangeF32) {
         return thc_pipeline_kernel<MODE, 4, true, KB>;
-    } else if constexpr (MODE == kErrorFeedback) {
+    } else if constexpr (MODE == kErrorFeedback || MODE == kAggDecompress) {
         switch (bits) {
         case 1: return thc_pipeline_kernel<MODE, 1, true, KB>;
         case 2: return thc_pipeline_kernel<MODE, 2, true, KB>;
@@ -1229,7 +1241,7 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
                            const thc_sizes_t &sz, uint64_t d, uint32_t n_local, uint32_t worker_base, uint32_t round, uint32_t divisor,
                            const float *scales, void *workspace, const PtrArrayP &in,
                            const MutPtrArrayP &out, const MutPtrArrayP &rot, cudaStream_t st,
-                           float *fused_scales_out = nullptr, bool compress_bf16 = false)
+                           float *fused_scales_out = nullptr, bool compress_bf16 = false, uint32_t agg_n = 0)
 {
     const uint32_t k = ctx->cfg.log2_block;
     PipeParams P;
@@ -1263,6 +1275,8 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
     P.c_block = (float)(1.0 / sqrt((double)(1ull << k)));
     P.exact_range = ctx->cfg.range_mode == THC_RANGE_MINMAX ? 1u : 0u;
     P.nblocks = (uint32_t)sz.nblocks;
+    P.agg_n = agg_n;
+    P.agg_acc_bits = ctx->acc_bits;
     P.range_keys = reinterpret_cast<uint32_t *>(static_cast<unsigned char *>(workspace) +
                                                 ((uint64_t)pl.ring << k) * 4);
     const uint64_t nblk_cached = sz.nblocks < (uint64_t)kBlockConstMax ? sz.nblocks : (uint64_t)kBlockConstMax;
@@ -1519,6 +1533,48 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
                            prot, st);
 }
 
+// thc_aggregate followed by thc_decompress in one launch for the simulated cluster, whose workers'
+// packed indices all sit in this GPU's memory (Algorithm 2: the PS line Y = sum_i T[Z_i] feeding
+// the worker's estimate line and the inverse RHT): pass A of the inverse transform adds up the
+// table values itself, so the sums need not travel through HBM; they are written only on request.
+int thc_aggregate_decompress(thc_ctx *ctx, const void *const *packed, uint32_t n, uint64_t d, uint32_t round,
+                             const float *scales, float *outp, void *sum_or_null, void *workspace,
+                             uint64_t workspace_bytes, void *stream)
+{
+    int rc = check_launch_ctx(ctx);
+    if (rc != THC_OK) return rc;
+    if (n == 0 || n > ctx->cfg.workers) return THC_EINVAL;
+    thc_sizes_t sz;
+    if ((rc = thc_sizes(ctx, d, 1, &sz)) != THC_OK) return rc;
+    if ((rc = check_ptr_array(packed, n)) != THC_OK) return rc;
+    if (outp == nullptr || scales == nullptr || !aligned16(outp)) return THC_EINVAL;
+    if (sum_or_null != nullptr && !aligned16(sum_or_null)) return THC_EINVAL;
+    const uint32_t k = ctx->cfg.log2_block;
+    if (k <= (uint32_t)kTileLog2) {
+        // small blocks: the two calls (the sums go to the caller's buffer or to the workspace)
+        if (workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
+        if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
+        void *sum = sum_or_null != nullptr ? sum_or_null
+                  : static_cast<unsigned char *>(workspace) + (sz.workspace_bytes - round_up(sz.sum_bytes, 256));
+        if ((rc = thc_aggregate(ctx, packed, n, d, sum, stream)) != THC_OK) return rc;
+        return thc_decompress(ctx, sum, n, d, round, scales, outp, workspace,
+                              sz.workspace_bytes - round_up(sz.sum_bytes, 256), stream);
+    }
+    if (workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
+    if (workspace_bytes < sz.workspace_bytes - round_up(sz.sum_bytes, 256)) return THC_EWORKSPACE;
+    PtrArrayP pin;
+    MutPtrArrayP pout, prot;
+    memset(&pin, 0, sizeof pin);
+    memset(&pout, 0, sizeof pout);
+    memset(&prot, 0, sizeof prot);
+    for (uint32_t i = 0; i < n; ++i) pin.p[i] = packed[i];
+    pout.p[0] = outp;
+    pout.p[1] = sum_or_null;
+    pipe_kernel_t kern = pick_pipe_kernel<kAggDecompress>(ctx->cfg.bits, true, k);
+    return launch_pipeline(ctx, kern, false, sz, d, 1, 0, round, n, scales, workspace, pin, pout, prot,
+                           static_cast<cudaStream_t>(stream), nullptr, false, n);
+}
+
 int thc_quantize_rotated(thc_ctx *ctx, const float *const *rotated, uint32_t n_local,
                          uint32_t worker_base, uint64_t d, uint32_t round, const float *scales,
                          void *const *packed, void *stream)
@@ -1578,25 +1634,25 @@ int thc_aggregate(thc_ctx *ctx, const void *const *packed, uint32_t n, uint64_t 
     const uint64_t cap = (uint64_t)ctx->sm_count * 16;
     if (blocks > cap) blocks = cap;
     unsigned char *s = static_cast<unsigned char *>(sum);
-    if (ctx->cfg.bits == 4 && ctx->acc_bits == 8 && ctx->cfg.granularity < 128 && sz.d_pad % 16 == 0) {
-        const uint64_t units16 = sz.d_pad / 16;
-        uint64_t nb = (units16 + kThreads - 1) / kThreads;
-        const uint64_t cap16 = (uint64_t)ctx->sm_count * 8;
-        if (nb > cap16) nb = cap16;
-        aggregate_b4w8_kernel<<<(unsigned)nb, kThreads, 0, st>>>(in, n, units16, ctx->dev,
+    if (ctx->cfg.bits == 4 && ctx->acc_bits == 8 && ctx->cfg.granularity < 128 && sz.d_pad % 32 == 0) {
+        const uint64_t units32 = sz.d_pad / 32;
+        uint64_t nb = (units32 + kThreads - 1) / kThreads;
+        const uint64_t cap32 = (uint64_t)ctx->sm_count * 64;     // a unit or two per thread: no uneven tail
+        if (nb > cap32) nb = cap32;
+        aggregate_b4w8_kernel<<<(unsigned)nb, kThreads, 0, st>>>(in, n, units32, ctx->dev,
                                                                   reinterpret_cast<uint4 *>(s));
         THC_CUDA(cudaGetLastError());
         return THC_OK;
     }
     const uint32_t bits = ctx->cfg.bits, g = ctx->cfg.granularity, w = ctx->acc_bits;
-    if (bits == 4 && w == 16 && g < 128 && sz.d_pad % 16 == 0) {
-        const uint64_t units16 = sz.d_pad / 16;
-        uint64_t nb = (units16 + kThreads - 1) / kThreads;
-        if (nb > (uint64_t)ctx->sm_count * 8) nb = (uint64_t)ctx->sm_count * 8;
+    if (bits == 4 && w == 16 && g < 128 && sz.d_pad % 32 == 0) {
+        const uint64_t units32 = sz.d_pad / 32;
+        uint64_t nb = (units32 + kThreads - 1) / kThreads;
+        if (nb > (uint64_t)ctx->sm_count * 64) nb = (uint64_t)ctx->sm_count * 64;
         uint4 *s4 = reinterpret_cast<uint4 *>(s);
-        if (g <= 31) aggregate_b4w16_kernel<8><<<(unsigned)nb, kThreads, 0, st>>>(in, n, units16, ctx->dev, s4);
-        else if (g <= 63) aggregate_b4w16_kernel<4><<<(unsigned)nb, kThreads, 0, st>>>(in, n, units16, ctx->dev, s4);
-        else aggregate_b4w16_kernel<2><<<(unsigned)nb, kThreads, 0, st>>>(in, n, units16, ctx->dev, s4);
+        if (g <= 31) aggregate_b4w16_kernel<8><<<(unsigned)nb, kThreads, 0, st>>>(in, n, units32, ctx->dev, s4);
+        else if (g <= 63) aggregate_b4w16_kernel<4><<<(unsigned)nb, kThreads, 0, st>>>(in, n, units32, ctx->dev, s4);
+        else aggregate_b4w16_kernel<2><<<(unsigned)nb, kThreads, 0, st>>>(in, n, units32, ctx->dev, s4);
         THC_CUDA(cudaGetLastError());
         return THC_OK;
     }

@@ -149,6 +149,7 @@ extern "C" int thc_prepare_noalloc(const void *const *grads, uint32_t n, uint64_
     if (!(t_p > 0.0) || !isfinite(t_p)) return THC_EINVAL;
     for (uint32_t i = 0; i < n; ++i)
         if (grads[i] == nullptr || (reinterpret_cast<uintptr_t>(grads[i]) & 15u) != 0) return THC_EINVAL;
+    if (d > (1ull << 40)) return THC_EINVAL;          // the bound every other entry point applies
     const uint64_t B = 1ull << log2_block;
     const uint64_t d_pad = (d + B - 1) / B * B;
     const uint64_t nblocks = d_pad / B;

@@ -64,7 +64,8 @@ constexpr uint32_t kMaxPolls = 1u << 21;
 enum PipeMode { kCompressF32, kCompressBF16, kDecompress8, kDecompress16, kDecompress32,
                 kCompressF32Fused,     // fp32 compress that also computes the block scales (below)
                 kErrorFeedback,        // e_i = x_i - RHT^-1(X_i) from worker i's own packed indices
-                kRangeF32 };           // exact min / max of the rotated coordinates per RHT block
+                kRangeF32,             // exact min / max of the rotated coordinates per RHT block
+                kAggDecompress };      // decompress straight from the workers' packed indices (PS line + estimate line)
 
 // Layout inside DeviceBlock::counters.  Every CTA hits `head` and `abort` for every task and
 // the completion counters of the slots in use: each gets its own 128-byte line (head, exited,
@@ -106,6 +107,8 @@ struct PipeParams {
     uint32_t nblocks;
     uint32_t *range_keys;      // range mode: nblocks min keys then nblocks max keys
     uint32_t b_swz_mask;       // run-time geometry, pass-B tiles: chunk c sits at c ^ ((c >> 3) & mask)
+    uint32_t agg_n;            // kAggDecompress: workers whose table values are summed
+    uint32_t agg_acc_bits;     // ... and the width of the sums written on request (outp.p[1])
     uint32_t b_tma;            // ... and are fetched by TMA in this many boxes of 256 rows (k = 21: one;
                                // k = 22: two, 64-byte rows with the 64-byte swizzle); 0: by the compute warps
 };
@@ -555,6 +558,163 @@ __device__ __forceinline__ void pass_a_round1_inverse(float4 *tile, const unsign
     }
 }
 
+// First round of a pass-A tile of thc_aggregate_decompress: the PS line and the estimate line of
+// Algorithm 2 in one place.  The thread fetches the packed indices of its two rows from every
+// worker, adds up the table values (as floats: the sums stay below 2^24, so they are exact and
+// equal the integer sums thc_aggregate writes), optionally writes the sums, and goes on as
+// pass_a_round1_inverse does with v = m + Y (M - m)/(g n).
+template <int BITS, int FREP>
+__device__ __forceinline__ void pass_a_round1_aggregate(float4 *tile, const PtrArrayP &in, uint32_t agg_n,
+                                                        size_t byte_off, float2 bc, const float *ft,
+                                                        void *sum_out, size_t coord_off, uint32_t acc_bits, int tid,
+                                                        const uint32_t (&tb)[4], uint32_t swar_chunk)
+{
+    const int x = tid & 7;
+    const int r0 = ((tid >> 5) << 6) | (tid & 31);
+    float4 v[16];
+#pragma unroll
+    for (int m = 0; m < 16; ++m) v[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (BITS == 4 && swar_chunk != 0) {
+        // 4-bit indices, table values below 128: four look-ups per byte-permute instruction and
+        // sums in byte lanes (see aggregate_b4w8_kernel), `swar_chunk` workers at a time so that
+        // no byte overflows; the byte sums are then widened exactly into the float accumulators.
+#pragma unroll 1
+        for (uint32_t i0 = 0; i0 < agg_n; i0 += swar_chunk) {
+            uint32_t acc[2][8];
+#pragma unroll
+            for (int g = 0; g < 2; ++g)
+#pragma unroll
+                for (int q = 0; q < 8; ++q) acc[g][q] = 0u;
+            const uint32_t i1 = min(agg_n, i0 + swar_chunk);
+#pragma unroll 2
+            for (uint32_t i = i0; i < i1; ++i) {
+                const unsigned char *src = static_cast<const unsigned char *>(in.p[i]) + byte_off;
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    const uint4 t4 = __ldg(reinterpret_cast<const uint4 *>(src + (size_t)(r0 + 32 * g) * 16));
+                    const uint32_t words[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        const uint32_t a = words[h], b = a ^ 0x88888888u;
+                        uint32_t lo, hi, lo2, hi2;
+                        asm("prmt.b32 %0, %1, %2, %3;" : "=r"(lo) : "r"(tb[0]), "r"(tb[1]), "r"(a));
+                        asm("prmt.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(tb[2]), "r"(tb[3]), "r"(b));
+                        asm("prmt.b32 %0, %1, %2, %3;" : "=r"(lo2) : "r"(tb[0]), "r"(tb[1]), "r"(a >> 16));
+                        asm("prmt.b32 %0, %1, %2, %3;" : "=r"(hi2) : "r"(tb[2]), "r"(tb[3]), "r"(b >> 16));
+                        acc[g][2 * h] += lo + hi;
+                        acc[g][2 * h + 1] += lo2 + hi2;
+                    }
+                }
+            }
+#pragma unroll
+            for (int g = 0; g < 2; ++g)
+#pragma unroll
+                for (int m = 0; m < 8; ++m) {
+                    const uint32_t wv = acc[g][m];
+                    v[8 * g + m].x += __uint_as_float(__byte_perm(wv, 0x4B000000u, 0x7440)) - 8388608.0f;
+                    v[8 * g + m].y += __uint_as_float(__byte_perm(wv, 0x4B000000u, 0x7441)) - 8388608.0f;
+                    v[8 * g + m].z += __uint_as_float(__byte_perm(wv, 0x4B000000u, 0x7442)) - 8388608.0f;
+                    v[8 * g + m].w += __uint_as_float(__byte_perm(wv, 0x4B000000u, 0x7443)) - 8388608.0f;
+                }
+        }
+    } else
+#pragma unroll 1
+    for (uint32_t i = 0; i < agg_n; ++i) {
+        const unsigned char *src = static_cast<const unsigned char *>(in.p[i]) + byte_off;
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            const unsigned char *p = src + (size_t)(r0 + 32 * g) * (BITS * 4);
+            uint32_t w[BITS];
+            if constexpr (BITS >= 4) {
+#pragma unroll
+                for (int q = 0; q < BITS / 4; ++q) {
+                    const uint4 t4 = __ldg(reinterpret_cast<const uint4 *>(p) + q);
+                    w[4 * q] = t4.x; w[4 * q + 1] = t4.y; w[4 * q + 2] = t4.z; w[4 * q + 3] = t4.w;
+                }
+            } else if constexpr (BITS == 3) {
+                w[0] = __ldg(reinterpret_cast<const uint32_t *>(p));
+                w[1] = __ldg(reinterpret_cast<const uint32_t *>(p) + 1);
+                w[2] = __ldg(reinterpret_cast<const uint32_t *>(p) + 2);
+            } else if constexpr (BITS == 2) {
+                const uint2 t2 = __ldg(reinterpret_cast<const uint2 *>(p));
+                w[0] = t2.x; w[1] = t2.y;
+            } else {
+                w[0] = __ldg(reinterpret_cast<const uint32_t *>(p));
+            }
+#pragma unroll
+            for (int m = 0; m < 8; ++m) {
+                float sv[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int bit = (m * 4 + e) * BITS;
+                    const uint32_t nxt = w[((bit >> 5) + 1) < BITS ? (bit >> 5) + 1 : (bit >> 5)];
+                    const uint32_t val = __funnelshift_r(w[bit >> 5], nxt, bit & 31) & ((1u << BITS) - 1u);
+                    sv[e] = ft[val * FREP];
+                }
+                v[8 * g + m].x += sv[0]; v[8 * g + m].y += sv[1]; v[8 * g + m].z += sv[2]; v[8 * g + m].w += sv[3];
+            }
+        }
+    }
+    if (sum_out != nullptr) {
+        // the sums of the thread's two rows of 32 coordinates, acc_bits each
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            const size_t j = coord_off + (size_t)(r0 + 32 * g) * 32;
+            uint32_t y[32];
+#pragma unroll
+            for (int m = 0; m < 8; ++m) {
+                y[4 * m] = (uint32_t)v[8 * g + m].x; y[4 * m + 1] = (uint32_t)v[8 * g + m].y;
+                y[4 * m + 2] = (uint32_t)v[8 * g + m].z; y[4 * m + 3] = (uint32_t)v[8 * g + m].w;
+            }
+            if (acc_bits == 8) {
+                uint4 *o = reinterpret_cast<uint4 *>(static_cast<unsigned char *>(sum_out) + j);
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    uint32_t ww[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int b0 = 16 * q + 4 * c;
+                        ww[c] = y[b0] | (y[b0 + 1] << 8) | (y[b0 + 2] << 16) | (y[b0 + 3] << 24);
+                    }
+                    o[q] = make_uint4(ww[0], ww[1], ww[2], ww[3]);
+                }
+            } else if (acc_bits == 16) {
+                uint4 *o = reinterpret_cast<uint4 *>(static_cast<unsigned char *>(sum_out) + 2 * j);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t ww[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) ww[c] = y[8 * q + 2 * c] | (y[8 * q + 2 * c + 1] << 16);
+                    o[q] = make_uint4(ww[0], ww[1], ww[2], ww[3]);
+                }
+            } else {
+                uint4 *o = reinterpret_cast<uint4 *>(static_cast<unsigned char *>(sum_out) + 4 * j);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) o[q] = make_uint4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+            }
+        }
+    }
+#pragma unroll
+    for (int m = 0; m < 16; ++m) {
+        v[m].x = fmaf(v[m].x, bc.x, bc.y); v[m].y = fmaf(v[m].y, bc.x, bc.y);
+        v[m].z = fmaf(v[m].z, bc.x, bc.y); v[m].w = fmaf(v[m].w, bc.x, bc.y);
+    }
+#pragma unroll
+    for (int m = 0; m < 16; ++m) v[m] = stages01(v[m]);
+#pragma unroll
+    for (int t = 0; t < 3; ++t) {
+#pragma unroll
+        for (int m = 0; m < 16; ++m)
+            if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
+    }
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+        float4 *row = tile + (r0 + 32 * g) * 8;
+#pragma unroll
+        for (int m = 0; m < 8; ++m) row[m ^ x] = v[8 * g + m];
+    }
+}
+
 // Round on row bits 0..3: thread (rg = tid >> 3, cc = tid & 7) owns chunk cc of rows
 // 16 rg + m.  Serves pass A (second round) and the first round of a k = 20 pass-B tile, whose
 // two 128-row halves are simply rows 0..255.
@@ -770,6 +930,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
 {
     constexpr bool kFused = MODE == kCompressF32Fused;
     constexpr bool kEF = MODE == kErrorFeedback;
+    constexpr bool kAgg = MODE == kAggDecompress;      // sums of table values formed in pass A
     constexpr bool kRange = MODE == kRangeF32;       // pass A as compress, epilogue = min / max
     constexpr bool kF32In = MODE == kCompressF32 || kFused || kRange;
     constexpr bool kCompress = kF32In || MODE == kCompressBF16;
@@ -808,7 +969,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
     // error feedback: table values as floats, one copy per lane (8 copies for 8-bit indices)
     constexpr int kFRep = BITS <= 4 ? 32 : 8;
     float *ftab = reinterpret_cast<float *>(lut);
-    if (kEF) {
+    if (kEF || kAgg) {
         for (int idx = tid; idx < (1 << BITS) * kFRep; idx += kPCtaThreads)
             ftab[idx] = (float)P.dev->table[idx / kFRep];
     }
@@ -946,12 +1107,15 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                         const uint32_t in_bits = MODE == kCompressBF16 ? 16u : MODE == kDecompress8 ? 8u
                                                  : MODE == kDecompress16 ? 16u : MODE == kDecompress32 ? 32u
                                                  : (uint32_t)BITS;
-                        const unsigned char *src = static_cast<const unsigned char *>(in.p[kEF || kCompress ? wl : 0]);
                         const uint64_t first = j0 * in_bits / 8;
                         const uint64_t limit = (MODE == kCompressBF16 ? P.d : P.d_pad) * in_bits / 8;
                         const uint32_t lines = (uint32_t)kPElems * in_bits / 8 / 128;
-                        for (uint32_t l = (uint32_t)lane; l < lines; l += 32u)
-                            if (first + 128ull * l < limit) prefetch_l2(src + first + 128ull * l);
+                        const uint32_t sources = kAgg ? P.agg_n : 1u;
+                        for (uint32_t si = 0; si < sources; ++si) {
+                            const unsigned char *src = static_cast<const unsigned char *>(in.p[kAgg ? si : (kEF || kCompress ? wl : 0)]);
+                            for (uint32_t l = (uint32_t)lane; l < lines; l += 32u)
+                                if (first + 128ull * l < limit) prefetch_l2(src + first + 128ull * l);
+                        }
                     }
                     if (kCompress) {
                         // sign words of the tile (64 Philox calls, two per lane), while the copy is in flight
@@ -1117,6 +1281,17 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
             }
         };
 
+        // kAggDecompress with 4-bit indices and table values below 128: the table as 16 bytes
+        uint32_t agg_tb[4] = {0u, 0u, 0u, 0u};
+        uint32_t agg_chunk = 0;
+        if (kAgg && BITS == 4 && P.granularity < 128u) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                agg_tb[q] = P.dev->table[4 * q] | (P.dev->table[4 * q + 1] << 8) | (P.dev->table[4 * q + 2] << 16) |
+                            (P.dev->table[4 * q + 3] << 24);
+            agg_chunk = 255u / P.granularity;
+        }
+        (void)agg_tb; (void)agg_chunk;
         bar_sync(1, kPCtaThreads);
         TaskInfo me = s_info[0];
         fence_proxy_async();
@@ -1162,6 +1337,11 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                         pass_a_round1<true, false>(tile, sw + 256 * cur, tid);
                 } else if constexpr (kCompress) {
                     sq = pass_a_round1<true, kFused>(tile, sw + 256 * cur, tid);
+                } else if constexpr (kAgg) {
+                    const size_t coord = r * B + ((uint64_t)idx << kPLog2);
+                    pass_a_round1_aggregate<BITS, kFRep>(tile, in, P.agg_n, coord * BITS / 8, bc,
+                                                         ftab + (tid & (kFRep - 1)), outp.p[1], coord, P.agg_acc_bits, tid,
+                                                         agg_tb, agg_chunk);
                 } else {
                     constexpr int kInBits = MODE == kDecompress8 ? 8 : MODE == kDecompress16 ? 16
                                             : MODE == kDecompress32 ? 32 : BITS;

@@ -77,6 +77,10 @@ class Round:
         self.ctx.decompress(self.total, self.n, self.d, rnd, self.scales, self.out,
                             self.workspace, stream)
 
+    def aggregate_decompress(self, rnd: int = 0, want_sums: bool = False, stream=None):
+        self.ctx.aggregate_decompress(self.packed, self.d, rnd, self.scales, self.out, self.workspace,
+                                      total=self.total if want_sums else None, stream=stream)
+
     def run(self, rnd: int = 0, with_prepare: bool = True, stream=None, fused: bool = False):
         if with_prepare and fused:
             self.prepare_compress(rnd, stream)

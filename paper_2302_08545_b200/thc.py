@@ -20,7 +20,7 @@ THC_MAX_WORKERS = 64
 STATUS_NONFINITE, STATUS_ZERO_BLOCK, STATUS_WAIT_TIMEOUT = 1, 2, 4
 
 EXPORTS = ("thc_create", "thc_destroy", "thc_sizes", "thc_prepare", "thc_compress",
-           "thc_quantize_rotated", "thc_aggregate", "thc_decompress", "thc_prepare_noalloc",
+           "thc_quantize_rotated", "thc_aggregate", "thc_decompress", "thc_aggregate_decompress", "thc_prepare_noalloc",
            "thc_error_feedback", "thc_accumulate_error", "thc_prepare_compress", "thc_prepare_minmax", "thc_debug_skip_tasks", "thc_status", "thc_strerror", "thc_version")
 NOALLOC_SCRATCH_BYTES = 4 << 20
 
@@ -79,6 +79,7 @@ def lib():
     L.thc_quantize_rotated.argtypes = [vp, pp, u32, u32, u64, u32, vp, pp, vp]
     L.thc_aggregate.argtypes = [vp, pp, u32, u64, vp, vp]
     L.thc_decompress.argtypes = [vp, vp, u32, u64, u32, vp, vp, vp, u64, vp]
+    L.thc_aggregate_decompress.argtypes = [vp, pp, u32, u64, u32, vp, vp, vp, vp, u64, vp]
     L.thc_prepare_noalloc.argtypes = [pp, u32, u64, u32, u32, ctypes.c_double, vp, vp, vp]
     L.thc_prepare_minmax.argtypes = [vp, pp, u32, u64, u32, vp, pp, vp, u64, vp]
     L.thc_prepare_compress.argtypes = [vp, pp, u32, u32, u64, u32, vp, pp, pp, vp, u64, vp]
@@ -230,6 +231,14 @@ class Context:
         ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
         _check(lib().thc_decompress(self._h, _dp(total), divisor, d, rnd, _dp(scales), _dp(out),
                                     _dp(workspace), ws_bytes, _stream(stream)), "thc_decompress")
+
+    def aggregate_decompress(self, packed, d: int, rnd: int, scales, out, workspace, total=None,
+                             stream=None):
+        pa = _ptr_array([_dp(p) for p in packed])
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        _check(lib().thc_aggregate_decompress(self._h, pa, len(packed), d, rnd, _dp(scales), _dp(out),
+                                              _dp(total), _dp(workspace), ws_bytes, _stream(stream)),
+               "thc_aggregate_decompress")
 
     def error_feedback(self, grads, packed, d: int, rnd: int, scales, ef, workspace, stream=None):
         ga = _ptr_array([_dp(g) for g in grads])

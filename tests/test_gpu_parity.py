@@ -622,3 +622,55 @@ def test_exact_range_with_rotated_output_needs_one_transform(k, d, n):
         assert np.array_equal(one_pass[i], r.packed[i].cpu().numpy())
         assert np.array_equal(rot[i].view(np.uint32), O.rht_forward(x[i], c, 6).view(np.uint32))
     assert ctx.status() == 0
+
+
+@pytest.mark.parametrize("bits,g,table,n,k,d", [
+    (4, 30, T4_30, 8, 20, (1 << 21) + 777),              # one launch, 8-bit sums
+    (4, 30, T4_30, 17, 16, 3 * (1 << 16) + 5),           # 16-bit sums, run-time geometry
+    (3, 20, (0, 1, 5, 8, 10, 13, 17, 20), 5, 20, 1 << 20),
+    (2, 3, (0, 1, 2, 3), 64, 15, (1 << 17) + 1),
+    (1, 200, (0, 200), 3, 20, (1 << 20) + 12345),        # 3 * 200 = 600: 16-bit sums
+    (8, 255, tuple(range(256)), 64, 20, 1 << 20),        # 64 * 255: 16-bit sums
+    (8, 255, tuple(range(256)), 2, 18, 1 << 19),
+    (4, 30, T4_30, 6, 10, 33_001),                       # small blocks: the composed form
+])
+@pytest.mark.parametrize("want_sums", [False, True])
+def test_aggregate_decompress_in_one_call(bits, g, table, n, k, d, want_sums):
+    """thc_aggregate_decompress (Algorithm 2's PS line feeding the estimate line and the inverse
+    RHT in one launch) on uniformly random packed indices: the output equals, bit for bit, the
+    oracle's decompression of the oracle's sums and the library's two separate calls; the sums,
+    when asked for, equal the oracle's."""
+    import torch
+    from paper_2302_08545_b200 import runner
+    w = _mk(n, d, k, bits=bits, g=g, table=table)
+    ctx = runner.context_for(w)
+    r = runner.Round(ctx, n, d, "f32")
+    rng = np.random.default_rng(7000 + 10 * bits + n + k)
+    packed = rng.integers(0, 256, size=(n, r.sz.packed_bytes), dtype=np.uint8)
+    for i in range(n):
+        r.packed[i].copy_(torch.from_numpy(packed[i]))
+    nblk = r.sz.nblocks
+    scl = (0.5 + rng.random(nblk)).astype(np.float32)
+    if nblk > 1:
+        scl[nblk - 1] = 0.0                               # a degenerate block decodes to zeros
+    r.scales.copy_(torch.from_numpy(scl))
+    r.total.fill_(0xAB)
+    r.aggregate_decompress(rnd=3, want_sums=want_sums)
+    torch.cuda.synchronize()
+    fused_out = r.out.cpu().numpy().copy()
+    c = _ocfg(w)
+    ref_sum = O.aggregate(packed, r.sz.d_pad, c, r.sz.acc_bits)
+    ref_out = O.decompress(ref_sum, n, d, scl, c, 3)
+    assert np.array_equal(fused_out.view(np.uint32), ref_out.view(np.uint32))
+    dt = {8: np.uint8, 16: np.uint16, 32: np.uint32}[r.sz.acc_bits]
+    got_sum = r.total.cpu().numpy().view(dt)
+    if want_sums:
+        assert np.array_equal(got_sum, ref_sum)
+    elif k > 14:
+        assert np.all(r.total.cpu().numpy() == 0xAB)      # not asked for: not written
+    r.out.zero_()
+    r.aggregate()
+    r.decompress(3)
+    torch.cuda.synchronize()
+    assert np.array_equal(r.out.cpu().numpy().view(np.uint32), fused_out.view(np.uint32))
+    assert ctx.status() in (0, 2)

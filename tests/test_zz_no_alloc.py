@@ -1,12 +1,13 @@
 """thc_prepare_noalloc: the entry point for callers that may not allocate device memory (it
 keeps its scratch in a fixed array inside the library instead of a caller workspace and
-needs no context).  Checked through the C ABI against thc_prepare on the same inputs, on two
-calls in a row with different data: the shared scratch keeps the first call's contents, and
+needs no context).  Checked through the C ABI against thc_prepare and against the CPU oracle
+on the same inputs, on two calls in a row with different data: the shared scratch keeps the first call's contents, and
 the second call must not be affected by them.  Collected last (file name) so that a failure
 here cannot hide the other GPU tests in a stop-at-first-failure run."""
 import numpy as np
 import pytest
 
+from oracle import oracle as O
 from paper_2302_08545_b200 import thc, workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -30,16 +31,26 @@ def test_noalloc_prepare_matches_prepare_twice_in_a_row(k, d, n, dtype):
     scales2 = torch.full_like(r.scales, -1.0)
     status = torch.zeros(1, dtype=torch.int32, device=r.device)
     code = thc.THC_BF16 if dtype == "bf16" else thc.THC_F32
+    cfg = O.Config(bits=4, granularity=30, table=tuple(W.TABLES[(4, 30)]), t_p=w.t_p, log2_block=k,
+                   seed=w.seed)
     for call in range(2):
         W.fill_torch(w, r.grads, seed_offset=call * 100)
         if call == 1:
             r.grads[0][: min(d, 1 << k)].zero_()          # changes the first block's winner
         r.prepare()
+        torch.cuda.synchronize()
+        held = torch.cuda.memory_allocated()
+        free_before = torch.cuda.mem_get_info()[0]
         thc.prepare_noalloc(r.grads, d, k, code, w.t_p, scales2, status=status)
         torch.cuda.synchronize()
+        if call == 1:                                     # the first call may load the module lazily
+            assert torch.cuda.memory_allocated() == held
+            assert torch.cuda.mem_get_info()[0] >= free_before
         a, b = r.scales.cpu().numpy(), scales2.cpu().numpy()
         assert np.all(b > 0)
-        assert _within_one_ulp(a, b), f"call {call}: scales differ"
+        assert _within_one_ulp(a, b), f"call {call}: scales differ from thc_prepare"
+        x = np.stack([g.float().cpu().numpy() for g in r.grads])
+        assert _within_one_ulp(O.scales(x, cfg), b), f"call {call}: scales differ from the oracle"
         assert int(status.item()) == 0
 
 
@@ -66,3 +77,6 @@ def test_noalloc_prepare_sets_status_and_rejects_oversized_inputs():
     assert e.value.code == thc.THC_EWORKSPACE
     with pytest.raises(thc.ThcError):
         thc.prepare_noalloc(g, d, 2, thc.THC_F32, 2.0, scales)
+    with pytest.raises(thc.ThcError) as e:                # a length whose padding would wrap
+        thc.prepare_noalloc([g[0].data_ptr(), g[1].data_ptr()], (1 << 64) - 5, 20, thc.THC_F32, 2.0, scales)
+    assert e.value.code == thc.THC_EINVAL
