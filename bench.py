@@ -35,17 +35,17 @@ from paper_2302_08545_b200 import workloads as W  # noqa: E402
 METRIC = "gradient GB/s per compress+aggregate+decompress round; % of HBM roofline"
 UNIT = "GB/s"
 KERNELS_PER_STEP = {"prepare": 2, "compress": 1, "prepare_compress": 1, "aggregate": 1, "decompress": 1}
-# DRAM bytes per (worker, padded coordinate) of the compress kernel and of its fused-scales
-# variant, measured with ncu on the d=2^24, n=4, b=4 sweep point
-# (profiles/thc_pipeline_kernel_sweep_d2p24_b4_n4.md); traffic grows in proportion to n*d_pad,
-# so a full launch is this times n*d_pad.
-NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.277}
-NCU_FUSED_DRAM_BYTES_PER_COORD = {("f32", 4): 6.227}
+# DRAM bytes per (worker, padded coordinate) of the compress kernel (n = 4, d = 2^24, b = 4) and of
+# its fused-scales variant (n = 8, d = 2^24, b = 4: its ring grows with n), measured with ncu
+# (profiles/thc_pipeline_kernel_d2p24_b4.md); traffic grows in proportion to n*d_pad, so a full
+# launch is this times n*d_pad.
+NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.308}
+NCU_FUSED_DRAM_BYTES_PER_COORD = {("f32", 4): 9.277}
 # Executed thread-instructions per (worker, padded coordinate) from the same captures
-# (smsp__inst_executed x 32 / coordinates): the kernel is bound by instruction issue and the
-# shared-memory pipe rather than by HBM, so the issue rate is reported beside the HBM fraction.
-NCU_COMPRESS_THREAD_INST_PER_COORD = {("f32", 4): 47.5}
-NCU_FUSED_THREAD_INST_PER_COORD = {("f32", 4): 50.7}
+# (smsp__inst_executed x 32 / coordinates): the kernel is bound by the shared-memory data pipe
+# and instruction issue rather than by HBM, so the issue rate is reported beside the HBM fraction.
+NCU_COMPRESS_THREAD_INST_PER_COORD = {("f32", 4): 45.8}
+NCU_FUSED_THREAD_INST_PER_COORD = {("f32", 4): 48.9}
 
 
 def pick_workload(name: str) -> W.Workload:
@@ -444,7 +444,7 @@ def run_gpu(args):
         lane_rate = inst * w.n * w.d_pad / (comp_ms * 1e-3)
         issue = {"thread_inst_per_coord": inst, "achieved_lane_inst_per_s": lane_rate,
                  "peak_lane_inst_per_s": lane_peak, "frac": lane_rate / lane_peak,
-                 "source": "ncu smsp__inst_executed on the d=2^24 n=4 b=4 sweep point; peak = SMs x 128 lanes x sampled SM clock"}
+                 "source": "ncu smsp__inst_executed on a d=2^24 b=4 case of the same kernel; peak = SMs x 128 lanes x sampled SM clock"}
     # `roofline` is the HBM view the metric is stated in, for the step's dominant kernel:
     # algorithmic bytes of one launch (every input read once, every output written once) over
     # its CUDA-event duration, against the measured copy rate.  `roofline.step` is the same for
@@ -465,7 +465,7 @@ def run_gpu(args):
         "peak_source": peak_src, "algorithmic_bytes_per_launch": ab["compress"],
         "ms_per_launch": comp_ms,
         "traffic": traffic,
-        "traffic_source": "ncu dram bytes on the d=2^24 n=4 b=4 sweep point, scaled by n*d_pad"
+        "traffic_source": "ncu dram bytes on a d=2^24 b=4 case of the same kernel (n=8 fused, n=4 plain), scaled by n*d_pad"
                           if traffic is not None else None,
         "step": {"algorithmic_bytes": step_bytes, "ms": ms,
                  "achieved": step_bytes / (ms * 1e-3) / 1e9, "unit": "GB/s",

@@ -172,9 +172,10 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
 /* thc_aggregate followed by thc_decompress as one call, for a caller that holds all n workers'
  * packed indices on this GPU (the simulated cluster): Algorithm 2's PS line, Y = sum_i T[Z_i],
  * feeding the worker's estimate line and the inverse RHT (Algorithm 3) directly.  For RHT blocks
- * above 2^14 coordinates this is one launch and the sums never travel through memory; they are
- * written (d_pad unsigned integers of acc_bits bits, as thc_aggregate writes them) only if
- * sum_or_null is given.  `out` is bit for bit what the two calls give with divisor n.  The paper's
+ * above 2^14 coordinates, 4-bit indices and table values below 128 this is one launch and the
+ * sums never travel through memory; they are written (d_pad unsigned integers of acc_bits bits,
+ * as thc_aggregate writes them) only if sum_or_null is given.  Elsewhere the call runs
+ * thc_aggregate and thc_decompress (sums in the workspace unless a buffer is given).  `out` is bit for bit what the two calls give with divisor n.  The paper's
  * PS is another machine, so the separate calls remain the general form.
  *   packed       host array of n device pointers (n <= thc_config.workers)
  *   out          device, d fp32, written

@@ -10,6 +10,7 @@
 #include "thc_device.cuh"
 
 #include <math.h>
+#include <mutex>
 #include <new>
 #include <stdio.h>
 #include <string.h>
@@ -794,6 +795,14 @@ struct thc_ctx {
     PhiloxKeys keys;
     uint32_t lut_rep;
     int sm_count;
+    // Encoded tensor maps of recent launches, keyed by what they describe: a training loop calls
+    // with the same buffers every step, and encoding up to n + 1 maps per call costs more host
+    // time than a small launch takes on the device.
+    struct MapEntry { const void *base; uint64_t cols, rows, pitch; uint32_t box_rows, box_cols, half; CUtensorMap map; };
+    static constexpr int kMapCache = 2 * (THC_MAX_WORKERS + 2);
+    mutable MapEntry map_cache[kMapCache];
+    mutable int map_cache_used, map_cache_next;
+    mutable std::mutex map_mutex;
 };
 
 static thread_local cudaError_t g_last_cuda = cudaSuccess;
@@ -874,6 +883,8 @@ int thc_create(const thc_config *cfg, thc_ctx **out)
     ctx->device = -1;
     ctx->dev = nullptr;
     ctx->sm_count = 148;
+    ctx->map_cache_used = 0;
+    ctx->map_cache_next = 0;
     uint32_t k0 = (uint32_t)cfg->seed, k1 = (uint32_t)(cfg->seed >> 32);
     for (int r = 0; r < 10; ++r) {
         ctx->keys.k[2 * r] = k0;
@@ -1097,11 +1108,11 @@ static size_t tile_smem_bytes(const thc_ctx *ctx, const TileGeom &g)
 }
 
 // cudaFuncSetAttribute is needed once per kernel and dynamic shared-memory size; remember
-// what has been set per (kernel, device); a larger request raises the recorded size.  Not
-// thread-safe: concurrent first calls from several host threads may both set the attribute,
-// which is harmless.
+// what has been set per (kernel, device); a larger request raises the recorded size.
 static int ensure_dynamic_smem(const void *kern, size_t smem)
 {
+    static std::mutex guard;
+    std::lock_guard<std::mutex> lock(guard);
     static const void *seen_kern[96];
     static size_t seen_size[96];
     static int seen_dev[96];
@@ -1166,7 +1177,9 @@ static pipe_kernel_t pick_pipe_kernel_kb(uint32_t bits, bool identity)
 {
     if constexpr (MODE == kRangeF32) {
         return thc_pipeline_kernel<MODE, 4, true, KB>;
-    } else if constexpr (MODE == kErrorFeedback || MODE == kAggDecompress) {
+    } else if constexpr (MODE == kAggDecompress) {
+        return thc_pipeline_kernel<MODE, 4, true, KB>;     // one launch only for 4-bit indices (see the entry point)
+    } else if constexpr (MODE == kErrorFeedback) {
         switch (bits) {
         case 1: return thc_pipeline_kernel<MODE, 1, true, KB>;
         case 2: return thc_pipeline_kernel<MODE, 2, true, KB>;
@@ -1191,6 +1204,12 @@ static pipe_kernel_t pick_pipe_kernel_kb(uint32_t bits, bool identity)
 template <int MODE>
 static pipe_kernel_t pick_pipe_kernel(uint32_t bits, bool identity, uint32_t k)
 {
+    if constexpr (MODE == kCompressF32 || MODE == kCompressBF16) {
+        // 2^21 and 2^22 (the largest configuration): the generic path with its geometry fixed at
+        // compile time
+        if (k == 21) return pick_pipe_kernel_kb<MODE, 8>(bits, identity);
+        if (k == 22) return pick_pipe_kernel_kb<MODE, 9>(bits, identity);
+    }
     return k == 20 ? pick_pipe_kernel_kb<MODE, 7>(bits, identity)
                    : pick_pipe_kernel_kb<MODE, 0>(bits, identity);
 }
@@ -1203,14 +1222,14 @@ typedef CUresult (*encode_tiled_t)(CUtensorMap *, CUtensorMapDataType, cuuint32_
 
 static encode_tiled_t get_encode_tiled()
 {
-    static encode_tiled_t fn = nullptr;
-    if (fn == nullptr) {
+    static const encode_tiled_t fn = []() -> encode_tiled_t {     // initialised once, thread-safe
         void *p = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
             q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<encode_tiled_t>(p);
-    }
+            return reinterpret_cast<encode_tiled_t>(p);
+        return nullptr;
+    }();
     return fn;
 }
 
@@ -1235,6 +1254,29 @@ static int encode_map(CUtensorMap *map, const void *base, uint64_t cols, uint64_
                            rows64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? THC_OK : THC_ECUDA;
+}
+
+// encode_map through the context's cache.
+static int cached_map(const thc_ctx *ctx, CUtensorMap *map, const void *base, uint64_t cols, uint64_t rows,
+                      uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols = 32u, bool half_words = false)
+{
+    std::lock_guard<std::mutex> lock(ctx->map_mutex);
+    for (int i = 0; i < ctx->map_cache_used; ++i) {
+        const thc_ctx::MapEntry &e = ctx->map_cache[i];
+        if (e.base == base && e.cols == cols && e.rows == rows && e.pitch == pitch_bytes && e.box_rows == box_rows &&
+            e.box_cols == box_cols && e.half == (half_words ? 1u : 0u)) {
+            *map = e.map;
+            return THC_OK;
+        }
+    }
+    const int rc = encode_map(map, base, cols, rows, pitch_bytes, box_rows, box_cols, half_words);
+    if (rc != THC_OK) return rc;
+    int slot = ctx->map_cache_used < thc_ctx::kMapCache ? ctx->map_cache_used++ : ctx->map_cache_next;
+    ctx->map_cache_next = (slot + 1) % thc_ctx::kMapCache;
+    thc_ctx::MapEntry &e = ctx->map_cache[slot];
+    e.base = base; e.cols = cols; e.rows = rows; e.pitch = pitch_bytes; e.box_rows = box_rows; e.box_cols = box_cols;
+    e.half = half_words ? 1u : 0u; e.map = *map;
+    return THC_OK;
 }
 
 static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress_f32,
@@ -1290,31 +1332,31 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
     memset(&maps, 0, sizeof maps);
     P.b_swz_mask = 7u;
     if (k == 20) {
-        const int rc = encode_map(&maps.ring, workspace, (uint64_t)kPElems,
+        const int rc = cached_map(ctx, &maps.ring, workspace, (uint64_t)kPElems,
                                   (uint64_t)pl.ring << (k - kPLog2), (uint64_t)kPElems * 4, 128u);
         if (rc != THC_OK) return rc;
     } else if (k == 22) {
         // panels of 512 rows x 16 columns: boxes of 16 x 256, 64-byte swizzle
-        const int rc = encode_map(&maps.ring, workspace, (uint64_t)kPElems,
+        const int rc = cached_map(ctx, &maps.ring, workspace, (uint64_t)kPElems,
                                   (uint64_t)pl.ring << (k - kPLog2), (uint64_t)kPElems * 4, 256u, 16u);
         if (rc != THC_OK) return rc;
         P.b_swz_mask = 3u;
         P.b_tma = 2u;
     } else if (k == 21) {
-        const int rc = encode_map(&maps.ring, workspace, (uint64_t)kPElems,
+        const int rc = cached_map(ctx, &maps.ring, workspace, (uint64_t)kPElems,
                                   (uint64_t)pl.ring << (k - kPLog2), (uint64_t)kPElems * 4, 256u);
         if (rc != THC_OK) return rc;
         P.b_tma = 1u;
     }
     if (compress_f32 && (d >> 5) >= 256) {
         for (uint32_t i = 0; i < n_local; ++i) {
-            const int rc = encode_map(&maps.in[i], in.p[i], 32u, d >> 5, 128u, 256u);
+            const int rc = cached_map(ctx, &maps.in[i], in.p[i], 32u, d >> 5, 128u, 256u);
             if (rc != THC_OK) return rc;
         }
     }
     if (compress_bf16 && (d >> 5) >= 256) {
         for (uint32_t i = 0; i < n_local; ++i) {
-            const int rc = encode_map(&maps.in[i], in.p[i], 32u, d >> 5, 64u, 256u, 32u, true);
+            const int rc = cached_map(ctx, &maps.in[i], in.p[i], 32u, d >> 5, 64u, 256u, 32u, true);
             if (rc != THC_OK) return rc;
         }
     }
@@ -1550,8 +1592,9 @@ int thc_aggregate_decompress(thc_ctx *ctx, const void *const *packed, uint32_t n
     if (outp == nullptr || scales == nullptr || !aligned16(outp)) return THC_EINVAL;
     if (sum_or_null != nullptr && !aligned16(sum_or_null)) return THC_EINVAL;
     const uint32_t k = ctx->cfg.log2_block;
-    if (k <= (uint32_t)kTileLog2) {
-        // small blocks: the two calls (the sums go to the caller's buffer or to the workspace)
+    if (k <= (uint32_t)kTileLog2 || ctx->cfg.bits != 4 || ctx->cfg.granularity >= 128) {
+        // small blocks, and index widths without the byte-lane look-up (there the one launch is
+        // slower than the two): the two calls; the sums go to the caller's buffer or to the workspace
         if (workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
         if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
         void *sum = sum_or_null != nullptr ? sum_or_null

@@ -560,12 +560,12 @@ __device__ __forceinline__ void pass_a_round1_inverse(float4 *tile, const unsign
 
 // First round of a pass-A tile of thc_aggregate_decompress: the PS line and the estimate line of
 // Algorithm 2 in one place.  The thread fetches the packed indices of its two rows from every
-// worker, adds up the table values (as floats: the sums stay below 2^24, so they are exact and
-// equal the integer sums thc_aggregate writes), optionally writes the sums, and goes on as
-// pass_a_round1_inverse does with v = m + Y (M - m)/(g n).
-template <int BITS, int FREP>
+// worker, adds up the table values (in byte lanes, then exactly in floats: the sums stay below
+// 2^24 and equal the integer sums thc_aggregate writes), optionally writes the sums, and goes on
+// as pass_a_round1_inverse does with v = m + Y (M - m)/(g n).  4-bit indices and table values
+// below 128 only (the host sends every other configuration through the two separate kernels).
 __device__ __forceinline__ void pass_a_round1_aggregate(float4 *tile, const PtrArrayP &in, uint32_t agg_n,
-                                                        size_t byte_off, float2 bc, const float *ft,
+                                                        size_t byte_off, float2 bc,
                                                         void *sum_out, size_t coord_off, uint32_t acc_bits, int tid,
                                                         const uint32_t (&tb)[4], uint32_t swar_chunk)
 {
@@ -574,7 +574,7 @@ __device__ __forceinline__ void pass_a_round1_aggregate(float4 *tile, const PtrA
     float4 v[16];
 #pragma unroll
     for (int m = 0; m < 16; ++m) v[m] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (BITS == 4 && swar_chunk != 0) {
+    {
         // 4-bit indices, table values below 128: four look-ups per byte-permute instruction and
         // sums in byte lanes (see aggregate_b4w8_kernel), `swar_chunk` workers at a time so that
         // no byte overflows; the byte sums are then widened exactly into the float accumulators.
@@ -616,43 +616,6 @@ __device__ __forceinline__ void pass_a_round1_aggregate(float4 *tile, const PtrA
                     v[8 * g + m].z += __uint_as_float(__byte_perm(wv, 0x4B000000u, 0x7442)) - 8388608.0f;
                     v[8 * g + m].w += __uint_as_float(__byte_perm(wv, 0x4B000000u, 0x7443)) - 8388608.0f;
                 }
-        }
-    } else
-#pragma unroll 1
-    for (uint32_t i = 0; i < agg_n; ++i) {
-        const unsigned char *src = static_cast<const unsigned char *>(in.p[i]) + byte_off;
-#pragma unroll
-        for (int g = 0; g < 2; ++g) {
-            const unsigned char *p = src + (size_t)(r0 + 32 * g) * (BITS * 4);
-            uint32_t w[BITS];
-            if constexpr (BITS >= 4) {
-#pragma unroll
-                for (int q = 0; q < BITS / 4; ++q) {
-                    const uint4 t4 = __ldg(reinterpret_cast<const uint4 *>(p) + q);
-                    w[4 * q] = t4.x; w[4 * q + 1] = t4.y; w[4 * q + 2] = t4.z; w[4 * q + 3] = t4.w;
-                }
-            } else if constexpr (BITS == 3) {
-                w[0] = __ldg(reinterpret_cast<const uint32_t *>(p));
-                w[1] = __ldg(reinterpret_cast<const uint32_t *>(p) + 1);
-                w[2] = __ldg(reinterpret_cast<const uint32_t *>(p) + 2);
-            } else if constexpr (BITS == 2) {
-                const uint2 t2 = __ldg(reinterpret_cast<const uint2 *>(p));
-                w[0] = t2.x; w[1] = t2.y;
-            } else {
-                w[0] = __ldg(reinterpret_cast<const uint32_t *>(p));
-            }
-#pragma unroll
-            for (int m = 0; m < 8; ++m) {
-                float sv[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int bit = (m * 4 + e) * BITS;
-                    const uint32_t nxt = w[((bit >> 5) + 1) < BITS ? (bit >> 5) + 1 : (bit >> 5)];
-                    const uint32_t val = __funnelshift_r(w[bit >> 5], nxt, bit & 31) & ((1u << BITS) - 1u);
-                    sv[e] = ft[val * FREP];
-                }
-                v[8 * g + m].x += sv[0]; v[8 * g + m].y += sv[1]; v[8 * g + m].z += sv[2]; v[8 * g + m].w += sv[3];
-            }
         }
     }
     if (sum_out != nullptr) {
@@ -956,7 +919,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
     const uint32_t T = 1u << kb;                      // tiles (= panels) per worker-block
     const uint64_t B = 1ull << P.k;
     const int ccl = 11 - kb;                          // log2 chunks per pass-B row
-    const int bmask = (int)P.b_swz_mask;              // swizzle of run-time-geometry pass-B tiles
+    const int bmask = KB == 9 ? 3 : KB == 8 ? 7 : (int)P.b_swz_mask;   // swizzle of the pass-B tiles of the generic path
     const uint64_t d_rows32 = P.d >> 5;               // whole 32-coordinate rows of a gradient
 
     if (tid == 0) {
@@ -969,7 +932,7 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
     // error feedback: table values as floats, one copy per lane (8 copies for 8-bit indices)
     constexpr int kFRep = BITS <= 4 ? 32 : 8;
     float *ftab = reinterpret_cast<float *>(lut);
-    if (kEF || kAgg) {
+    if (kEF) {
         for (int idx = tid; idx < (1 << BITS) * kFRep; idx += kPCtaThreads)
             ftab[idx] = (float)P.dev->table[idx / kFRep];
     }
@@ -1339,9 +1302,8 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     sq = pass_a_round1<true, kFused>(tile, sw + 256 * cur, tid);
                 } else if constexpr (kAgg) {
                     const size_t coord = r * B + ((uint64_t)idx << kPLog2);
-                    pass_a_round1_aggregate<BITS, kFRep>(tile, in, P.agg_n, coord * BITS / 8, bc,
-                                                         ftab + (tid & (kFRep - 1)), outp.p[1], coord, P.agg_acc_bits, tid,
-                                                         agg_tb, agg_chunk);
+                    pass_a_round1_aggregate(tile, in, P.agg_n, coord / 2, bc, outp.p[1], coord, P.agg_acc_bits, tid,
+                                            agg_tb, agg_chunk);
                 } else {
                     constexpr int kInBits = MODE == kDecompress8 ? 8 : MODE == kDecompress16 ? 16
                                             : MODE == kDecompress32 ? 32 : BITS;

@@ -666,8 +666,8 @@ def test_aggregate_decompress_in_one_call(bits, g, table, n, k, d, want_sums):
     got_sum = r.total.cpu().numpy().view(dt)
     if want_sums:
         assert np.array_equal(got_sum, ref_sum)
-    elif k > 14:
-        assert np.all(r.total.cpu().numpy() == 0xAB)      # not asked for: not written
+    elif k > 14 and bits == 4:
+        assert np.all(r.total.cpu().numpy() == 0xAB)      # one launch, sums not asked for: not written
     r.out.zero_()
     r.aggregate()
     r.decompress(3)
