@@ -1207,8 +1207,12 @@ static pipe_kernel_t pick_pipe_kernel(uint32_t bits, bool identity, uint32_t k)
     if constexpr (MODE == kCompressF32 || MODE == kCompressBF16) {
         // 2^21 and 2^22 (the largest configuration): the generic path with its geometry fixed at
         // compile time
-        if (k == 21) return pick_pipe_kernel_kb<MODE, 8>(bits, identity);
-        if (k == 22) return pick_pipe_kernel_kb<MODE, 9>(bits, identity);
+        // (4-bit indices only, the width of every benchmark configuration with such blocks: each
+        // further instantiation costs build time)
+        if (k == 21 && bits == 4)
+            return identity ? thc_pipeline_kernel<MODE, 4, true, 8> : thc_pipeline_kernel<MODE, 4, false, 8>;
+        if (k == 22 && bits == 4)
+            return identity ? thc_pipeline_kernel<MODE, 4, true, 9> : thc_pipeline_kernel<MODE, 4, false, 9>;
     }
     return k == 20 ? pick_pipe_kernel_kb<MODE, 7>(bits, identity)
                    : pick_pipe_kernel_kb<MODE, 0>(bits, identity);
