@@ -994,6 +994,14 @@ static bool plan_pipeline_fused(const thc_ctx *ctx, uint64_t nblocks, uint32_t n
     return true;
 }
 
+// Workspace a pipeline launch over `wb_count` worker-blocks really touches when it computes no
+// scales: the ring and, behind it, one word pair per block for the exact-range keys.
+static uint64_t pipeline_workspace_need(const thc_ctx *ctx, uint64_t nblocks, uint64_t wb_count)
+{
+    const PipePlan pl = plan_pipeline(ctx, wb_count);
+    return ((uint64_t)pl.ring << ctx->cfg.log2_block) * 4 + nblocks * 8;
+}
+
 int thc_sizes(const thc_ctx *ctx, uint64_t d, uint32_t n_local, thc_sizes_t *s)
 {
     if (ctx == nullptr || s == nullptr || d == 0 || n_local == 0 || n_local > THC_MAX_WORKERS)
@@ -1545,7 +1553,7 @@ int thc_decompress(thc_ctx *ctx, const void *sum, uint32_t divisor, uint64_t d, 
     const bool two_pass = k > (uint32_t)kTileLog2;
     if (two_pass) {
         if (workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
-        if (workspace_bytes < sz.workspace_bytes - round_up(sz.sum_bytes, 256)) return THC_EWORKSPACE;
+        if (workspace_bytes < pipeline_workspace_need(ctx, sz.nblocks, sz.nblocks)) return THC_EWORKSPACE;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     PtrArray in;
@@ -1599,16 +1607,22 @@ int thc_aggregate_decompress(thc_ctx *ctx, const void *const *packed, uint32_t n
     if (k <= (uint32_t)kTileLog2 || ctx->cfg.bits != 4 || ctx->cfg.granularity >= 128) {
         // small blocks, and index widths without the byte-lane look-up (there the one launch is
         // slower than the two): the two calls; the sums go to the caller's buffer or to the workspace
-        if (workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
-        if (workspace_bytes < sz.workspace_bytes) return THC_EWORKSPACE;
-        void *sum = sum_or_null != nullptr ? sum_or_null
-                  : static_cast<unsigned char *>(workspace) + (sz.workspace_bytes - round_up(sz.sum_bytes, 256));
+        // (without a buffer the sums take the end of the workspace; thc_decompress checks that what
+        // is left in front of them is enough for it)
+        uint64_t ws_for_decompress = workspace_bytes;
+        void *sum = sum_or_null;
+        if (sum == nullptr) {
+            if (workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
+            const uint64_t room = round_up(sz.sum_bytes, 256);
+            if (workspace_bytes < room) return THC_EWORKSPACE;
+            ws_for_decompress = (workspace_bytes - room) & ~(uint64_t)255;
+            sum = static_cast<unsigned char *>(workspace) + ws_for_decompress;
+        }
         if ((rc = thc_aggregate(ctx, packed, n, d, sum, stream)) != THC_OK) return rc;
-        return thc_decompress(ctx, sum, n, d, round, scales, outp, workspace,
-                              sz.workspace_bytes - round_up(sz.sum_bytes, 256), stream);
+        return thc_decompress(ctx, sum, n, d, round, scales, outp, workspace, ws_for_decompress, stream);
     }
     if (workspace == nullptr || !aligned16(workspace)) return THC_EINVAL;
-    if (workspace_bytes < sz.workspace_bytes - round_up(sz.sum_bytes, 256)) return THC_EWORKSPACE;
+    if (workspace_bytes < pipeline_workspace_need(ctx, sz.nblocks, sz.nblocks)) return THC_EWORKSPACE;
     PtrArrayP pin;
     MutPtrArrayP pout, prot;
     memset(&pin, 0, sizeof pin);

@@ -76,6 +76,26 @@ def check_full_size(w, blocks, rnd=0):
         out_got = r.out[lo:hi].cpu().numpy()
         err = np.abs(out_got.astype(np.float64) - out_ref.astype(np.float64)).max()
         assert err <= 1e-5 * float(scl[0]), f"block {blk}: output error {err}"
+    # the one-call tail (thc_aggregate_decompress) and the launch that also computes the scales
+    # (thc_prepare_compress), at this size: the same bits as the separate calls checked above
+    out_two_calls = r.out.clone()
+    sums_two_calls = r.total.clone()
+    r.out.zero_()
+    r.total.zero_()
+    r.aggregate_decompress(rnd, want_sums=True)
+    torch.cuda.synchronize()
+    assert torch.equal(r.out.view(torch.int32), out_two_calls.view(torch.int32))
+    assert torch.equal(r.total, sums_two_calls)
+    if r.sz.fused_scales:
+        packed_two_calls = [p.clone() for p in r.packed]
+        scales_two_calls = r.scales.clone()
+        r.prepare_compress(rnd)
+        torch.cuda.synchronize()
+        ulps = (r.scales.view(torch.int32) - scales_two_calls.view(torch.int32)).abs().max().item()
+        assert ulps <= 1
+        if ulps == 0:
+            assert all(torch.equal(a, b) for a, b in zip(r.packed, packed_two_calls))
+    assert ctx.status() == 0
     del r
     torch.cuda.empty_cache()
 
