@@ -1,6 +1,7 @@
 """Seeded random configurations (block size, length, workers, index width, table, accumulator
 width, round, range mode) through the whole path on the GPU, each compared with the oracle:
-scales or ranges, packed indices, sums, output and error feedback."""
+scales or ranges, packed indices, sums, output (from the two calls and from the one-call tail)
+and error feedback."""
 import numpy as np
 import pytest
 
@@ -79,6 +80,14 @@ def test_random_configuration(case):
     assert np.array_equal(total, O.aggregate(packed, r.sz.d_pad, c, r.sz.acc_bits)), p
     out_ref = O.decompress(total, w.n, w.d, hi, c, rnd, lo=lo)
     assert np.array_equal(r.out.cpu().numpy().view(np.uint32), out_ref.view(np.uint32)), p
+    # the same tail as one call (sums into a fresh buffer on odd cases, not written on even ones)
+    r.out.zero_()
+    r.total.fill_(0x5A)
+    r.aggregate_decompress(rnd, want_sums=bool(case & 1))
+    torch.cuda.synchronize()
+    assert np.array_equal(r.out.cpu().numpy().view(np.uint32), out_ref.view(np.uint32)), p
+    if case & 1:
+        assert np.array_equal(r.sum_numpy(), total), p
     for i in range(w.n):
         z = O.unpack(packed[i], r.sz.d_pad, w.bits)
         e = O.error_feedback(x[i], z, hi, c, rnd, lo=lo)
