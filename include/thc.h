@@ -9,7 +9,9 @@
  *     thc_decompress  Y/n -> real values -> inverse RHT
  * and around them: thc_prepare_compress (the first two in one launch), thc_prepare_minmax (the
  * exact range of Algorithm 1's preliminary stage instead of the norm-based one),
- * thc_quantize_rotated, thc_error_feedback / thc_accumulate_error (Algorithm 3's residual).
+ * thc_quantize_rotated, thc_error_feedback / thc_accumulate_error (Algorithm 3's residual),
+ * thc_aggregate_decompress (the last two in one launch, for a caller that holds every
+ * worker's indices on one GPU).
  *
  * Conventions shared by every call
  *   - "device" pointers are CUDA device addresses on the device that was current when the

@@ -28,8 +28,10 @@
 //
 // Modes: compress (fp32 or bf16 gradients in, packed indices out), the same with fused scales,
 // exact range (pass A as compress, the epilogue only takes min / max), decompress (sums of 8,
-// 16 or 32 bits in, fp32 out) and error feedback (a worker's own packed indices in,
-// x - RHT^-1(X) out).  The 2^20 block has a compile-time geometry (KB = 7).
+// 16 or 32 bits in, fp32 out), aggregate + decompress (all workers' 4-bit indices in, pass A
+// sums their table values in byte lanes before it transforms; the sums are written only on
+// request) and error feedback (a worker's own packed indices in, x - RHT^-1(X) out).  The 2^20
+// block has a compile-time geometry (KB = 7); 2^21 and 2^22 have one for 4-bit compress.
 //
 // Fused scales (kCompressF32Fused; Section 5.3 notes that the norm exchange can run beside the
 // RHT).  Pass A does not need the clamp bound M, only the epilogue of pass B does.  So every
