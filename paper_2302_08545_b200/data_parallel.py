@@ -18,6 +18,14 @@ Every slice lands in the rank's own memory (a plain collective) before a kernel 
 rank and round the exchanges move about d (b + w)/8 bytes each way instead of the 8 d of an
 fp32 ring all-reduce.
 
+PeerMemoryRound is the same round without the two data collectives, for the GPUs of one node:
+every rank's packed indices and sums live in buffers all ranks can address (CudaIpcPeers: CUDA
+IPC mappings, NVLink peer memory between GPUs), the thc_aggregate kernel of rank q loads range q
+of every worker's indices straight from the owners' memory (compute and transfer in one kernel,
+plain loads only), and q stores its sums into every rank's buffer.  Two stream-ordered fences
+per round (a one-element all-reduce each) replace the all-to-all and the all-gather; no kernel
+ever waits on another rank.
+
 The exchange logic takes the per-rank steps as an `ops` object, so that it can be exercised on
 CPU process groups; the only implementation in this package, CudaOps, calls the library.
 """
@@ -52,15 +60,18 @@ class CudaOps:
         self.ctx.prepare([grad], self.d, scales, self.workspace)
         return scales
 
-    def compress(self, grad, rnd: int, scales, worker: int):
-        packed = torch.empty(self.sz.packed_bytes, dtype=torch.uint8, device=self.device)
+    def compress(self, grad, rnd: int, scales, worker: int, out=None):
+        packed = out if out is not None else \
+            torch.empty(self.sz.packed_bytes, dtype=torch.uint8, device=self.device)
         self.ctx.compress([grad], self.d, rnd, scales, [packed], self.workspace, worker_base=worker)
         return packed
 
-    def aggregate(self, slices, coords: int):
-        """slices: n tensors of packed indices covering `coords` coordinates (whole blocks)."""
+    def aggregate(self, slices, coords: int, out=None):
+        """slices: n tensors of packed indices covering `coords` coordinates (whole blocks);
+        they may live in another rank's memory."""
         sz = self.ctx.sizes(coords, len(slices))
-        total = torch.empty(sz.sum_bytes, dtype=torch.uint8, device=self.device)
+        total = out if out is not None else torch.empty(sz.sum_bytes, dtype=torch.uint8, device=self.device)
+        assert total.numel() == sz.sum_bytes
         self.ctx.aggregate(slices, coords, total)
         return total
 
@@ -127,3 +138,86 @@ class DataParallelRound:
         # 6. estimate + inverse RHT with divisor n
         out = ops.decompress(total, world, rnd, scales)
         return out, scales, packed, total
+
+
+class CudaIpcPeers:
+    """Device buffers of this rank that every rank of the node can address.
+
+    share(nbytes) allocates nbytes on this rank's GPU, hands its CUDA IPC handle to the other
+    ranks of the group and returns one uint8 tensor per rank: the own buffer and the others'
+    mappings (peer memory over NVLink when the owners are other GPUs).  All GPUs of the node must
+    be visible to every process.  close() drops the mappings on all ranks before any owner
+    frees its buffer."""
+
+    def __init__(self, device, group=None):
+        self.device, self.group = device, group
+        self.world, self.rank = dist.get_world_size(group), dist.get_rank(group)
+        self._own, self._mapped = [], []
+
+    def share(self, nbytes: int):
+        local = torch.empty(max(nbytes, 1), dtype=torch.uint8, device=self.device)[:nbytes]
+        self._own.append(local)
+        if self.world == 1:
+            return [local]
+        from torch.multiprocessing.reductions import reduce_tensor
+        # one handle per reader: torch counts the readers of a shared CUDA block per handle
+        mine = [None if q == self.rank else reduce_tensor(local) for q in range(self.world)]
+        handles = [None] * self.world
+        dist.all_gather_object(handles, mine, group=self.group)
+        bufs = []
+        for q in range(self.world):
+            if q == self.rank:
+                bufs.append(local)
+            else:
+                fn, args = handles[q][self.rank]
+                bufs.append(fn(*args))
+        self._mapped.append([b for q, b in enumerate(bufs) if q != self.rank])
+        return bufs
+
+    def close(self):
+        if torch.cuda.is_available():
+            torch.cuda.synchronize()
+        self._mapped.clear()
+        if self.world > 1:
+            dist.barrier(group=self.group)
+        self._own.clear()
+
+
+class PeerMemoryRound(DataParallelRound):
+    """The round over buffers all ranks can address: `peers.share(nbytes)` returns one uint8
+    tensor per rank (index = owner).  The caller keeps `peers` and this object alive together
+    and drops this object (its views of the peers' buffers) before peers.close()."""
+
+    def __init__(self, ops, peers, d: int, log2_block: int, bits: int, acc_bits: int, group=None):
+        super().__init__(ops, d, log2_block, bits, acc_bits, group)
+        self.packed = peers.share(self._idx_bytes(self.nblocks))
+        self.total = peers.share(self._sum_bytes(self.nblocks))
+        self._token = torch.zeros(1, dtype=torch.int32, device=self.packed[self.rank].device)
+
+    def _fence(self):
+        """Everything every rank enqueued before its fence is complete before anything a rank
+        enqueues after it starts: a collective on the compute stream cannot finish anywhere
+        before every rank has reached it."""
+        dist.all_reduce(self._token, group=self.group)
+
+    def step(self, grad, rnd: int):
+        ops, world, rank = self.ops, self.world, self.rank
+        scales = ops.local_scales(grad)
+        dist.all_reduce(scales, op=dist.ReduceOp.MAX, group=self.group)
+        # own indices, into the buffer the other ranks read.  No rank still reads the previous
+        # round's: all aggregates were complete at that round's second fence.
+        ops.compress(grad, rnd, scales, rank, out=self.packed[rank])
+        self._fence()
+        first, mine = self.ranges[rank]
+        if mine > 0:
+            lo, hi = self._idx_bytes(first), self._idx_bytes(first + mine)
+            slo, shi = self._sum_bytes(first), self._sum_bytes(first + mine)
+            part = self.total[rank][slo:shi]
+            # the PS line on the own range: the kernel loads the n slices from their owners
+            ops.aggregate([self.packed[q][lo:hi] for q in range(world)], mine * self.block, out=part)
+            for q in range(world):                  # "receive Y", pushed
+                if q != rank:
+                    self.total[q][slo:shi].copy_(part, non_blocking=True)
+        self._fence()
+        out = ops.decompress(self.total[rank], world, rnd, scales)
+        return out, scales, self.packed[rank], self.total[rank]

@@ -1,6 +1,7 @@
 """The multi-GPU round (one worker per rank; all_reduce(max) of the scales, all-to-all of the
-packed indices, local PS aggregation of a block range, all-gather of the sums, local decompress)
-on CPU process groups.  The exchange logic of paper_2302_08545_b200.data_parallel is run by
+packed indices, local PS aggregation of a block range, all-gather of the sums, local decompress;
+and its peer-memory form, where the aggregate step reads the other ranks' buffers and pushes its
+sums into them between two fences) on CPU process groups.  The exchange logic of paper_2302_08545_b200.data_parallel is run by
 2, 3 and 4 gloo ranks whose per-rank steps are bound to the CPU oracle (the product binds them to
 the CUDA library only); every rank's result must equal the oracle's single-process round over
 all workers bit for bit: scales, the rank's own indices, the sums and the output."""
@@ -21,7 +22,7 @@ sys.path.insert(0, os.environ["THC_ROOT"])
 import numpy as np, torch
 import torch.distributed as dist
 from oracle import oracle as O
-from paper_2302_08545_b200.data_parallel import DataParallelRound
+from paper_2302_08545_b200.data_parallel import DataParallelRound, PeerMemoryRound
 
 dist.init_process_group("gloo")
 rank, world = dist.get_rank(), dist.get_world_size()
@@ -36,22 +37,38 @@ x = (np.random.default_rng(99).standard_normal((world, d)) * np.linspace(0.5, 2.
 class OracleOps:                                   # the four per-rank steps, on host tensors
     def local_scales(self, grad):
         return torch.from_numpy(O.scales(grad.numpy()[None, :], cfg))
-    def compress(self, grad, rnd, scales, worker):
+    def compress(self, grad, rnd, scales, worker, out=None):
         r = O.rht_forward(grad.numpy(), cfg, rnd)
-        return torch.from_numpy(O.pack(O.quantize(r, scales.numpy(), cfg, rnd, worker), 4))
-    def aggregate(self, slices, coords):
-        packed = np.stack([s.numpy() for s in slices])
-        return torch.from_numpy(O.aggregate(packed, coords, cfg, w).view(np.uint8).copy())
+        res = torch.from_numpy(O.pack(O.quantize(r, scales.numpy(), cfg, rnd, worker), 4))
+        return res if out is None else out.copy_(res)
+    def aggregate(self, slices, coords, out=None):
+        packed = np.stack([np.array(s.numpy()) for s in slices])
+        res = torch.from_numpy(O.aggregate(packed, coords, cfg, w).view(np.uint8).copy())
+        return res if out is None else out.copy_(res)
     def decompress(self, total, divisor, rnd, scales):
-        return torch.from_numpy(O.decompress(total.numpy().view(dt), divisor, d, scales.numpy(), cfg, rnd))
+        return torch.from_numpy(O.decompress(np.array(total.numpy()).view(dt), divisor, d, scales.numpy(), cfg, rnd))
 
-dp = DataParallelRound(OracleOps(), d, k, 4, w)
-out, scales, packed, total = dp.step(torch.from_numpy(x[rank].copy()), rnd)
-ref = O.thc_round(x, cfg, rnd)
-assert np.array_equal(scales.numpy().view(np.uint32), ref["scales"].view(np.uint32))
-assert np.array_equal(packed.numpy(), ref["packed"][rank])
-assert np.array_equal(total.numpy().view(dt), ref["sum"])
-assert np.array_equal(out.numpy().view(np.uint32), ref["out"].view(np.uint32))
+class FilePeers:                                   # buffers all ranks address: files mapped by every rank
+    count = 0
+    def share(self, nbytes):
+        name = os.path.join(os.environ["THC_OUT"], "buf%d_rank%%d.bin" % self.count)
+        self.count += 1
+        np.memmap(name % rank, dtype=np.uint8, mode="w+", shape=(nbytes,)).flush()
+        dist.barrier()
+        return [torch.from_numpy(np.memmap(name % q, dtype=np.uint8, mode="r+", shape=(nbytes,))) for q in range(world)]
+
+if os.environ["THC_MODE"] == "peer":
+    dp = PeerMemoryRound(OracleOps(), FilePeers(), d, k, 4, w)
+else:
+    dp = DataParallelRound(OracleOps(), d, k, 4, w)
+for rnd in (5, 6):                                 # the second round reuses the peer buffers
+    xr = (x * (1.0 + 0.25 * (rnd - 5))).astype(np.float32)
+    out, scales, packed, total = dp.step(torch.from_numpy(xr[rank].copy()), rnd)
+    ref = O.thc_round(xr, cfg, rnd)
+    assert np.array_equal(scales.numpy().view(np.uint32), ref["scales"].view(np.uint32))
+    assert np.array_equal(np.array(packed.numpy()), ref["packed"][rank])
+    assert np.array_equal(np.array(total.numpy()).view(dt), ref["sum"])
+    assert np.array_equal(out.numpy().view(np.uint32), ref["out"].view(np.uint32))
 dist.barrier()
 dist.destroy_process_group()
 open(os.path.join(os.environ["THC_OUT"], f"rank{rank}.ok"), "w").write("ok")
@@ -73,11 +90,13 @@ def test_block_ranges_cover_every_block_once():
             assert max(c for _, c in r) - min(c for _, c in r) <= 1 and r[0][1] == max(c for _, c in r)
 
 
+@pytest.mark.parametrize("mode", ["collective", "peer"])
 @pytest.mark.parametrize("world", [2, 3, 4])
-def test_round_across_gloo_ranks_equals_the_single_process_round(tmp_path, world):
+def test_round_across_gloo_ranks_equals_the_single_process_round(tmp_path, world, mode):
     script = tmp_path / "worker.py"
     script.write_text(WORKER)
-    env = dict(os.environ, THC_ROOT=ROOT, THC_OUT=str(tmp_path), MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="1")
+    env = dict(os.environ, THC_ROOT=ROOT, THC_OUT=str(tmp_path), THC_MODE=mode, MASTER_ADDR="127.0.0.1",
+               OMP_NUM_THREADS="1")
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={world}",
            "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), str(script)]
     res = subprocess.run(cmd, capture_output=True, text=True, env=env, timeout=300)
