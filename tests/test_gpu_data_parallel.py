@@ -1,7 +1,9 @@
 """The multi-GPU round with its product binding (CUDA library + NCCL) at world size 1, the only
-size a single GPU allows: every collective of the round runs (on one rank they copy), and the
-result must equal the plain single-process round on the same gradient bit for bit.  The
-exchange logic at world sizes 2 to 4 is covered on CPU in test_data_parallel.py."""
+size NCCL allows on a single GPU: every collective of the round runs (on one rank they copy),
+and the result must equal the plain single-process round on the same gradient bit for bit.  The
+peer-memory form also runs as 2 and 3 processes on the one GPU (CUDA IPC mappings between them,
+gloo for the fences) against the oracle.  The exchange logic at world sizes 2 to 4 is covered
+on CPU in test_data_parallel.py."""
 import os
 import socket
 
