@@ -48,37 +48,44 @@ def block_ranges(nblocks: int, world: int):
 
 
 class CudaOps:
-    """The per-rank steps on the rank's GPU through the C ABI (thc.Context)."""
+    """The per-rank steps on the rank's GPU through the C ABI (thc.Context).  Buffers are
+    allocated once: what a step returns is overwritten by the same step of the next round."""
 
     def __init__(self, ctx, d: int, device):
         self.ctx, self.d, self.device = ctx, d, device
         self.sz = ctx.sizes(d, 1)
-        self.workspace = torch.empty(self.sz.workspace_bytes, dtype=torch.uint8, device=device)
+        u8 = dict(dtype=torch.uint8, device=device)
+        self.workspace = torch.empty(self.sz.workspace_bytes, **u8)
+        self.scales = torch.empty(self.sz.nblocks, dtype=torch.float32, device=device)
+        self.packed = torch.empty(self.sz.packed_bytes, **u8)
+        self.out = torch.empty(d, dtype=torch.float32, device=device)
+        self._part = {}
 
     def local_scales(self, grad):
-        scales = torch.empty(self.sz.nblocks, dtype=torch.float32, device=self.device)
-        self.ctx.prepare([grad], self.d, scales, self.workspace)
-        return scales
+        self.ctx.prepare([grad], self.d, self.scales, self.workspace)
+        return self.scales
 
     def compress(self, grad, rnd: int, scales, worker: int, out=None):
-        packed = out if out is not None else \
-            torch.empty(self.sz.packed_bytes, dtype=torch.uint8, device=self.device)
+        packed = out if out is not None else self.packed
         self.ctx.compress([grad], self.d, rnd, scales, [packed], self.workspace, worker_base=worker)
         return packed
 
     def aggregate(self, slices, coords: int, out=None):
         """slices: n tensors of packed indices covering `coords` coordinates (whole blocks);
         they may live in another rank's memory."""
-        sz = self.ctx.sizes(coords, len(slices))
-        total = out if out is not None else torch.empty(sz.sum_bytes, dtype=torch.uint8, device=self.device)
-        assert total.numel() == sz.sum_bytes
+        total = out
+        if total is None:
+            key = (coords, len(slices))
+            if key not in self._part:
+                self._part[key] = torch.empty(self.ctx.sizes(coords, len(slices)).sum_bytes,
+                                              dtype=torch.uint8, device=self.device)
+            total = self._part[key]
         self.ctx.aggregate(slices, coords, total)
         return total
 
     def decompress(self, total, divisor: int, rnd: int, scales):
-        out = torch.empty(self.d, dtype=torch.float32, device=self.device)
-        self.ctx.decompress(total, divisor, self.d, rnd, scales, out, self.workspace)
-        return out
+        self.ctx.decompress(total, divisor, self.d, rnd, scales, self.out, self.workspace)
+        return self.out
 
 
 class DataParallelRound:
@@ -98,6 +105,7 @@ class DataParallelRound:
         self.ranges = block_ranges(self.nblocks, self.world)
         if (self.block * bits) % 128 != 0 and self.world > 1:
             raise ValueError("slices of packed indices must start on 16-byte boundaries")
+        self._recv = self._padded = self._gathered = self._total = None
 
     def _idx_bytes(self, blocks: int) -> int:
         return blocks * self.block * self.bits // 8
@@ -105,36 +113,53 @@ class DataParallelRound:
     def _sum_bytes(self, blocks: int) -> int:
         return blocks * self.block * self.acc_bits // 8
 
+    def _buffers(self, like):
+        if self._recv is None:
+            u8 = dict(dtype=torch.uint8, device=like.device)
+            mine = self.ranges[self.rank][1]
+            longest = self._sum_bytes(self.ranges[0][1])
+            self._recv = torch.empty(self.world * self._idx_bytes(mine), **u8)
+            self._gathered = torch.empty(self.world * longest, **u8)
+            self._even = all(c == self.ranges[0][1] for _, c in self.ranges)
+            # ranges of equal length: the gathered sums are the sum buffer; else ranges are
+            # padded to the longest for the all-gather and copied out
+            self._padded = None if self._even else torch.zeros(longest, **u8)
+            self._total = self._gathered if self._even else torch.empty(self._sum_bytes(self.nblocks), **u8)
+        return self._recv, self._padded, self._gathered, self._total
+
     def step(self, grad, rnd: int):
         """Returns (out, scales, packed, total): the decompressed average and the intermediates
-        (for checks).  Collectives are issued on the current stream of the tensors' device."""
+        (for checks; buffers of this object and of `ops`, overwritten by the next step).
+        Collectives are issued on the current stream of the tensors' device."""
         ops, world, rank = self.ops, self.world, self.rank
         # 1. scales: max over workers of the per-worker M
         scales = ops.local_scales(grad)
         dist.all_reduce(scales, op=dist.ReduceOp.MAX, group=self.group)
         # 2. own indices
         packed = ops.compress(grad, rnd, scales, rank)
+        recv, padded, gathered, total = self._buffers(packed)
         # 3. all-to-all: range q of every worker goes to rank q
         in_splits = [self._idx_bytes(c) for (_, c) in self.ranges]
         mine = self.ranges[rank][1]
-        recv = torch.empty(world * self._idx_bytes(mine), dtype=torch.uint8, device=packed.device)
         out_splits = [self._idx_bytes(mine)] * world
         dist.all_to_all_single(recv, packed, output_split_sizes=out_splits, input_split_sizes=in_splits,
                                group=self.group)
-        # 4. the PS line on the own range
-        if mine > 0:
-            slices = list(recv.split(self._idx_bytes(mine)))
-            part = ops.aggregate(slices, mine * self.block)
-        else:
-            part = torch.empty(0, dtype=torch.uint8, device=packed.device)
-        # 5. all-gather of the sums (ranges may differ by one block: padded to the longest)
+        # 4. the PS line on the own range, 5. all-gather of the sums
         longest = self._sum_bytes(self.ranges[0][1])
-        padded = torch.zeros(longest, dtype=torch.uint8, device=packed.device)
-        padded[: part.numel()] = part
-        gathered = torch.empty(world * longest, dtype=torch.uint8, device=packed.device)
-        dist.all_gather_into_tensor(gathered, padded, group=self.group)
-        total = torch.cat([gathered[q * longest: q * longest + self._sum_bytes(c)]
-                           for q, (_, c) in enumerate(self.ranges)])
+        slices = list(recv.split(self._idx_bytes(mine))) if mine > 0 else []
+        if self._even:
+            part = gathered[rank * longest: (rank + 1) * longest]
+            ops.aggregate(slices, mine * self.block, out=part)
+            dist.all_gather_into_tensor(gathered, part, group=self.group)
+        else:
+            if mine > 0:
+                ops.aggregate(slices, mine * self.block, out=padded[: self._sum_bytes(mine)])
+            dist.all_gather_into_tensor(gathered, padded, group=self.group)
+            at = 0
+            for q, (_, c) in enumerate(self.ranges):
+                n = self._sum_bytes(c)
+                total[at: at + n].copy_(gathered[q * longest: q * longest + n])
+                at += n
         # 6. estimate + inverse RHT with divisor n
         out = ops.decompress(total, world, rnd, scales)
         return out, scales, packed, total

@@ -26,7 +26,8 @@ from paper_2302_08545_b200.data_parallel import DataParallelRound, PeerMemoryRou
 
 dist.init_process_group("gloo")
 rank, world = dist.get_rank(), dist.get_world_size()
-k, d, rnd = 8, 256 * 6 + 77, 5                     # 7 blocks: uneven ranges for 2, 3 and 4 ranks
+nblk = int(os.environ["THC_BLOCKS"])               # 7 blocks: uneven ranges for 2, 3 and 4 ranks; 8: even for 2 and 4
+k, d, rnd = 8, 256 * (nblk - 1) + 77, 5
 T = (0, 3, 5, 7, 9, 11, 13, 14, 15, 17, 19, 21, 23, 25, 27, 30)
 cfg = O.Config(bits=4, granularity=30, table=T, t_p=2.1538746940614564, log2_block=k,
                seed=0x0123456789ABCDEF)
@@ -90,13 +91,14 @@ def test_block_ranges_cover_every_block_once():
             assert max(c for _, c in r) - min(c for _, c in r) <= 1 and r[0][1] == max(c for _, c in r)
 
 
-@pytest.mark.parametrize("mode", ["collective", "peer"])
-@pytest.mark.parametrize("world", [2, 3, 4])
-def test_round_across_gloo_ranks_equals_the_single_process_round(tmp_path, world, mode):
+@pytest.mark.parametrize("world,blocks,mode", [(2, 7, "collective"), (3, 7, "collective"), (4, 7, "collective"),
+                                               (2, 8, "collective"), (4, 8, "collective"),
+                                               (2, 7, "peer"), (3, 7, "peer"), (4, 7, "peer")])
+def test_round_across_gloo_ranks_equals_the_single_process_round(tmp_path, world, blocks, mode):
     script = tmp_path / "worker.py"
     script.write_text(WORKER)
-    env = dict(os.environ, THC_ROOT=ROOT, THC_OUT=str(tmp_path), THC_MODE=mode, MASTER_ADDR="127.0.0.1",
-               OMP_NUM_THREADS="1")
+    env = dict(os.environ, THC_ROOT=ROOT, THC_OUT=str(tmp_path), THC_MODE=mode, THC_BLOCKS=str(blocks),
+               MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="1")
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={world}",
            "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), str(script)]
     res = subprocess.run(cmd, capture_output=True, text=True, env=env, timeout=300)
