@@ -1164,23 +1164,15 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                         tma = 1; phase = uses[s] & 1u; ++uses[s];
                     }
                 }
-                if (t.is_b && !kCompress && KB == 7) {
-                    // inverse transform: sign words of the panel's 128 rows x 64 columns (two
-                    // words per row), and for error feedback the x values the epilogue will read
+                if (t.is_b && kEF && KB == 7) {
+                    // error feedback: the x values the epilogue will read (128 rows x 64 columns)
                     const uint64_t j_panel = (uint64_t)r * B + ((uint64_t)t.idx << 6);
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        const int row = lane + 32 * c;
-                        const uint64_t jr = j_panel + ((uint64_t)row << kPLog2);
-                        const uint4 ph = sign_call(jr, P.round, keys);
-                        const bool hi = ((jr >> 5) & 3u) != 0;         // words 2,3 of the call
-                        sw[256 * s + 2 * row] = hi ? ph.z : ph.x;
-                        sw[256 * s + 2 * row + 1] = hi ? ph.w : ph.y;
-                        if (kEF) {
-                            const float *xr = static_cast<const float *>(rotated.p[t.wb - r * P.n_local]) + jr;
-                            if (jr < P.d) prefetch_l2(xr);
-                            if (jr + 32 < P.d) prefetch_l2(xr + 32);
-                        }
+                        const uint64_t jr = j_panel + ((uint64_t)(lane + 32 * c) << kPLog2);
+                        const float *xr = static_cast<const float *>(rotated.p[t.wb - r * P.n_local]) + jr;
+                        if (jr < P.d) prefetch_l2(xr);
+                        if (jr + 32 < P.d) prefetch_l2(xr + 32);
                     }
                 }
                 ti.tma = tma;
@@ -1344,6 +1336,16 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 }
                 const int e1 = kb < 4 ? kb : 4;
                 if (KB == 7) {
+                    if (!kCompress) {
+                        // inverse transform: sign words of the panel's 128 rows x 64 columns, two
+                        // words of one Philox call per row and thread; the epilogue reads them
+                        // after the block barrier below.  (Slot `cur` was last read two tasks ago.)
+                        const uint64_t jr = j_tile + ((uint64_t)tid << kPLog2);
+                        const uint4 ph = sign_call(jr, P.round, keys);
+                        const bool hi = ((jr >> 5) & 3u) != 0;         // words 2,3 of the call
+                        sw[256 * cur + 2 * tid] = hi ? ph.z : ph.x;
+                        sw[256 * cur + 2 * tid + 1] = hi ? ph.w : ph.y;
+                    }
                     round_rows_0_3(tile, tid);
                 } else {
                     switch (e1) {
