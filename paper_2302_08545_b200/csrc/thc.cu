@@ -798,7 +798,7 @@ struct thc_ctx {
     // Encoded tensor maps of recent launches, keyed by what they describe: a training loop calls
     // with the same buffers every step, and encoding up to n + 1 maps per call costs more host
     // time than a small launch takes on the device.
-    struct MapEntry { const void *base; uint64_t cols, rows, pitch; uint32_t box_rows, box_cols, half; CUtensorMap map; };
+    struct MapEntry { const void *base; uint64_t cols, rows, pitch; uint32_t box_rows, box_cols, half, groups; CUtensorMap map; };
     static constexpr int kMapCache = 2 * (THC_MAX_WORKERS + 2);
     mutable MapEntry map_cache[kMapCache];
     mutable int map_cache_used, map_cache_next;
@@ -1248,11 +1248,26 @@ static encode_tiled_t get_encode_tiled()
 // A 2-D map over `rows` rows of `cols` 32-bit words (row pitch in bytes), box box_cols x
 // box_rows (32 columns with the 128-byte swizzle, 16 with the 64-byte one).  The data type is
 // UINT32 so that bits travel unchanged.
+// With box_groups > 0 the rows are seen as cols / 32 groups of 32 words and the map is 3-D
+// (word in group, group, row) with a box of 32 x box_groups x box_rows: one copy then brings
+// box_rows rows of 32 * box_groups words each, and they land densely, row after row, in the
+// 128-byte swizzle (16-byte chunk c at c ^ ((c >> 3) & 7)).
 static int encode_map(CUtensorMap *map, const void *base, uint64_t cols, uint64_t rows,
-                      uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols = 32u, bool half_words = false)
+                      uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols = 32u, bool half_words = false,
+                      uint32_t box_groups = 0u)
 {
     encode_tiled_t enc = get_encode_tiled();
     if (enc == nullptr) return THC_ECUDA;
+    if (box_groups != 0u) {
+        const cuuint64_t dims3[3] = {32u, cols / 32u, rows};
+        const cuuint64_t strides3[2] = {128u, pitch_bytes};
+        const cuuint32_t box3[3] = {32u, box_groups, box_rows};
+        const cuuint32_t estr3[3] = {1u, 1u, 1u};
+        const CUresult r3 = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void *>(base), dims3, strides3,
+                                box3, estr3, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        return r3 == CUDA_SUCCESS ? THC_OK : THC_ECUDA;
+    }
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {pitch_bytes};
     const cuuint32_t box[2] = {box_cols, box_rows};
@@ -1270,24 +1285,25 @@ static int encode_map(CUtensorMap *map, const void *base, uint64_t cols, uint64_
 
 // encode_map through the context's cache.
 static int cached_map(const thc_ctx *ctx, CUtensorMap *map, const void *base, uint64_t cols, uint64_t rows,
-                      uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols = 32u, bool half_words = false)
+                      uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols = 32u, bool half_words = false,
+                      uint32_t box_groups = 0u)
 {
     std::lock_guard<std::mutex> lock(ctx->map_mutex);
     for (int i = 0; i < ctx->map_cache_used; ++i) {
         const thc_ctx::MapEntry &e = ctx->map_cache[i];
         if (e.base == base && e.cols == cols && e.rows == rows && e.pitch == pitch_bytes && e.box_rows == box_rows &&
-            e.box_cols == box_cols && e.half == (half_words ? 1u : 0u)) {
+            e.box_cols == box_cols && e.half == (half_words ? 1u : 0u) && e.groups == box_groups) {
             *map = e.map;
             return THC_OK;
         }
     }
-    const int rc = encode_map(map, base, cols, rows, pitch_bytes, box_rows, box_cols, half_words);
+    const int rc = encode_map(map, base, cols, rows, pitch_bytes, box_rows, box_cols, half_words, box_groups);
     if (rc != THC_OK) return rc;
     int slot = ctx->map_cache_used < thc_ctx::kMapCache ? ctx->map_cache_used++ : ctx->map_cache_next;
     ctx->map_cache_next = (slot + 1) % thc_ctx::kMapCache;
     thc_ctx::MapEntry &e = ctx->map_cache[slot];
     e.base = base; e.cols = cols; e.rows = rows; e.pitch = pitch_bytes; e.box_rows = box_rows; e.box_cols = box_cols;
-    e.half = half_words ? 1u : 0u; e.map = *map;
+    e.half = half_words ? 1u : 0u; e.groups = box_groups; e.map = *map;
     return THC_OK;
 }
 
@@ -1337,7 +1353,7 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
     const size_t smem = (size_t)1024 + (size_t)2 * kPElems * 4 + kPSignWords * 4 +
                         (size_t)(ctx->cfg.granularity + 1) * kLutEntryBytes + (size_t)nblk_cached * 8;
     { const int rc = ensure_dynamic_smem(reinterpret_cast<const void *>(kern), smem); if (rc != THC_OK) return rc; }
-    // Tensor maps: the ring (k = 20 panels are fetched by TMA) and, for fp32 compress, every
+    // Tensor maps: the ring (pass-B panels are fetched by TMA at every block size) and, for fp32 compress, every
     // worker's gradient viewed as rows of 32 floats (whole rows only; a ragged last tile is
     // loaded by the compute warps).
     TmaMaps maps;
@@ -1359,6 +1375,13 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
                                   (uint64_t)pl.ring << (k - kPLog2), (uint64_t)kPElems * 4, 256u);
         if (rc != THC_OK) return rc;
         P.b_tma = 1u;
+    } else {
+        // k = 15 .. 19: panels of 2^(k-13) rows x 2^(26-k) columns, one 3-D box each
+        const uint32_t kb = k - kPLog2;
+        const int rc = cached_map(ctx, &maps.ring, workspace, (uint64_t)kPElems,
+                                  (uint64_t)pl.ring << kb, (uint64_t)kPElems * 4, 1u << kb, 32u, false, 1u << (8u - kb));
+        if (rc != THC_OK) return rc;
+        P.b_tma = 3u;
     }
     if (compress_f32 && (d >> 5) >= 256) {
         for (uint32_t i = 0; i < n_local; ++i) {

@@ -112,7 +112,8 @@ struct PipeParams {
     uint32_t agg_n;            // kAggDecompress: workers whose table values are summed
     uint32_t agg_acc_bits;     // ... and the width of the sums written on request (outp.p[1])
     uint32_t b_tma;            // ... and are fetched by TMA in this many boxes of 256 rows (k = 21: one;
-                               // k = 22: two, 64-byte rows with the 64-byte swizzle); 0: by the compute warps
+                               // k = 22: two, 64-byte rows with the 64-byte swizzle); 3: k = 15 .. 19, one
+                               // 3-D box; 0: by the compute warps
 };
 
 struct PtrArrayP { const void *p[THC_MAX_WORKERS]; };
@@ -271,6 +272,18 @@ __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *m
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
                  ".L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
                  :: "r"(d), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(b), "l"(policy)
+                 : "memory");
+}
+
+// One 3-D tile: box of the tensor map at element coordinates (x, y, z) -> shared memory.
+__device__ __forceinline__ void tma_load_3d(void *smem_dst, const CUtensorMap *map, int x, int y, int z,
+                                            uint64_t *bar, uint64_t policy)
+{
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(bar);
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+                 ".L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+                 :: "r"(d), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(b), "l"(policy)
                  : "memory");
 }
 
@@ -1151,6 +1164,13 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                         const int y0 = (int)(t.slot << 7);
                         tma_load_2d(bufs[s], &maps.ring, x0, y0, &s_mbar[s], pol_ring);
                         tma_load_2d(bufs[s] + 1024, &maps.ring, x0 + 32, y0, &s_mbar[s], pol_ring);
+                        tma = 1; phase = uses[s] & 1u; ++uses[s];
+                    } else if (P.b_tma == 3u) {
+                        // k = 15 .. 19: 2^kb ring rows x 2^(13-kb) columns as one 3-D box
+                        // (word, group of 32 columns, row); it lands in the run-time layout
+                        mbar_expect_tx(&s_mbar[s], kPElems * 4);
+                        tma_load_3d(bufs[s], &maps.ring, 0, (int)(t.idx << (8 - kb)), (int)(t.slot << kb),
+                                    &s_mbar[s], pol_ring);
                         tma = 1; phase = uses[s] & 1u; ++uses[s];
                     } else if (P.b_tma) {
                         // k = 21: 256 ring rows x 32 columns, one box; k = 22: 512 rows x 16
