@@ -1323,6 +1323,9 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
     P.total_tasks = P.wb_count * T * 2;
     if (P.wb_count >= 0x7FFFFFFFull || P.total_tasks >= 0x7FFFFFFFull) return THC_EUNSUPPORTED;
     PipePlan pl = plan_pipeline(ctx, P.wb_count);
+    // Compress of 2^22 blocks: pass B trails by two worker-blocks in a ring of four slots
+    // (64 MB stay in L2 better than the planned six slots of 16 MB; the workspace holds those).
+    if ((compress_f32 || compress_bf16) && k == 22 && pl.ring > 4) { pl.lag = 2; pl.ring = 4; }
     if (fused_scales_out != nullptr) {
         if (!plan_pipeline_fused(ctx, sz.nblocks, n_local, &pl)) return THC_EUNSUPPORTED;
         P.tile_sq = reinterpret_cast<double *>(static_cast<unsigned char *>(workspace) +
