@@ -1325,6 +1325,8 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
     PipePlan pl = plan_pipeline(ctx, P.wb_count);
     // Compress of 2^22 blocks: pass B trails by two worker-blocks in a ring of four slots
     // (64 MB stay in L2 better than the planned six slots of 16 MB; the workspace holds those).
+    // The exact-range keys stay where the planned ring ends: thc_prepare_minmax looks there.
+    const uint32_t planned_ring = pl.ring;
     if ((compress_f32 || compress_bf16) && k == 22 && pl.ring > 4) { pl.lag = 2; pl.ring = 4; }
     if (fused_scales_out != nullptr) {
         if (!plan_pipeline_fused(ctx, sz.nblocks, n_local, &pl)) return THC_EUNSUPPORTED;
@@ -1351,7 +1353,7 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
     P.agg_n = agg_n;
     P.agg_acc_bits = ctx->acc_bits;
     P.range_keys = reinterpret_cast<uint32_t *>(static_cast<unsigned char *>(workspace) +
-                                                ((uint64_t)pl.ring << k) * 4);
+                                                ((uint64_t)planned_ring << k) * 4);
     const uint64_t nblk_cached = sz.nblocks < (uint64_t)kBlockConstMax ? sz.nblocks : (uint64_t)kBlockConstMax;
     const size_t smem = (size_t)1024 + (size_t)2 * kPElems * 4 + kPSignWords * 4 +
                         (size_t)(ctx->cfg.granularity + 1) * kLutEntryBytes + (size_t)nblk_cached * 8;

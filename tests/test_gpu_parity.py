@@ -386,7 +386,8 @@ def test_error_feedback_other_index_widths(bits, g):
         assert np.array_equal(ef[i].cpu().numpy().view(np.uint32), ref.view(np.uint32)), f"worker {i}"
 
 
-@pytest.mark.parametrize("k,d,n", [(5, 1000, 2), (10, 33_001, 3), (16, 150_000, 2), (20, (1 << 21) + 99, 2)])
+@pytest.mark.parametrize("k,d,n", [(5, 1000, 2), (10, 33_001, 3), (16, 150_000, 2), (20, (1 << 21) + 99, 2),
+                                   (22, (1 << 22) + 12_345, 3)])      # six worker-blocks: the compress ring is shorter than the planned one
 def test_exact_range_round_matches_oracle(k, d, n):
     """THC_RANGE_MINMAX contexts (Algorithm 1's preliminary stage on the rotated coordinates):
     the (min, max) planes equal the oracle's bit for bit (the rotated coordinates do), and so
