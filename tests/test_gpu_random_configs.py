@@ -35,7 +35,7 @@ def _random_case(rng):
                 exact=bool(rng.random() < 0.35), t_p=float(rng.choice([0.8, W.T_P["1/32"], 3.3])))
 
 
-@pytest.mark.parametrize("case", range(36))
+@pytest.mark.parametrize("case", range(96))
 def test_random_configuration(case):
     import torch
     from paper_2302_08545_b200 import runner
