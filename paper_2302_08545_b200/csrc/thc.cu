@@ -1025,7 +1025,8 @@ int thc_sizes(const thc_ctx *ctx, uint64_t d, uint32_t n_local, thc_sizes_t *s)
         two_pass_ws = (uint64_t)pl.ring * B * 4 + s->nblocks * 8;       // + range keys
         PipePlan pf;
         if (plan_pipeline_fused(ctx, s->nblocks, n_local, &pf)) {
-            const uint64_t fused_ws = (uint64_t)pf.ring * B * 4 + s->nblocks * n_local * (B >> kPLog2) * 8;
+            const uint64_t fused_ws = (uint64_t)pf.ring * B * 4 + s->nblocks * n_local * (B >> kPLog2) * 8 +
+                                      s->nblocks * 8;       // ring, tile sums, per-block quantiser constants
             if (fused_ws > two_pass_ws) two_pass_ws = fused_ws;
             s->fused_scales = 1;
         }
@@ -1332,6 +1333,7 @@ static int launch_pipeline(const thc_ctx *ctx, pipe_kernel_t kern, bool compress
         if (!plan_pipeline_fused(ctx, sz.nblocks, n_local, &pl)) return THC_EUNSUPPORTED;
         P.tile_sq = reinterpret_cast<double *>(static_cast<unsigned char *>(workspace) +
                                                ((uint64_t)pl.ring << k) * 4);
+        P.fused_const = reinterpret_cast<float2 *>(P.tile_sq + P.wb_count * T);
         P.scales_out = fused_scales_out;
         P.t_p = ctx->cfg.t_p;
     }

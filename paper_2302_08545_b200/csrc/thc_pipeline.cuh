@@ -104,6 +104,7 @@ struct PipeParams {
     // fused scales only
     double  *tile_sq;          // wb_count * T sums of squares, one per pass-A tile
     float   *scales_out;       // = scales, written by the kernel
+    float2  *fused_const;      // per block (kappa, offset) of the quantiser, written with M
     double   t_p;
     uint32_t exact_range;      // scales = nblocks minima then nblocks maxima (else M per block)
     uint32_t nblocks;
@@ -1028,6 +1029,11 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 if (!isfinite(M)) { M = 0.0f; flags |= THC_STATUS_NONFINITE; }
                 if (M == 0.0f) flags |= THC_STATUS_ZERO_BLOCK;
                 __stcg(P.scales_out + r, M);
+                // the quantiser's constants for the block's pass-B tasks (a division in fp64:
+                // done once here instead of once per task)
+                BlockRange br;
+                br.hi = M; br.lo = -M;
+                __stcg(P.fused_const + r, compress_constants(br));
                 if (flags) atomicOr(&P.dev->status, flags);
                 red_release_add(&pc->a_done[16u + (r & 15u)].v, 1u);
             }
@@ -1149,11 +1155,8 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                 pend_valid[s] = true;
                 if (lane == 0 && t.is_b) {
                     if (kFused) {
-                        BlockRange br;
-                        br.hi = ld_relaxed_f32(P.scales + r);
-                        br.lo = -br.hi;
-                        const float2 c = compress_constants(br);
-                        ti.bcx = c.x; ti.bcy = c.y;
+                        ti.bcx = ld_relaxed_f32(&P.fused_const[r].x);
+                        ti.bcy = ld_relaxed_f32(&P.fused_const[r].y);
                     }
                     // the ring was written through the generic proxy; the TMA unit reads it
                     fence_proxy_async_global();
