@@ -2,7 +2,7 @@
 must give the same scales, packed indices and output every time with no status flag (a late
 dependency, a lost completion signal or a buffer handed over too early would show here first),
 for the fused scales + compress launch, run-time and compile-time geometries, exact-range mode
-and the one-call tail."""
+and the one-call tail.  And two contexts driven from two host threads on two streams at once."""
 import pytest
 
 from paper_2302_08545_b200 import workloads as W
@@ -56,3 +56,52 @@ def test_repeated_rounds_are_identical(k, d, n, dtype, exact, iters):
         assert all(torch.equal(a, b) for a, b in zip(r.packed, ref_p)), f"indices, iteration {i}"
         assert torch.equal(r.out, ref_o), f"output, iteration {i}"
     assert ctx.status() == 0
+
+
+def test_two_contexts_on_two_host_threads_and_streams():
+    """Contexts are independent: two host threads, each with its own context, buffers and
+    stream, run rounds at the same time (the persistent kernels share the GPU); every round of
+    both must equal the one computed alone."""
+    import threading
+    import torch
+    from paper_2302_08545_b200 import runner
+    cases = [W.Workload("thr_a", n=3, d=3 * (1 << 20) + 11, log2_block=20, bits=4, granularity=30, table=T, data_seed=1),
+             W.Workload("thr_b", n=4, d=(1 << 21) + 7, log2_block=16, bits=4, granularity=30, table=T, data_seed=2)]
+    rounds, refs = [], []
+    for w in cases:
+        ctx = runner.context_for(w)
+        r = runner.Round(ctx, w.n, w.d)
+        W.fill_torch(w, r.grads)
+        r.run(7, fused=bool(r.sz.fused_scales))
+        torch.cuda.synchronize()
+        rounds.append((ctx, r))
+        refs.append(([p.clone() for p in r.packed], r.out.clone()))
+    errors = []
+
+    def worker(i):
+        try:
+            torch.cuda.set_device(0)
+            ctx, r = rounds[i]
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                for it in range(150):
+                    r.run(7, stream=stream, fused=bool(r.sz.fused_scales))
+                    if it % 10 == 9:
+                        stream.synchronize()
+                        ok = all(torch.equal(a, b) for a, b in zip(r.packed, refs[i][0])) and torch.equal(r.out, refs[i][1])
+                        if not ok:
+                            errors.append((i, it))
+                            return
+                stream.synchronize()
+            if ctx.status() != 0:
+                errors.append((i, "status", ctx.status()))
+        except Exception as e:                         # surfaced by the assert below
+            errors.append((i, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=300)
+    assert not any(t.is_alive() for t in threads)
+    assert errors == []
