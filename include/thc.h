@@ -27,6 +27,8 @@
  *     (a cudaStream_t passed as void*; NULL = the legacy default stream) and return without
  *     synchronising.  They allocate nothing.  Calls that share a context must be issued
  *     on one stream (or be ordered by the caller): they share the context's counters.
+ *     Different contexts are independent: they may be used from different host threads and
+ *     on different streams at the same time.
  *   - Return value: THC_OK or a negative THC_E* code; thc_strerror() gives text, and for
  *     THC_ECUDA the text of the CUDA error last seen by this thread's library calls.
  *   - Conditions met on the device never trap: they set bits that thc_status() reports.
