@@ -413,48 +413,41 @@ __device__ __forceinline__ double pass_a_round1(float4 *tile, const uint32_t *sw
 {
     const int x = tid & 7;
     const int r0 = ((tid >> 5) << 6) | (tid & 31);
-    float4 v[16];
-#pragma unroll
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    // The two rows are independent: a loop of two iterations instead of 16 chunks at once
+    // halves the code of this round (the kernel is large enough for instruction fetch to show).
+#pragma unroll 1
     for (int g = 0; g < 2; ++g) {
+        float4 v[8];
         float4 *row = tile + (r0 + 32 * g) * 8;
 #pragma unroll
-        for (int m = 0; m < 8; ++m) v[8 * g + m] = row[m ^ x];
-    }
-    double sq = 0.0;
-    if (SQ) {
-        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+        for (int m = 0; m < 8; ++m) v[m] = row[m ^ x];
+        if (SQ) {
 #pragma unroll
-        for (int m = 0; m < 16; ++m) {
-            a0 = fma((double)v[m].x, (double)v[m].x, a0);
-            a1 = fma((double)v[m].y, (double)v[m].y, a1);
-            a2 = fma((double)v[m].z, (double)v[m].z, a2);
-            a3 = fma((double)v[m].w, (double)v[m].w, a3);
+            for (int m = 0; m < 8; ++m) {
+                a0 = fma((double)v[m].x, (double)v[m].x, a0);
+                a1 = fma((double)v[m].y, (double)v[m].y, a1);
+                a2 = fma((double)v[m].z, (double)v[m].z, a2);
+                a3 = fma((double)v[m].w, (double)v[m].w, a3);
+            }
         }
-        sq = (a0 + a1) + (a2 + a3);
-    }
-    if (FLIP) {
-#pragma unroll
-        for (int g = 0; g < 2; ++g) {
+        if (FLIP) {
             const uint32_t w = sw[r0 + 32 * g];
 #pragma unroll
-            for (int m = 0; m < 8; ++m) v[8 * g + m] = flip4(v[8 * g + m], w >> (m * 4));
+            for (int m = 0; m < 8; ++m) v[m] = flip4(v[m], w >> (m * 4));
         }
+#pragma unroll
+        for (int m = 0; m < 8; ++m) v[m] = stages01(v[m]);
+#pragma unroll
+        for (int t = 0; t < 3; ++t) {
+#pragma unroll
+            for (int m = 0; m < 8; ++m)
+                if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
+        }
+#pragma unroll
+        for (int m = 0; m < 8; ++m) row[m ^ x] = v[m];
     }
-#pragma unroll
-    for (int m = 0; m < 16; ++m) v[m] = stages01(v[m]);
-#pragma unroll
-    for (int t = 0; t < 3; ++t) {
-#pragma unroll
-        for (int m = 0; m < 16; ++m)
-            if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
-    }
-#pragma unroll
-    for (int g = 0; g < 2; ++g) {
-        float4 *row = tile + (r0 + 32 * g) * 8;
-#pragma unroll
-        for (int m = 0; m < 8; ++m) row[m ^ x] = v[8 * g + m];
-    }
-    return sq;
+    return SQ ? (a0 + a1) + (a2 + a3) : 0.0;
 }
 
 // First round of a pass-A tile of a bf16 gradient that lies wholly inside the vector: the TMA
@@ -475,34 +468,34 @@ __device__ __forceinline__ void pass_a_round1_bf16(float4 *tile, const uint32_t 
         for (int q = 0; q < 4; ++q) raw[4 * g + q] = stage[row * 4 + (q ^ ((row >> 1) & 3))];
     }
     compute_barrier();
-    float4 v[16];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const uint4 t4 = raw[i];
-        v[2 * i] = make_float4(__uint_as_float(t4.x << 16), __uint_as_float(t4.x & 0xFFFF0000u),
-                               __uint_as_float(t4.y << 16), __uint_as_float(t4.y & 0xFFFF0000u));
-        v[2 * i + 1] = make_float4(__uint_as_float(t4.z << 16), __uint_as_float(t4.z & 0xFFFF0000u),
-                                   __uint_as_float(t4.w << 16), __uint_as_float(t4.w & 0xFFFF0000u));
-    }
-#pragma unroll
+    // one row per iteration (see pass_a_round1); the second row's staged words move down
+#pragma unroll 1
     for (int g = 0; g < 2; ++g) {
+        float4 v[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint4 t4 = raw[i];
+            v[2 * i] = make_float4(__uint_as_float(t4.x << 16), __uint_as_float(t4.x & 0xFFFF0000u),
+                                   __uint_as_float(t4.y << 16), __uint_as_float(t4.y & 0xFFFF0000u));
+            v[2 * i + 1] = make_float4(__uint_as_float(t4.z << 16), __uint_as_float(t4.z & 0xFFFF0000u),
+                                       __uint_as_float(t4.w << 16), __uint_as_float(t4.w & 0xFFFF0000u));
+        }
         const uint32_t w = sw[r0 + 32 * g];
 #pragma unroll
-        for (int m = 0; m < 8; ++m) v[8 * g + m] = flip4(v[8 * g + m], w >> (m * 4));
-    }
+        for (int m = 0; m < 8; ++m) v[m] = flip4(v[m], w >> (m * 4));
 #pragma unroll
-    for (int m = 0; m < 16; ++m) v[m] = stages01(v[m]);
+        for (int m = 0; m < 8; ++m) v[m] = stages01(v[m]);
 #pragma unroll
-    for (int t = 0; t < 3; ++t) {
+        for (int t = 0; t < 3; ++t) {
 #pragma unroll
-        for (int m = 0; m < 16; ++m)
-            if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
-    }
-#pragma unroll
-    for (int g = 0; g < 2; ++g) {
+            for (int m = 0; m < 8; ++m)
+                if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
+        }
         float4 *row = tile + (r0 + 32 * g) * 8;
 #pragma unroll
-        for (int m = 0; m < 8; ++m) row[m ^ x] = v[8 * g + m];
+        for (int m = 0; m < 8; ++m) row[m ^ x] = v[m];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) raw[i] = raw[i + 4];
     }
 }
 
@@ -519,27 +512,33 @@ __device__ __forceinline__ void pass_a_round1_inverse(float4 *tile, const unsign
                             : MODE == kDecompress32 ? 32 : BITS;
     const int x = tid & 7;
     const int r0 = ((tid >> 5) << 6) | (tid & 31);
-    float4 v[16];
+    // the words of both rows first (all loads in flight together), then one row per iteration
+    // (see pass_a_round1) with the second row's words moving down
+    uint32_t w[2 * IN_BITS];
 #pragma unroll
     for (int g = 0; g < 2; ++g) {
         const unsigned char *p = src + (size_t)(r0 + 32 * g) * (IN_BITS * 4);
-        uint32_t w[IN_BITS];
+        uint32_t *wg = w + g * IN_BITS;
         if constexpr (IN_BITS >= 4) {
 #pragma unroll
             for (int q = 0; q < IN_BITS / 4; ++q) {
                 const uint4 t4 = __ldg(reinterpret_cast<const uint4 *>(p) + q);
-                w[4 * q] = t4.x; w[4 * q + 1] = t4.y; w[4 * q + 2] = t4.z; w[4 * q + 3] = t4.w;
+                wg[4 * q] = t4.x; wg[4 * q + 1] = t4.y; wg[4 * q + 2] = t4.z; wg[4 * q + 3] = t4.w;
             }
         } else if constexpr (IN_BITS == 3) {
-            w[0] = __ldg(reinterpret_cast<const uint32_t *>(p));
-            w[1] = __ldg(reinterpret_cast<const uint32_t *>(p) + 1);
-            w[2] = __ldg(reinterpret_cast<const uint32_t *>(p) + 2);
+            wg[0] = __ldg(reinterpret_cast<const uint32_t *>(p));
+            wg[1] = __ldg(reinterpret_cast<const uint32_t *>(p) + 1);
+            wg[2] = __ldg(reinterpret_cast<const uint32_t *>(p) + 2);
         } else if constexpr (IN_BITS == 2) {
             const uint2 t2 = __ldg(reinterpret_cast<const uint2 *>(p));
-            w[0] = t2.x; w[1] = t2.y;
+            wg[0] = t2.x; wg[1] = t2.y;
         } else {
-            w[0] = __ldg(reinterpret_cast<const uint32_t *>(p));
+            wg[0] = __ldg(reinterpret_cast<const uint32_t *>(p));
         }
+    }
+#pragma unroll 1
+    for (int g = 0; g < 2; ++g) {
+        float4 v[8];
 #pragma unroll
         for (int m = 0; m < 8; ++m) {
             float sv[4];
@@ -555,22 +554,21 @@ __device__ __forceinline__ void pass_a_round1_inverse(float4 *tile, const unsign
                 else yf = __uint_as_float(0x4B000000u | val) - 8388608.0f;
                 sv[e] = fmaf(yf, bc.x, bc.y);
             }
-            v[8 * g + m] = make_float4(sv[0], sv[1], sv[2], sv[3]);
+            v[m] = make_float4(sv[0], sv[1], sv[2], sv[3]);
         }
-    }
 #pragma unroll
-    for (int m = 0; m < 16; ++m) v[m] = stages01(v[m]);
+        for (int m = 0; m < 8; ++m) v[m] = stages01(v[m]);
 #pragma unroll
-    for (int t = 0; t < 3; ++t) {
+        for (int t = 0; t < 3; ++t) {
 #pragma unroll
-        for (int m = 0; m < 16; ++m)
-            if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
-    }
-#pragma unroll
-    for (int g = 0; g < 2; ++g) {
+            for (int m = 0; m < 8; ++m)
+                if (!(m & (1 << t))) butterfly(v[m], v[m | (1 << t)]);
+        }
         float4 *row = tile + (r0 + 32 * g) * 8;
 #pragma unroll
-        for (int m = 0; m < 8; ++m) row[m ^ x] = v[8 * g + m];
+        for (int m = 0; m < 8; ++m) row[m ^ x] = v[m];
+#pragma unroll
+        for (int q = 0; q < IN_BITS; ++q) w[q] = w[q + IN_BITS];
     }
 }
 
