@@ -1331,8 +1331,23 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     if ((tid & 31) == 0) s_sq[cur][tid >> 5] = sq;
                 }
                 __syncwarp();                          // the next round stays inside the warp's rows
+            } else if (KB == 7 && !kCompress) {
+                // inverse transform, pass B: sign words of the panel's 128 rows x 64 columns, two
+                // words of one Philox call per row and thread; the epilogue reads them after the
+                // block barrier below.  (Slot `cur` was last read two tasks ago.)
+                const uint64_t jr = r * B + ((uint64_t)idx << (kPLog2 - kb)) + ((uint64_t)tid << kPLog2);
+                const uint4 ph = sign_call(jr, P.round, keys);
+                const bool hi = ((jr >> 5) & 3u) != 0;         // words 2,3 of the call
+                sw[256 * cur + 2 * tid] = hi ? ph.z : ph.x;
+                sw[256 * cur + 2 * tid + 1] = hi ? ph.w : ph.y;
+            }
+            // The round on row bits 0..3 is the second round of every pass-A tile and the first
+            // of a 2^20 block's pass-B panel: one copy of its code serves both.
+            if (KB == 7 || !is_b) {
                 round_rows_0_3(tile, tid);
                 compute_barrier();
+            }
+            if (!is_b) {
                 pass_a_round3_store(tile, P.ring + (size_t)slot * B + ((size_t)idx << kPLog2), tid);
             } else {
                 // ================================ pass B: panel idx of worker-block wb
@@ -1356,26 +1371,14 @@ thc_pipeline_kernel(const __grid_constant__ TmaMaps maps, PipeParams P, PtrArray
                     fill_sign_words(sw, g, j_tile, keys, tid, kPThreads);
                 }
                 const int e1 = kb < 4 ? kb : 4;
-                if (KB == 7) {
-                    if (!kCompress) {
-                        // inverse transform: sign words of the panel's 128 rows x 64 columns, two
-                        // words of one Philox call per row and thread; the epilogue reads them
-                        // after the block barrier below.  (Slot `cur` was last read two tasks ago.)
-                        const uint64_t jr = j_tile + ((uint64_t)tid << kPLog2);
-                        const uint4 ph = sign_call(jr, P.round, keys);
-                        const bool hi = ((jr >> 5) & 3u) != 0;         // words 2,3 of the call
-                        sw[256 * cur + 2 * tid] = hi ? ph.z : ph.x;
-                        sw[256 * cur + 2 * tid + 1] = hi ? ph.w : ph.y;
-                    }
-                    round_rows_0_3(tile, tid);
-                } else {
+                if (KB != 7) {
                     switch (e1) {
                     case 4: p_round<4>(tile, ccl, tid, bmask); break;
                     case 3: p_round<3>(tile, ccl, tid, bmask); break;
                     default: p_round<2>(tile, ccl, tid, bmask); break;
                     }
+                    compute_barrier();
                 }
-                compute_barrier();
                 uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
                 if (KB == 7) {
                     pass_b_last_round_kb7<kCompress, BITS, IDENTITY, kRange>(tile, tid, ep, keys, kmin, kmax);
