@@ -39,13 +39,13 @@ KERNELS_PER_STEP = {"prepare": 2, "compress": 1, "prepare_compress": 1, "aggrega
 # its fused-scales variant (n = 8, d = 2^24, b = 4: its ring grows with n), measured with ncu
 # (profiles/thc_pipeline_kernel_d2p24_b4.md); traffic grows in proportion to n*d_pad, so a full
 # launch is this times n*d_pad.
-NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.308}
-NCU_FUSED_DRAM_BYTES_PER_COORD = {("f32", 4): 9.277}
+NCU_COMPRESS_DRAM_BYTES_PER_COORD = {("f32", 4): 5.296}
+NCU_FUSED_DRAM_BYTES_PER_COORD = {("f32", 4): 9.206}
 # Executed thread-instructions per (worker, padded coordinate) from the same captures
 # (smsp__inst_executed x 32 / coordinates): the kernel is bound by the shared-memory data pipe
 # and instruction issue rather than by HBM, so the issue rate is reported beside the HBM fraction.
-NCU_COMPRESS_THREAD_INST_PER_COORD = {("f32", 4): 45.8}
-NCU_FUSED_THREAD_INST_PER_COORD = {("f32", 4): 48.9}
+NCU_COMPRESS_THREAD_INST_PER_COORD = {("f32", 4): 46.1}
+NCU_FUSED_THREAD_INST_PER_COORD = {("f32", 4): 49.0}
 
 
 def pick_workload(name: str) -> W.Workload:
