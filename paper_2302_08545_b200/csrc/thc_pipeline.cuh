@@ -844,11 +844,27 @@ __device__ __forceinline__ void pass_b_last_round(const float4 *tile, int kb, in
                     butterfly(b[m], b[m | (1 << t)]);
                 }
         }
+        if constexpr (N == 8) {
+            // eight rows: a loop of two iterations over four rows each, as in the 2^20 form
+            // (the second iteration's rows move down the register arrays): half the code
+#pragma unroll 1
+            for (int half = 0; half < 2; ++half) {
 #pragma unroll
-        for (int m = 0; m < N; ++m) {
-            const int row = row_low + (m << rl);
-            const uint64_t j = ep.j_tile + ((uint64_t)row << kPLog2) + 8 * uu;
-            epilogue_unit<COMPRESS, BITS, IDENTITY, RANGE>(a[m], b[m], j, row, uu, ep, keys, kmin, kmax);
+                for (int m = 0; m < 4; ++m) {
+                    const int row = row_low + ((4 * half + m) << rl);
+                    const uint64_t j = ep.j_tile + ((uint64_t)row << kPLog2) + 8 * uu;
+                    epilogue_unit<COMPRESS, BITS, IDENTITY, RANGE>(a[m], b[m], j, row, uu, ep, keys, kmin, kmax);
+                }
+#pragma unroll
+                for (int m = 0; m < 4; ++m) { a[m] = a[m + 4]; b[m] = b[m + 4]; }
+            }
+        } else {
+#pragma unroll
+            for (int m = 0; m < N; ++m) {
+                const int row = row_low + (m << rl);
+                const uint64_t j = ep.j_tile + ((uint64_t)row << kPLog2) + 8 * uu;
+                epilogue_unit<COMPRESS, BITS, IDENTITY, RANGE>(a[m], b[m], j, row, uu, ep, keys, kmin, kmax);
+            }
         }
     }
 }
